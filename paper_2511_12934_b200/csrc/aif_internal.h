@@ -1,0 +1,165 @@
+// Internal declarations of libaif: context layout, device-side descriptors, kernel launchers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <vector>
+
+#include "../../include/aif.h"
+
+namespace aif {
+
+constexpr int kMaxHidden = 4;
+constexpr int kSimtTile = 8;        // candidates per block in the CUDA-core scoring kernel
+constexpr int kSimtThreads = 256;
+constexpr int kTcTile = 128;        // candidates per tile in the tensor-core kernels (UMMA M)
+
+// One user-state slot as the kernels see it.  Pointers are fixed when the arena is laid out; only L changes.
+struct SlotDev {
+    const void *u;          // [d] storage type
+    const float *u32;       // [d] fp32
+    const void *S;          // [L x d] storage type: projected behaviour sequence
+    const void *T;          // [F x B x dc] storage type: cross pre-cache
+    const void *V;          // [n_bridge x d] storage type
+    const uint8_t *sigS;    // [L x lsh_bits/8]
+    const float *p_u;       // [H1] fp32: W1[:, user columns] u + b1
+    const void *smallB;     // [H1 x 16] bf16: per-request B operand of the narrow feature chunk (tensor path)
+    int32_t L;
+    int32_t pad_;
+};
+
+// One request of a scoring launch.
+struct ReqDev {
+    int32_t slot;
+    int32_t n;            // candidates
+    int64_t off;          // first candidate in ids / logits
+    int32_t tile_begin;   // first tile of this request in the launch
+    int32_t pad_;
+};
+
+struct ModelDev {
+    int32_t d, F, B, dc, n_hidden, hidden[kMaxHidden];
+    int32_t bucket_mode, blocks, n_bridge, lsh_bits, n_tiers, lsh_din_norm, simtier_norm, emit_sigmoid;
+    int32_t k1;           // candidate-dependent input columns = input width - d
+    int32_t mini_batch;
+    int64_t M;
+    const void *E;
+    const void *bea_w;
+    const uint8_t *sig;
+    const void *Wt[kMaxHidden];   // transposed weights [in x out] storage type; Wt[0] = full first layer incl. user rows
+    const float *b[kMaxHidden];
+    const void *w_out;
+    const float *b_out;
+};
+
+struct ScoreLaunch {
+    const SlotDev *slots;   // device array of all slots
+    const ReqDev *reqs;     // device array [n_req], or nullptr: use `single`
+    ReqDev single;
+    int32_t n_req;
+    int32_t n_tiles;
+    const int32_t *ids;
+    float *logits;
+    uint32_t *status;
+};
+
+struct HostSlot {
+    bool in_use = false;
+    bool ready = false;
+    int32_t L = 0;
+    uint64_t key = 0;
+    uint64_t model_version = 0;
+    cudaEvent_t ev = nullptr;
+    SlotDev dev{};
+    // scratch for the user-side network
+    float *prof_hat = nullptr;   // [d]
+    float *partial = nullptr;    // [kUserPartials x d]
+};
+
+constexpr int kUserPartials = 1184;   // warps of the self-attention launch (148 SMs x 8)
+
+struct PinnedRing {
+    static constexpr int kSlots = 8;
+    ReqDev *host[kSlots] = {};
+    ReqDev *dev[kSlots] = {};
+    cudaEvent_t ev[kSlots] = {};
+    bool used[kSlots] = {};
+    int next = 0;
+    int capacity = 0;   // requests per slot
+};
+
+}  // namespace aif
+
+struct aif_user_state {
+    aif_ctx *ctx;
+    int32_t index;
+};
+
+struct aif_ctx {
+    aif_config cfg;
+    int device = 0;
+    size_t el = 4;
+    int input_width = 0;
+    bool weights_loaded = false;
+    bool tensor_path = false;
+    uint64_t model_version = 0, table_version = 0;
+    int64_t device_bytes = 0;
+
+    void *E = nullptr;
+    void *bea_w = nullptr;
+    uint8_t *sig = nullptr;
+
+    // weights
+    void *Wt[aif::kMaxHidden] = {};      // [in x out]
+    void *Wk[aif::kMaxHidden] = {};      // [out x in] (K-major), first layer: candidate-dependent columns only, K padded
+    float *b[aif::kMaxHidden] = {};
+    void *w_out = nullptr;
+    float *b_out = nullptr;
+    void *Wprofile_t = nullptr, *Wseq_t = nullptr, *Wa_t = nullptr, *Wb_t = nullptr;
+    float *b_a = nullptr, *b_b = nullptr;
+    bool user_weights = false;
+
+    char *arena = nullptr;
+    size_t slot_bytes = 0;
+    aif::SlotDev *slots_dev = nullptr;
+    std::vector<aif::HostSlot> slots;
+    std::vector<aif_user_state> handles;
+    uint32_t *status = nullptr;
+
+    // scratch owned by the context
+    int32_t *ids_stage = nullptr;     // device staging of host ids (aif_score_host)
+    float *logits_stage = nullptr;
+    void *att_scratch = nullptr;      // [max_batch_candidates x d] bf16: attention output between the two tensor kernels
+    aif::PinnedRing ring;
+
+    aif_stats stats{};
+    std::vector<void *> allocations;
+};
+
+namespace aif {
+
+extern std::atomic<uint64_t> g_launches;
+inline void count_launch(int n = 1) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+ModelDev make_model(const aif_ctx *ctx);
+
+// aif_simt.cu
+cudaError_t launch_scatter_rows(const aif_ctx *ctx, const int32_t *ids, int64_t n, const void *rows, const void *bea_w,
+                                const uint8_t *sig, cudaStream_t st);
+cudaError_t launch_gather_rows(const aif_ctx *ctx, const int32_t *ids, int64_t n, void *out, cudaStream_t st);
+cudaError_t launch_transpose(const void *in, void *out, int rows, int cols, size_t el, cudaStream_t st);
+cudaError_t launch_score_simt(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st);
+cudaError_t launch_user_network(const aif_ctx *ctx, HostSlot &hs, int slot_index, const aif_user_inputs *in, int L,
+                                cudaStream_t st);
+int simt_tiles_for(const aif_ctx *ctx, int n);
+
+// tensor-core path (aif_tc.cu)
+bool tc_supported(const aif_config &cfg);
+cudaError_t tc_prepare_weights(aif_ctx *ctx, const aif_weights *w, cudaStream_t st);
+cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t total_candidates, cudaStream_t st);
+int tc_tiles_for(const aif_ctx *ctx, int n);
+
+}  // namespace aif

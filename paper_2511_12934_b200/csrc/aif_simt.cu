@@ -1,0 +1,686 @@
+// CUDA-core kernels of libaif: table scatter / gather, the general scoring kernel (any storage type, all
+// interaction blocks, fp32 arithmetic) and the user-side network.  The tensor-core kernels live in aif_tc.cu.
+#include "aif_internal.h"
+
+namespace aif {
+
+std::atomic<uint64_t> g_launches{0};
+
+// ------------------------------------------------------------------------------------------------
+// small device helpers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ void from_f(float &dst, float v) { dst = v; }
+__device__ __forceinline__ void from_f(__nv_bfloat16 &dst, float v) { dst = __float2bfloat16_rn(v); }
+
+// Cross-feature bucket hash: splitmix64 output function of id * golden + field (Section 3.3 leaves the
+// candidate attribute open; the id-derived bucket stands in for the category).
+__device__ __forceinline__ uint64_t mix64(uint64_t id, uint64_t field)
+{
+    uint64_t z = id * 0x9E3779B97F4A7C15ull + field;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+__device__ __forceinline__ int bucket_of(int id, int f, int B, int mode)
+{
+    if (mode == AIF_BUCKET_MOD) return id % B;
+    return (int)(mix64((uint64_t)id, (uint64_t)f) % (uint64_t)B);
+}
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// row (storage type, global) . q (fp32, shared), d a multiple of 8
+__device__ __forceinline__ float dot_row(const float *row, const float *q, int d)
+{
+    float acc = 0.f;
+    const float4 *r4 = reinterpret_cast<const float4 *>(row);
+    const float4 *q4 = reinterpret_cast<const float4 *>(q);
+    for (int k = 0; k < d / 4; ++k) {
+        float4 r = __ldg(r4 + k), w = q4[k];
+        acc = fmaf(r.x, w.x, acc);
+        acc = fmaf(r.y, w.y, acc);
+        acc = fmaf(r.z, w.z, acc);
+        acc = fmaf(r.w, w.w, acc);
+    }
+    return acc;
+}
+
+__device__ __forceinline__ float dot_row(const __nv_bfloat16 *row, const float *q, int d)
+{
+    float acc = 0.f;
+    const uint4 *r4 = reinterpret_cast<const uint4 *>(row);
+    const float4 *q4 = reinterpret_cast<const float4 *>(q);
+    for (int k = 0; k < d / 8; ++k) {
+        uint4 r = __ldg(r4 + k);
+        float4 a = q4[2 * k], b = q4[2 * k + 1];
+        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&r);
+        float2 f0 = __bfloat1622float2(h[0]), f1 = __bfloat1622float2(h[1]);
+        float2 f2 = __bfloat1622float2(h[2]), f3 = __bfloat1622float2(h[3]);
+        acc = fmaf(f0.x, a.x, acc);
+        acc = fmaf(f0.y, a.y, acc);
+        acc = fmaf(f1.x, a.z, acc);
+        acc = fmaf(f1.y, a.w, acc);
+        acc = fmaf(f2.x, b.x, acc);
+        acc = fmaf(f2.y, b.y, acc);
+        acc = fmaf(f3.x, b.z, acc);
+        acc = fmaf(f3.y, b.w, acc);
+    }
+    return acc;
+}
+
+// One warp, one query: streams over the L rows of S in chunks of 32 keys.
+//   att  = softmax(q S^T * scale) S      (online softmax; dense target attention and eqs. 2-3)
+//   din  = sum_j sim_j S_j, sim_j = matches(sig_q, sigS_j) / lsh_bits      (eqs. 6-8)
+//   tiers[t] += #{ j : tier(matches_j) = t }                               (eq. 9; shared-memory counters)
+// Lane owns columns lane, lane+32, ... of the outputs (d <= 256).
+template <typename T>
+__device__ void warp_interact(const float *q, const T *S, int L, int d, float scale, bool do_att, bool do_lsh,
+                              bool do_tiers, const uint32_t *sig_q, const uint8_t *sigS, int lsh_bits, int n_tiers,
+                              int *tiers, float att[8], float din[8])
+{
+    const int lane = threadIdx.x & 31, dq = d >> 5, words = lsh_bits >> 5;
+    float m = -INFINITY, l = 0.f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) att[c] = 0.f, din[c] = 0.f;
+    const float inv_bits = do_lsh ? 1.0f / (float)lsh_bits : 0.f;
+    for (int j0 = 0; j0 < L; j0 += 32) {
+        const int j = j0 + lane;
+        const bool valid = j < L;
+        float s = -INFINITY, simv = 0.f;
+        if (valid) {
+            if (do_att) s = dot_row(S + (size_t)j * d, q, d) * scale;
+            if (do_lsh) {
+                const uint32_t *sj = reinterpret_cast<const uint32_t *>(sigS + (size_t)j * (lsh_bits >> 3));
+                int diff = 0;
+                for (int w = 0; w < words; ++w) diff += __popc(sig_q[w] ^ __ldg(sj + w));
+                const int matches = lsh_bits - diff;
+                simv = (float)matches * inv_bits;
+                if (do_tiers) {
+                    int t = (matches * n_tiers) / lsh_bits;
+                    atomicAdd(&tiers[t < n_tiers - 1 ? t : n_tiers - 1], 1);
+                }
+            }
+        }
+        float p = 0.f;
+        if (do_att) {
+            const float m_new = fmaxf(m, warp_max(s));
+            const float sc = expf(m - m_new);
+            p = valid ? expf(s - m_new) : 0.f;
+            l = l * sc + warp_sum(p);
+            m = m_new;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) att[c] *= sc;
+        }
+        const int cnt = min(32, L - j0);
+        for (int jj = 0; jj < cnt; ++jj) {
+            const float pj = __shfl_sync(0xffffffffu, p, jj);
+            const float sj = __shfl_sync(0xffffffffu, simv, jj);
+            const T *row = S + (size_t)(j0 + jj) * d + lane;
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                if (c < dq) {
+                    const float v = to_f(row[32 * c]);
+                    att[c] = fmaf(pj, v, att[c]);
+                    din[c] = fmaf(sj, v, din[c]);
+                }
+        }
+    }
+    if (do_att) {
+        const float inv = 1.0f / l;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) att[c] *= inv;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// item table: scatter (nearline refresh) and gather
+// ------------------------------------------------------------------------------------------------
+template <typename V>
+__global__ void k_scatter_rows(V *__restrict__ table, const V *__restrict__ rows, const int32_t *__restrict__ ids,
+                               int64_t n, int vec_per_row, int64_t M, uint32_t *status)
+{
+    const int64_t total = n * vec_per_row;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / vec_per_row;
+        const int c = (int)(i - r * vec_per_row);
+        const int64_t dst = ids ? (int64_t)ids[r] : r;
+        if (dst < 0 || dst >= M) {
+            if (c == 0) atomicOr(status, AIF_STATUS_BAD_ID);
+            continue;
+        }
+        table[dst * vec_per_row + c] = rows[i];
+    }
+}
+
+// rows_out[i] = table[ids[i]]; 16 bytes per thread and four independent rows in flight per thread.
+__global__ void __launch_bounds__(256) k_gather_rows(const uint4 *__restrict__ table, const int32_t *__restrict__ ids,
+                                                     int64_t n, int vec_per_row, int64_t M, uint4 *__restrict__ out,
+                                                     uint32_t *status)
+{
+    const int64_t total = n * vec_per_row;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i < total; i += 4 * stride) {
+        uint4 v[4];
+        bool ok[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t ii = i + u * stride;
+            ok[u] = false;
+            v[u] = make_uint4(0, 0, 0, 0);
+            if (ii < total) {
+                const int64_t r = ii / vec_per_row;
+                const int c = (int)(ii - r * vec_per_row);
+                const int64_t src = ids[r];
+                ok[u] = true;
+                if (src >= 0 && src < M) v[u] = __ldg(table + src * vec_per_row + c);
+                else if (c == 0) atomicOr(status, AIF_STATUS_BAD_ID);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (ok[u]) out[i + u * stride] = v[u];
+    }
+}
+
+static int grid_for(int64_t items, int per_block, int cap)
+{
+    int64_t g = (items + per_block - 1) / per_block;
+    if (g < 1) g = 1;
+    return (int)(g > cap ? cap : g);
+}
+
+template <typename V>
+static cudaError_t scatter_typed(void *table, const void *rows, const int32_t *ids, int64_t n, size_t row_bytes, int64_t M,
+                                 uint32_t *status, cudaStream_t st)
+{
+    const int vpr = (int)(row_bytes / sizeof(V));
+    k_scatter_rows<V><<<grid_for(n * vpr, 256, 148 * 32), 256, 0, st>>>((V *)table, (const V *)rows, ids, n, vpr, M, status);
+    count_launch();
+    return cudaGetLastError();
+}
+
+static cudaError_t scatter_bytes(void *table, const void *rows, const int32_t *ids, int64_t n, size_t row_bytes, int64_t M,
+                                 uint32_t *status, cudaStream_t st)
+{
+    if (row_bytes % 16 == 0) return scatter_typed<uint4>(table, rows, ids, n, row_bytes, M, status, st);
+    if (row_bytes % 8 == 0) return scatter_typed<uint2>(table, rows, ids, n, row_bytes, M, status, st);
+    if (row_bytes % 4 == 0) return scatter_typed<uint32_t>(table, rows, ids, n, row_bytes, M, status, st);
+    return scatter_typed<uint16_t>(table, rows, ids, n, row_bytes, M, status, st);
+}
+
+cudaError_t launch_scatter_rows(const aif_ctx *ctx, const int32_t *ids, int64_t n, const void *rows, const void *bea_w,
+                                const uint8_t *sig, cudaStream_t st)
+{
+    const aif_config &c = ctx->cfg;
+    cudaError_t e = scatter_bytes(ctx->E, rows, ids, n, (size_t)c.d * ctx->el, c.M, ctx->status, st);
+    if (e != cudaSuccess) return e;
+    if (ctx->bea_w) {
+        e = scatter_bytes(ctx->bea_w, bea_w, ids, n, (size_t)c.n_bridge * ctx->el, c.M, ctx->status, st);
+        if (e != cudaSuccess) return e;
+    }
+    if (ctx->sig) e = scatter_bytes(ctx->sig, sig, ids, n, (size_t)c.lsh_bits / 8, c.M, ctx->status, st);
+    return e;
+}
+
+cudaError_t launch_gather_rows(const aif_ctx *ctx, const int32_t *ids, int64_t n, void *out, cudaStream_t st)
+{
+    const int vpr = (int)((size_t)ctx->cfg.d * ctx->el / 16);
+    const int64_t total = n * vpr;
+    const int grid = grid_for((total + 3) / 4, 256, 148 * 16);
+    k_gather_rows<<<grid, 256, 0, st>>>((const uint4 *)ctx->E, ids, n, vpr, ctx->cfg.M, (uint4 *)out, ctx->status);
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <typename T>
+__global__ void k_transpose(const T *__restrict__ in, T *__restrict__ out, int rows, int cols)
+{
+    __shared__ T tile[32][33];
+    const int bx = blockIdx.x * 32, by = blockIdx.y * 32;
+    for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+        const int y = by + r, x = bx + threadIdx.x;
+        if (y < rows && x < cols) tile[r][threadIdx.x] = in[(size_t)y * cols + x];
+    }
+    __syncthreads();
+    for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+        const int x = bx + r, y = by + threadIdx.x;
+        if (y < rows && x < cols) out[(size_t)x * rows + y] = tile[threadIdx.x][r];
+    }
+}
+
+// out [cols x rows] = in [rows x cols]^T
+cudaError_t launch_transpose(const void *in, void *out, int rows, int cols, size_t el, cudaStream_t st)
+{
+    dim3 grid((cols + 31) / 32, (rows + 31) / 32), block(32, 8);
+    if (el == 4) k_transpose<float><<<grid, block, 0, st>>>((const float *)in, (float *)out, rows, cols);
+    else k_transpose<uint16_t><<<grid, block, 0, st>>>((const uint16_t *)in, (uint16_t *)out, rows, cols);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// tiles of a request: kTile candidates, never across a mini-batch boundary
+// ------------------------------------------------------------------------------------------------
+__host__ __device__ inline int tiles_of(int n, int tile, int mb)
+{
+    if (mb <= 0) return (n + tile - 1) / tile;
+    const int tpm = (mb + tile - 1) / tile;
+    const int full = n / mb, rem = n - full * mb;
+    return full * tpm + (rem + tile - 1) / tile;
+}
+
+__device__ inline void tile_range(int lt, int n, int tile, int mb, int &start, int &cnt)
+{
+    if (mb <= 0) {
+        start = lt * tile;
+        cnt = min(tile, n - start);
+        return;
+    }
+    const int tpm = (mb + tile - 1) / tile;
+    const int b = lt / tpm, w = lt - b * tpm;
+    start = b * mb + w * tile;
+    const int end = min(min(start + tile, (b + 1) * mb), n);
+    cnt = end - start;
+}
+
+__device__ inline ReqDev find_request(const ScoreLaunch &sl, int t)
+{
+    if (sl.reqs == nullptr) return sl.single;
+    int lo = 0, hi = sl.n_req - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (sl.reqs[mid].tile_begin <= t) lo = mid;
+        else hi = mid - 1;
+    }
+    return sl.reqs[lo];
+}
+
+int simt_tiles_for(const aif_ctx *ctx, int n) { return tiles_of(n, kSimtTile, ctx->cfg.mini_batch); }
+
+// ------------------------------------------------------------------------------------------------
+// general scoring kernel: one block = one tile of kSimtTile candidates, one warp per candidate for the
+// interaction blocks, then all threads for the MLP with the decomposed first layer.
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kSimtThreads) k_score_simt(ModelDev md, ScoreLaunch sl, int max_h)
+{
+    constexpr int TM = kSimtTile;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *xs = reinterpret_cast<float *>(smem_raw);        // [k1][TM]   candidate-dependent input, transposed
+    float *ha = xs + (size_t)md.k1 * TM;                     // [max_h][TM]
+    float *hb = ha + (size_t)max_h * TM;                     // [max_h][TM]
+    float *qv = hb + (size_t)max_h * TM;                     // [TM][d]    item vectors as fp32 rows (queries)
+    uint32_t *sigq = reinterpret_cast<uint32_t *>(qv + (size_t)TM * md.d);   // [TM][8]
+    int *tiers = reinterpret_cast<int *>(sigq + TM * 8);     // [TM][16]
+    int *bkt = tiers + TM * 16;                              // [TM][F]
+    int *id_s = bkt + TM * md.F;                             // [TM]
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const ReqDev rq = find_request(sl, blockIdx.x);
+    int start, cnt;
+    tile_range(blockIdx.x - rq.tile_begin, rq.n, TM, md.mini_batch, start, cnt);
+    const SlotDev slot = sl.slots[rq.slot];
+    const int32_t *ids = sl.ids + rq.off + start;
+    float *logits = sl.logits + rq.off + start;
+    const int d = md.d, dq = d >> 5;
+
+    if (tid < TM) {
+        int id = -1;
+        if (tid < cnt) {
+            id = ids[tid];
+            if (id < 0 || (int64_t)id >= md.M) {
+                id = -1;
+                atomicOr(sl.status, AIF_STATUS_BAD_ID);
+            }
+        }
+        id_s[tid] = id;
+    }
+    for (int i = tid; i < md.k1 * TM; i += kSimtThreads) xs[i] = 0.f;
+    for (int i = tid; i < TM * 16; i += kSimtThreads) tiers[i] = 0;
+    __syncthreads();
+
+    // ---- stage A: interaction blocks, warp c <-> candidate c
+    {
+        const int c = warp;
+        const int id = id_s[c];
+        if (id >= 0) {
+            const T *e = reinterpret_cast<const T *>(md.E) + (size_t)id * d;
+            int col = 0;
+            for (int k = lane; k < d; k += 32) {
+                const float v = to_f(e[k]);
+                qv[c * d + k] = v;
+                xs[(col + k) * TM + c] = v;
+            }
+            col += d;
+            const bool do_att = md.blocks & AIF_BLK_ATT, do_din = md.blocks & AIF_BLK_LSH_DIN,
+                       do_tier = md.blocks & AIF_BLK_SIMTIER, do_lsh = do_din || do_tier;
+            if (do_lsh && lane < (md.lsh_bits >> 5))
+                sigq[c * 8 + lane] = reinterpret_cast<const uint32_t *>(md.sig + (size_t)id * (md.lsh_bits >> 3))[lane];
+            if (md.blocks & AIF_BLK_CROSS)
+                for (int f = lane; f < md.F; f += 32) bkt[c * md.F + f] = bucket_of(id, f, md.B, md.bucket_mode);
+            __syncwarp();
+            float att[8], din[8];
+            if (do_att || do_lsh)
+                warp_interact<T>(qv + c * d, reinterpret_cast<const T *>(slot.S), slot.L, d, rsqrtf((float)d), do_att,
+                                 do_lsh, do_tier, sigq + c * 8, slot.sigS, md.lsh_bits, md.n_tiers, tiers + c * 16, att,
+                                 din);
+            if (do_att) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (q < dq) xs[(col + lane + 32 * q) * TM + c] = att[q];
+                col += d;
+            }
+            if (md.blocks & AIF_BLK_CROSS) {
+                const T *Tt = reinterpret_cast<const T *>(slot.T);
+                const int fdc = md.F * md.dc;
+                for (int i = lane; i < fdc; i += 32) {
+                    const int f = i / md.dc, k = i - f * md.dc;
+                    xs[(col + i) * TM + c] = to_f(Tt[((size_t)f * md.B + bkt[c * md.F + f]) * md.dc + k]);
+                }
+                col += fdc;
+            }
+            if (md.blocks & AIF_BLK_BEA) {
+                const T *wh = reinterpret_cast<const T *>(md.bea_w) + (size_t)id * md.n_bridge;
+                const T *V = reinterpret_cast<const T *>(slot.V);
+                for (int k = lane; k < d; k += 32) {
+                    float acc = 0.f;
+                    for (int b = 0; b < md.n_bridge; ++b) acc = fmaf(to_f(wh[b]), to_f(V[(size_t)b * d + k]), acc);
+                    xs[(col + k) * TM + c] = acc;
+                }
+                col += d;
+            }
+            if (do_din) {
+                const float nrm = md.lsh_din_norm == AIF_NORM_MEAN ? 1.0f / (float)slot.L : 1.0f;
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (q < dq) xs[(col + lane + 32 * q) * TM + c] = din[q] * nrm;
+                col += d;
+            }
+            if (do_tier) {
+                __syncwarp();
+                const float nrm = md.simtier_norm == AIF_NORM_MEAN ? 1.0f / (float)slot.L : 1.0f;
+                if (lane < md.n_tiers) xs[(col + lane) * TM + c] = (float)tiers[c * 16 + lane] * nrm;
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- stage B: MLP.  First layer = cached user partial + candidate-dependent columns.
+    const float *in_act = xs;
+    float *out_act = ha;
+    int in_w = md.k1;
+    for (int layer = 0; layer < md.n_hidden; ++layer) {
+        const int H = md.hidden[layer];
+        const T *W = reinterpret_cast<const T *>(md.Wt[layer]) + (layer == 0 ? (size_t)d * H : 0);
+        const float *bias = layer == 0 ? slot.p_u : md.b[layer];
+        for (int j = tid; j < H; j += kSimtThreads) {
+            float acc[TM];
+            const float b0 = bias[j];
+#pragma unroll
+            for (int c = 0; c < TM; ++c) acc[c] = b0;
+            for (int k = 0; k < in_w; ++k) {
+                const float w = to_f(W[(size_t)k * H + j]);
+                const float4 a = *reinterpret_cast<const float4 *>(in_act + k * TM);
+                const float4 b = *reinterpret_cast<const float4 *>(in_act + k * TM + 4);
+                acc[0] = fmaf(w, a.x, acc[0]);
+                acc[1] = fmaf(w, a.y, acc[1]);
+                acc[2] = fmaf(w, a.z, acc[2]);
+                acc[3] = fmaf(w, a.w, acc[3]);
+                acc[4] = fmaf(w, b.x, acc[4]);
+                acc[5] = fmaf(w, b.y, acc[5]);
+                acc[6] = fmaf(w, b.z, acc[6]);
+                acc[7] = fmaf(w, b.w, acc[7]);
+            }
+#pragma unroll
+            for (int c = 0; c < TM; ++c) out_act[j * TM + c] = fmaxf(acc[c], 0.f);
+        }
+        __syncthreads();
+        in_act = out_act;
+        out_act = (out_act == ha) ? hb : ha;
+        in_w = H;
+    }
+    // ---- output layer: warp c reduces candidate c in a fixed order
+    {
+        const int c = warp;
+        if (c < cnt) {
+            const T *wo = reinterpret_cast<const T *>(md.w_out);
+            float acc = 0.f;
+            for (int j = lane; j < in_w; j += 32) acc = fmaf(to_f(wo[j]), in_act[j * TM + c], acc);
+            acc = warp_sum(acc);
+            if (lane == 0) {
+                float logit = acc + md.b_out[0];
+                if (md.emit_sigmoid) logit = 1.0f / (1.0f + expf(-logit));
+                logits[c] = id_s[c] >= 0 ? logit : __int_as_float(0x7fc00000);
+            }
+        }
+    }
+}
+
+static size_t simt_smem_bytes(const aif_ctx *ctx, int &max_h)
+{
+    const aif_config &c = ctx->cfg;
+    max_h = 0;
+    for (int k = 0; k < c.n_hidden; ++k) max_h = c.hidden[k] > max_h ? c.hidden[k] : max_h;
+    const int k1 = ctx->input_width - c.d;
+    size_t fl = (size_t)(k1 + 2 * max_h + c.d) * kSimtTile;
+    size_t ints = (size_t)kSimtTile * (8 + 16 + c.F + 1);
+    return (fl + ints) * 4 + 16;
+}
+
+cudaError_t launch_score_simt(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st)
+{
+    if (sl.n_tiles <= 0) return cudaSuccess;
+    int max_h;
+    const size_t smem = simt_smem_bytes(ctx, max_h);
+    const ModelDev md = make_model(ctx);
+    cudaError_t e;
+    if (ctx->cfg.dtype == AIF_F32) {
+        e = cudaFuncSetAttribute(k_score_simt<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k_score_simt<float><<<sl.n_tiles, kSimtThreads, smem, st>>>(md, sl, max_h);
+    } else {
+        e = cudaFuncSetAttribute(k_score_simt<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k_score_simt<__nv_bfloat16><<<sl.n_tiles, kSimtThreads, smem, st>>>(md, sl, max_h);
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// user-side network (eqs. 1-3), fp32 arithmetic on storage-type inputs
+// ------------------------------------------------------------------------------------------------
+
+// eq. 1.  blockIdx.x < L: one sequence row -> S (storage type).  blockIdx.x == L: the profile -> prof_hat (fp32).
+template <typename T>
+__global__ void k_user_project(const T *__restrict__ seq, const T *__restrict__ profile, const T *__restrict__ Wseq_t,
+                               const T *__restrict__ Wprof_t, int L, int dU, int d, T *__restrict__ S,
+                               float *__restrict__ prof_hat)
+{
+    extern __shared__ float row[];
+    const bool is_prof = (int)blockIdx.x == L;
+    const T *src = is_prof ? profile : seq + (size_t)blockIdx.x * dU;
+    const T *W = is_prof ? Wprof_t : Wseq_t;
+    for (int k = threadIdx.x; k < dU; k += blockDim.x) row[k] = to_f(src[k]);
+    __syncthreads();
+    for (int j = threadIdx.x; j < d; j += blockDim.x) {
+        float acc = 0.f;
+        for (int k = 0; k < dU; ++k) acc = fmaf(row[k], to_f(W[(size_t)k * d + j]), acc);
+        if (is_prof) prof_hat[j] = acc;
+        else from_f(S[(size_t)blockIdx.x * d + j], acc);
+    }
+}
+
+// eq. 2.  Warp g handles rows g, g + n_warps, ...: attention over the whole sequence, FFN, and a running sum
+// for the mean pooling; partial[g] holds the warp's sum (summed later in a fixed order).
+template <typename T>
+__global__ void __launch_bounds__(256) k_user_self(const T *__restrict__ S, int L, int d, const T *__restrict__ Wa_t,
+                                                   const float *__restrict__ b_a, const T *__restrict__ Wb_t,
+                                                   const float *__restrict__ b_b, float *__restrict__ partial,
+                                                   int n_warps)
+{
+    extern __shared__ float sm[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = blockIdx.x * 8 + warp, dq = d >> 5;
+    float *q = sm + (size_t)warp * 3 * d, *ctx = q + d, *hid = ctx + d;
+    float pooled[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) pooled[c] = 0.f;
+    const float scale = rsqrtf((float)d);
+    for (int i = g; i < L; i += n_warps) {
+        for (int k = lane; k < d; k += 32) q[k] = to_f(S[(size_t)i * d + k]);
+        __syncwarp();
+        float att[8], din[8];
+        warp_interact<T>(q, S, L, d, scale, true, false, false, nullptr, nullptr, 0, 0, nullptr, att, din);
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+            if (c < dq) ctx[lane + 32 * c] = att[c];
+        __syncwarp();
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+            if (c < dq) {
+                const int j = lane + 32 * c;
+                float acc = b_a[j];
+                for (int k = 0; k < d; ++k) acc = fmaf(ctx[k], to_f(Wa_t[(size_t)k * d + j]), acc);
+                hid[j] = fmaxf(acc, 0.f);
+            }
+        __syncwarp();
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+            if (c < dq) {
+                const int j = lane + 32 * c;
+                float acc = b_b[j];
+                for (int k = 0; k < d; ++k) acc = fmaf(hid[k], to_f(Wb_t[(size_t)k * d + j]), acc);
+                pooled[c] += acc;
+            }
+        __syncwarp();
+    }
+    if (g < n_warps) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+            if (c < dq) partial[(size_t)g * d + lane + 32 * c] = pooled[c];
+    }
+}
+
+// eq. 3, the combined vector, and the cached first-layer partial product p_u = W1[:, 0:d] u + b1.
+// raw = 1: u = mean-pooled self-attention + profile attention.  raw = 0: u is given (u_in, storage type).
+template <typename T>
+__global__ void __launch_bounds__(256) k_user_finish(int raw, const T *__restrict__ S, int L, int d,
+                                                     const float *__restrict__ prof_hat,
+                                                     const float *__restrict__ partial, int n_warps,
+                                                     const T *__restrict__ u_in, T *__restrict__ u_out,
+                                                     float *__restrict__ u32, const T *__restrict__ W1t,
+                                                     const float *__restrict__ b1, int H1, float *__restrict__ p_u)
+{
+    __shared__ float q[256], uprof[256], us[256];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, dq = d >> 5;
+    if (raw) {
+        for (int k = tid; k < d; k += 256) q[k] = prof_hat[k];
+        __syncthreads();
+        if (warp == 0) {
+            float att[8], din[8];
+            warp_interact<T>(q, S, L, d, rsqrtf((float)d), true, false, false, nullptr, nullptr, 0, 0, nullptr, att, din);
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                if (c < dq) uprof[lane + 32 * c] = att[c];
+        }
+        __syncthreads();
+        for (int k = tid; k < d; k += 256) {
+            float acc = 0.f;
+            for (int g = 0; g < n_warps; ++g) acc += partial[(size_t)g * d + k];
+            const float u = acc / (float)L + uprof[k];
+            us[k] = u;
+            u32[k] = u;
+            from_f(u_out[k], u);
+        }
+    } else {
+        for (int k = tid; k < d; k += 256) {
+            const float u = to_f(u_in[k]);
+            us[k] = u;
+            u32[k] = u;
+        }
+    }
+    __syncthreads();
+    for (int j = tid; j < H1; j += 256) {
+        float acc = b1[j];
+        for (int k = 0; k < d; ++k) acc = fmaf(us[k], to_f(W1t[(size_t)k * H1 + j]), acc);
+        p_u[j] = acc;
+    }
+}
+
+__global__ void k_set_slot_len(SlotDev *slots, int index, int L) { slots[index].L = L; }
+
+template <typename T>
+static cudaError_t user_network_typed(const aif_ctx *ctx, HostSlot &hs, int slot_index, const aif_user_inputs *in, int L,
+                                      cudaStream_t st)
+{
+    const aif_config &c = ctx->cfg;
+    const int d = c.d, H1 = c.hidden[0];
+    cudaError_t e;
+    T *S = (T *)hs.dev.S;
+    const bool raw = in->mode == AIF_USER_RAW;
+    if (raw) {
+        k_user_project<T><<<L + 1, 128, c.dU * sizeof(float), st>>>((const T *)in->seq, (const T *)in->profile,
+                                                                    (const T *)ctx->Wseq_t, (const T *)ctx->Wprofile_t, L,
+                                                                    c.dU, d, S, hs.prof_hat);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        const int n_warps = kUserPartials;
+        k_user_self<T><<<n_warps / 8, 256, 8 * 3 * d * sizeof(float), st>>>(S, L, d, (const T *)ctx->Wa_t, ctx->b_a,
+                                                                            (const T *)ctx->Wb_t, ctx->b_b, hs.partial,
+                                                                            n_warps);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    } else {
+        if ((e = cudaMemcpyAsync(S, in->seq, (size_t)L * d * sizeof(T), cudaMemcpyDeviceToDevice, st)) != cudaSuccess) return e;
+        if ((e = cudaMemcpyAsync((void *)hs.dev.u, in->profile, (size_t)d * sizeof(T), cudaMemcpyDeviceToDevice, st)) !=
+            cudaSuccess)
+            return e;
+    }
+    k_user_finish<T><<<1, 256, 0, st>>>(raw ? 1 : 0, S, L, d, hs.prof_hat, hs.partial, kUserPartials,
+                                        (const T *)in->profile, (T *)hs.dev.u, (float *)hs.dev.u32, (const T *)ctx->Wt[0],
+                                        ctx->b[0], H1, (float *)hs.dev.p_u);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    k_set_slot_len<<<1, 1, 0, st>>>(ctx->slots_dev, slot_index, L);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_user_network(const aif_ctx *ctx, HostSlot &hs, int slot_index, const aif_user_inputs *in, int L,
+                                cudaStream_t st)
+{
+    const aif_config &c = ctx->cfg;
+    cudaError_t e;
+    if (c.blocks & AIF_BLK_CROSS) {
+        e = cudaMemcpyAsync((void *)hs.dev.T, in->cross_raw, (size_t)c.F * c.B * c.dc * ctx->el, cudaMemcpyDeviceToDevice, st);
+        if (e != cudaSuccess) return e;
+    }
+    if (c.blocks & AIF_BLK_BEA) {
+        e = cudaMemcpyAsync((void *)hs.dev.V, in->bea_V, (size_t)c.n_bridge * c.d * ctx->el, cudaMemcpyDeviceToDevice, st);
+        if (e != cudaSuccess) return e;
+    }
+    if (c.blocks & (AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER)) {
+        e = cudaMemcpyAsync((void *)hs.dev.sigS, in->seq_sig, (size_t)L * (c.lsh_bits / 8), cudaMemcpyDeviceToDevice, st);
+        if (e != cudaSuccess) return e;
+    }
+    if (c.dtype == AIF_F32) return user_network_typed<float>(ctx, hs, slot_index, in, L, st);
+    return user_network_typed<__nv_bfloat16>(ctx, hs, slot_index, in, L, st);
+}
+
+}  // namespace aif

@@ -1,0 +1,223 @@
+"""Parity of the CUDA library (through its C ABI) against the CPU oracle, on the same seeded inputs.
+
+Tolerances (written here, as the benchmark definition states them): |delta logit| <= 1e-5 for the fp32
+configuration, <= 2e-3 for bf16 storage with fp32 accumulation; ids, buckets, table rows and signatures are
+compared bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import aif_oracle as orc
+from paper_2511_12934_b200 import binding as B
+from paper_2511_12934_b200 import build as libbuild
+from paper_2511_12934_b200 import serving, synth
+from tests import helpers
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-5, "bf16": 2e-3}
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    libbuild.build()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    B.load_library()
+
+
+def _setup(wl, path=B.PATH_AUTO, zero_bias=False, **kw):
+    weights = synth.make_weights(wl, zero_bias=zero_bias)
+    table = synth.make_item_table(wl)
+    srv = serving.Server(wl, weights, table, path=path, **kw)
+    oracle = helpers.make_oracle(wl, weights, M=table["E"].shape[0])
+    return weights, table, srv, oracle
+
+
+def _check_logits(got, want, tol):
+    assert got.shape == want.shape
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    ok = ~np.isnan(want)
+    err = np.abs(got[ok].astype(np.float64) - want[ok]).max() if ok.any() else 0.0
+    assert err <= tol, f"max |delta| = {err:.3e} > {tol}"
+    return err
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4", "c5"])
+@pytest.mark.parametrize("path", [B.PATH_SIMT, B.PATH_AUTO])
+def test_scoring_matches_oracle_on_scaled_configs(name, path):
+    wl = helpers.MINI[name]
+    weights, table, srv, oracle = _setup(wl, path)
+    sampler = synth.IdSampler(wl)
+    states, id_lists, wants = [], [], []
+    for r in range(wl.R):
+        rq = synth.make_request(wl, r)
+        ids = sampler.request_ids(r)
+        st = srv.precompute(1000 + r, srv.upload_request(rq, B.USER_PROJECTED))
+        assert st.request_key == 1000 + r
+        want = oracle.score(table, helpers.projected_request(wl, rq), ids)
+        got = srv.score_ids(st, ids)
+        _check_logits(got, want, TOL[wl.dtype])
+        states.append(st), id_lists.append(ids), wants.append(want)
+        # mini-batch invariance: one call per chunk gives the same numbers as one call for the request
+        chunks = np.concatenate([srv.score_ids(st, ids[s:s + 77]) for s in range(0, len(ids), 77)])
+        _check_logits(chunks, want, TOL[wl.dtype])
+        if not srv.ctx.get_stats().tensor_path:
+            assert np.array_equal(chunks, got)
+        # permutation equivariance
+        perm = np.random.default_rng(r).permutation(len(ids))
+        gp = srv.score_ids(st, ids[perm])
+        _check_logits(gp, want[perm], TOL[wl.dtype])
+        if not srv.ctx.get_stats().tensor_path:
+            assert np.array_equal(gp, got[perm])
+    # all requests in one launch
+    outs = srv.score_many(states, id_lists)
+    for o, w in zip(outs, wants):
+        _check_logits(o, w, TOL[wl.dtype])
+    assert srv.ctx.poll_status() == 0
+    srv.close()
+
+
+@pytest.mark.parametrize("dtype,din_norm,tier_norm", [("f32", synth.NORM_NONE, synth.NORM_NONE),
+                                                      ("f32", synth.NORM_MEAN, synth.NORM_MEAN),
+                                                      ("bf16", synth.NORM_MEAN, synth.NORM_MEAN)])
+def test_all_interaction_blocks(dtype, din_norm, tier_norm):
+    base = helpers.MINI["c1"] if dtype == "f32" else helpers.MINI["c2"]
+    wl = base.with_(name=f"blocks_{dtype}_{din_norm}", blocks=helpers.ALL_BLOCKS, lsh_din_norm=din_norm,
+                    simtier_norm=tier_norm, N=200, L=75, emit_sigmoid=0)
+    weights, table, srv, oracle = _setup(wl)
+    rq = synth.make_request(wl, 0)
+    ids = synth.IdSampler(wl).request_ids(0)
+    st = srv.precompute(1, srv.upload_request(rq, B.USER_PROJECTED))
+    want = oracle.score(table, helpers.projected_request(wl, rq), ids)
+    # raw SimTier counts and unnormalised LSH-DIN sums are O(L): scale the absolute tolerance with the logit size
+    scale = max(1.0, float(np.abs(want).max()))
+    _check_logits(srv.score_ids(st, ids), want, TOL[dtype] * scale)
+    srv.close()
+
+
+@pytest.mark.parametrize("name", ["c1", "c2"])
+def test_user_precompute_raw_matches_eqs_1_to_3(name):
+    wl = helpers.MINI[name].with_(name=f"raw_{name}", dU=48, L=60, N=150)
+    weights, table, srv, oracle = _setup(wl)
+    rq = synth.make_request(wl, 0)
+    ids = synth.IdSampler(wl).request_ids(0)
+    st = srv.precompute(5, srv.upload_request(rq, B.USER_RAW))
+    u, S, pu = srv.ctx.user_state_export(st, wl.L)
+    torch.cuda.synchronize()
+    u_ref, S_ref = oracle.user_state(rq["profile"], rq["seq"])
+    W1 = synth.as_f32(weights["mlp"]["W"][0], wl.dtype).astype(np.float64)
+    pu_ref = W1[:, :wl.d] @ u_ref + weights["mlp"]["b"][0]
+    tol = 1e-5 if wl.dtype == "f32" else 2e-3
+    assert np.abs(u.cpu().numpy() - u_ref).max() <= tol
+    assert np.abs(S.float().cpu().numpy() - S_ref).max() <= (1e-6 if wl.dtype == "f32" else 2e-3)
+    assert np.abs(pu.cpu().numpy() - pu_ref).max() <= tol
+    want = oracle.score(table, helpers.raw_request(oracle, rq), ids)
+    _check_logits(srv.score_ids(st, ids), want, TOL[wl.dtype])
+    # cached state == recomputed state, bit for bit
+    st2 = srv.precompute(6, srv.upload_request(rq, B.USER_RAW))
+    u2, S2, pu2 = srv.ctx.user_state_export(st2, wl.L)
+    torch.cuda.synchronize()
+    assert torch.equal(u, u2) and torch.equal(S, S2) and torch.equal(pu, pu2)
+    assert np.array_equal(srv.score_ids(st2, ids), srv.score_ids(st, ids))
+    srv.close()
+
+
+def test_refresh_and_gather_are_bit_exact():
+    wl = helpers.MINI["c2"].with_(name="refresh", blocks=helpers.ALL_BLOCKS)
+    weights, table, srv, oracle = _setup(wl)
+    g = np.random.default_rng(3)
+    host = {k: v.copy() for k, v in table.items()}
+    upd_ids = np.concatenate([g.choice(wl.M, 500, replace=False), [-1, wl.M, 2**31 - 1]]).astype(np.int32)
+    new = synth.make_item_table(wl.with_(name="refresh_new"), rows=len(upd_ids))
+    for k in ("E", "bea_w", "sig"):
+        assert orc.table_refresh(host[k], upd_ids, new[k]) == 3
+    srv.refresh_rows(upd_ids, new["E"], new["bea_w"], new["sig"])
+    assert srv.ctx.poll_status() == B.STATUS_BAD_ID
+    probe = np.concatenate([upd_ids[:500], g.integers(0, wl.M, 2000)]).astype(np.int32)
+    ids_t = torch.from_numpy(probe).cuda()
+    out = torch.empty(len(probe), wl.d, dtype=torch.bfloat16, device="cuda")
+    srv.ctx.gather_rows(ids_t, out)
+    torch.cuda.synchronize()
+    got = out.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(got, host["E"][probe])
+    # scoring after the incremental update sees the new rows, sidecars included
+    rq = synth.make_request(wl, 0)
+    st = srv.precompute(1, srv.upload_request(rq, B.USER_PROJECTED))
+    ids = probe[:300]
+    want = oracle.score(host, helpers.projected_request(wl, rq), ids)
+    _check_logits(srv.score_ids(st, ids), want, TOL["bf16"])
+    assert srv.ctx.poll_status() == 0
+    srv.close()
+
+
+def test_bad_ids_edge_sizes_and_errors():
+    wl = helpers.MINI["c1"].with_(name="edges", L=1, N=40)
+    weights, table, srv, oracle = _setup(wl, max_user_states=2, max_batch_candidates=64)
+    rq = synth.make_request(wl, 0)
+    dev = srv.upload_request(rq, B.USER_PROJECTED)
+    st = srv.precompute(1, dev)
+    ids = synth.IdSampler(wl).request_ids(0)
+    req = helpers.projected_request(wl, rq)
+    # n = 1 and a sequence of length 1
+    _check_logits(srv.score_ids(st, ids[:1]), oracle.score(table, req, ids[:1]), TOL["f32"])
+    # bad ids -> NaN + status bit, neighbours untouched
+    bad = ids.copy()
+    bad[3], bad[17] = -5, wl.M
+    _check_logits(srv.score_ids(st, bad), oracle.score(table, req, bad), TOL["f32"])
+    assert srv.ctx.poll_status() == B.STATUS_BAD_ID and srv.ctx.poll_status() == 0
+    # n = 0 is a no-op
+    empty = torch.empty(0, dtype=torch.int32, device="cuda")
+    srv.ctx.score(st, empty, torch.empty(0, device="cuda"))
+    # too many candidates, too long a sequence, arena exhaustion
+    with pytest.raises(B.AifError) as e:
+        srv.score_ids(st, np.zeros(65, np.int32))
+    assert e.value.code == B.ERR_SHAPE
+    long_rq = synth.make_request(wl, 0, L=2)
+    with pytest.raises(B.AifError) as e:
+        srv.precompute(2, srv.upload_request(long_rq, B.USER_PROJECTED))
+    assert e.value.code == B.ERR_SHAPE
+    st2 = srv.precompute(2, dev)
+    with pytest.raises(B.AifError) as e:
+        srv.precompute(3, dev)
+    assert e.value.code == B.ERR_OOM
+    st2.release()
+    st3 = srv.precompute(3, dev)
+    # reloading weights invalidates cached user states (version consistency)
+    srv.ctx.load_weights_host(weights)
+    with pytest.raises(B.AifError) as e:
+        srv.score_ids(st3, ids)
+    assert e.value.code == B.ERR_VERSION
+    stats = srv.ctx.get_stats()
+    assert stats.model_version == 2 and stats.user_states_high_water == 2 and stats.bad_id_events == 1
+    srv.close()
+
+
+def test_precompute_overlaps_a_simulated_retrieval_phase():
+    """The user-side call runs on a side stream while the main stream is busy with 'retrieval'; scoring waits on
+    the state's event, so the result is the same as without overlap."""
+    wl = helpers.MINI["c3"].with_(name="overlap", R=1)
+    weights, table, srv, oracle = _setup(wl)
+    rq = synth.make_request(wl, 0)
+    ids = synth.IdSampler(wl).request_ids(0)
+    dev = srv.upload_request(rq, B.USER_RAW)
+    torch.cuda.synchronize()
+    torch.cuda._sleep(20_000_000)                      # retrieval stand-in on the main stream
+    st = srv.precompute(1, dev)                        # side stream, concurrent
+    got = srv.score_ids(st, ids)                       # main stream: waits for both
+    want = oracle.score(table, helpers.raw_request(oracle, rq), ids)
+    _check_logits(got, want, TOL["bf16"])
+    srv.close()
+
+
+def test_full_size_c1_and_sampled_c2():
+    for wl, n_check in ((synth.C1, None), (synth.C2, 1500)):
+        weights, table, srv, oracle = _setup(wl, zero_bias=True)
+        rq = synth.make_request(wl, 0)
+        ids = synth.IdSampler(wl).request_ids(0)
+        st = srv.precompute(1, srv.upload_request(rq, B.USER_PROJECTED))
+        got = srv.score_ids(st, ids)
+        pick = np.arange(len(ids)) if n_check is None else np.random.default_rng(0).choice(len(ids), n_check, False)
+        want = oracle.score(table, helpers.projected_request(wl, rq), ids[pick])
+        _check_logits(got[pick], want, TOL[wl.dtype])
+        assert np.isfinite(got).all()
+        srv.close()
