@@ -1,0 +1,368 @@
+#!/usr/bin/env python
+"""Benchmark of the AIF pre-ranking scoring pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+
+One "step" is one pass of the whole real-time path (gather, interaction blocks, scoring MLP) over one batch of
+synthetic candidates: one aif_score call on a 10^4-candidate request for the default workload (the paper-shaped
+single request), one aif_score_batch call for the multi-request workloads.  User states are computed beforehand by
+aif_user_precompute (they belong to the retrieval phase, not to the timed real-time phase).
+
+Prints ONE JSON line (rank 0).  `value` is candidates scored per second with ids already resident in GPU memory;
+`e2e` is the same metric through aif_score_host with host buffers (H2D of the ids and D2H of the logits inside the
+timed region).  With --gpus N > 1 (launched by torchrun) every rank runs an independent replica on its own GPU:
+the path does not shard, so there is no data-path collective; the time is the max over ranks.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2511_12934_b200 import synth
+
+METRIC = "candidates scored/s (p50 latency per request reported beside it), 1 B200"
+UNIT = "candidates/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # CUDA-core kernels: SMs x lanes x 2 x max clock
+
+# DRAM traffic per launch of the dominant kernel from the committed ncu summary (profiles/), bytes; None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# algorithmic work (what the method itself has to do; padding and recomputation are not counted)
+# ----------------------------------------------------------------------------------------------------------------
+def flops_per_candidate(wl: synth.Workload) -> dict:
+    k1 = wl.input_width() - wl.d                       # the user columns are done once per request
+    f = {"attention": 4.0 * wl.L * wl.d if wl.blocks & synth.BLK_ATT else 0.0}
+    f["lsh_din"] = 2.0 * wl.L * wl.d if wl.blocks & synth.BLK_LSH_DIN else 0.0
+    f["bea"] = 2.0 * wl.n_bridge * wl.d if wl.blocks & synth.BLK_BEA else 0.0
+    widths = [k1] + list(wl.hidden)
+    for i in range(len(wl.hidden)):
+        f[f"layer{i + 1}"] = 2.0 * widths[i] * widths[i + 1]
+    f[f"layer{len(wl.hidden)}"] += 2.0 * wl.hidden[-1]  # output dot rides in the last hidden layer's kernel
+    f["total"] = sum(f.values())
+    return f
+
+
+def kernel_flops(name: str, wl: synth.Workload, n: int) -> float:
+    f = flops_per_candidate(wl)
+    if name == "score_simt":
+        return f["total"] * n
+    if name == "interact":
+        return (f["attention"] + f["lsh_din"] + f["bea"]) * n
+    return f.get(name, 0.0) * n
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as fh:
+            return json.load(fh), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# clocks during the timed region
+# ----------------------------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", uuid, f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in out.strip().splitlines():
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])), mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# the oracle legs (CPU): cpu_baseline and --impl reference
+# ----------------------------------------------------------------------------------------------------------------
+def oracle_setup(wl):
+    from oracle import aif_oracle as orc
+    from tests import helpers
+    weights = synth.make_weights(wl)
+    table = synth.make_item_table(wl)
+    oracle = helpers.make_oracle(wl, weights, M=table["E"].shape[0])
+    rq = synth.make_request(wl, 0)
+    ids = synth.IdSampler(wl).request_ids(0)
+    return oracle, table, helpers.projected_request(wl, rq), ids, orc.num_threads()
+
+
+def oracle_sample_size(wl, core_seconds=12.0):
+    # the scalar fp64 oracle sustains roughly 1 GFLOP/s per core
+    n = int(core_seconds * 1.0e9 / flops_per_candidate(wl)["total"])
+    return max(32, min(wl.N, n))
+
+
+def cpu_baseline(wl, pre=None):
+    oracle, table, req, ids, threads = pre or oracle_setup(wl)
+    n = oracle_sample_size(wl)
+    t0 = time.perf_counter()
+    oracle.score(table, req, ids[:n])
+    dt = time.perf_counter() - t0
+    return {"value": n / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"first {n} candidates of request 0 of {wl.name}, scored once ({dt:.2f} s)",
+            "ms_per_1e4_candidates": 1e4 * dt / n * 1e3}
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    pre = oracle_setup(wl)
+    oracle, table, req, ids, threads = pre
+    # size the per-step sample so that warm-up + K steps end within about two minutes on this host
+    per_step_core_s = min(4.0, 110.0 * threads / max(1, args.steps + args.warmup))
+    n = max(32, oracle_sample_size(wl, core_seconds=per_step_core_s))
+    for _ in range(args.warmup):
+        oracle.score(table, req, ids[:n])
+    times = []
+    for _ in range(args.steps):
+        t0 = time.perf_counter()
+        oracle.score(table, req, ids[:n])
+        times.append(time.perf_counter() - t0)
+    total = sum(times)
+    value = n * args.steps / total
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "candidates_per_step": n, "note": "CPU oracle, bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": f"first {n} candidates of request 0 of {wl.name} per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------------------------------------
+def replica_plan(world: int, rank: int) -> dict:
+    """Multi-GPU plan: the path does not shard, every rank is an independent replica of the whole workload."""
+    return {"rank": rank, "world": world, "replica": True, "share_of_work": 1.0}
+
+
+def reduce_max(value: float, dist=None) -> float:
+    """Max over ranks of a scalar (device-side when NCCL is the backend)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return value
+    import torch
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([value], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def run_ours(args, wl):
+    import torch
+    from paper_2511_12934_b200 import binding as B
+    from paper_2511_12934_b200 import build as libbuild
+    from paper_2511_12934_b200 import serving
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    plan = replica_plan(world, rank)
+    libbuild.build()
+
+    path = {"auto": B.PATH_AUTO, "simt": B.PATH_SIMT, "tensor": B.PATH_TENSOR}[args.path]
+    weights = synth.make_weights(wl)
+    table = synth.make_item_table(wl)
+    batch = wl.R > 1
+    pool = 1 if batch else 8                      # distinct requests cycled over the steps (single-request workload)
+    n_states = wl.R if batch else pool
+    srv = serving.Server(wl, weights, table, path=path, max_user_states=n_states,
+                         max_batch_candidates=wl.R * wl.N if batch else wl.N)
+    sampler = synth.IdSampler(wl)
+    states, id_lists = [], []
+    for r in range(n_states):
+        rq = synth.make_request(wl, r)
+        states.append(srv.precompute(r, srv.upload_request(rq, B.USER_PROJECTED)))
+        id_lists.append(sampler.request_ids(r))
+    torch.cuda.synchronize()
+    if batch:
+        offs = np.zeros(wl.R + 1, dtype=np.int64)
+        offs[1:] = np.cumsum([len(x) for x in id_lists])
+        ids_dev = [torch.from_numpy(np.concatenate(id_lists)).cuda()]
+        cands = int(offs[-1])
+    else:
+        ids_dev = [torch.from_numpy(x).cuda() for x in id_lists]
+        cands = wl.N
+    logits = torch.empty(cands, dtype=torch.float32, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > L2 (126 MB)
+
+    def step(i):
+        if batch:
+            srv.ctx.score_batch(states, ids_dev[0], offs, logits)
+        else:
+            srv.ctx.score(states[i % pool], ids_dev[i % pool], logits)
+
+    def timed(n_steps, fn):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_steps)]
+        for i in range(n_steps):
+            flush.zero_()
+            ev[i][0].record()
+            fn(i)
+            ev[i][1].record()
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in ev]
+
+    for i in range(max(3, args.warmup)):
+        flush.zero_()
+        step(i)
+    torch.cuda.synchronize()
+    uuid = str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
+    sampler_proc = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = B.kernel_launches()
+    times = timed(args.steps, step)
+    launches = B.kernel_launches() - launches0
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    total_ms = reduce_max(sum(times), dist)
+
+    # end to end: host ids in, host logits out, through aif_score_host (one call per request)
+    host_ids = [torch.from_numpy(x).pin_memory() for x in id_lists]
+    host_out = [torch.empty(len(x), dtype=torch.float32).pin_memory() for x in id_lists]
+
+    def step_e2e(i):
+        if batch:
+            for r in range(wl.R):
+                srv.ctx.score_host(states[r], host_ids[r], host_out[r])
+        else:
+            srv.ctx.score_host(states[i % pool], host_ids[i % pool], host_out[i % pool])
+
+    e2e_steps = max(3, min(args.steps, 50))
+    step_e2e(0)
+    e2e_times = timed(e2e_steps, step_e2e)
+    e2e_ms = reduce_max(sum(e2e_times), dist)
+    clocks = sampler_proc.stop()
+
+    # per-kernel durations (events inside the library), for the roofline of the dominant kernel
+    srv.ctx.set_kernel_timing(True)
+    ksum, kcount = {}, 0
+    for i in range(min(args.steps, 50)):
+        flush.zero_()
+        step(i)
+        for k, v in srv.ctx.get_kernel_timing().items():
+            ksum[k] = ksum.get(k, 0.0) + v
+        kcount += 1
+    srv.ctx.set_kernel_timing(False)
+    kavg = {k: v / kcount for k, v in ksum.items()}
+    assert srv.ctx.poll_status() == 0, "device status word set during the benchmark"
+
+    peaks, peak_kind = load_peaks()
+    top = max(kavg, key=kavg.get)
+    tensor = bool(srv.ctx.get_stats().tensor_path) and top != "interact"
+    kf = kernel_flops(top, wl, cands)
+    if tensor:
+        peak = float(peaks["bf16_tflops"])
+        roof = {"bound": "tensor", "kernel": top, "achieved": kf / (kavg[top] * 1e-3) / 1e12, "peak": peak,
+                "unit": "TFLOP/s", "peak_kind": f"bf16 burst, {peak_kind}"}
+    else:
+        roof = {"bound": "alu", "kernel": top, "achieved": kf / (kavg[top] * 1e-3) / 1e12, "peak": FP32_FMA_PEAK_TFLOPS,
+                "unit": "TFLOP/s", "peak_kind": "fp32 FMA: 148 SMs x 128 lanes x 2 x 1.965 GHz"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((wl.name, top))
+    roof["kernel_ms"] = kavg
+
+    value = world * cands * args.steps / (total_ms * 1e-3)
+    per_request_ms = [t / (wl.R if batch else 1) for t in times]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "requests_per_step": wl.R, "candidates_per_step": cands, "M": wl.M, "d": wl.d,
+                   "L": wl.L, "F": wl.F, "hidden": list(wl.hidden), "mini_batch": wl.mini_batch,
+                   "l2": "flushed between timed steps (256 MiB memset)", "parallelism": "replicas only" if world > 1 else "1 GPU",
+                   "path": "tensor" if srv.ctx.get_stats().tensor_path else "cuda-core",
+                   "request_pool": pool},
+        "p50_ms_per_request": float(np.percentile(per_request_ms, 50)),
+        "p99_ms_per_request": float(np.percentile(per_request_ms, 99)),
+        "flops_per_candidate": flops_per_candidate(wl)["total"],
+        "e2e": {"value": world * cands * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * cands,
+                "d2h_bytes_per_step": 4 * cands, "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roof,
+        "replica_plan": plan,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl)
+    if rank == 0:
+        print(json.dumps(line))
+    srv.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(synth.SHORT))
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = synth.SHORT[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

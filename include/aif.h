@@ -81,7 +81,7 @@ typedef struct {
     uint32_t struct_size;          /* sizeof(aif_config), checked */
     int32_t dtype;                 /* AIF_F32 | AIF_BF16 */
     int64_t M;                     /* rows of the item table, 0 < M < 2^31 */
-    int32_t d;                     /* width of item and user vectors; multiple of 8; <= 256 */
+    int32_t d;                     /* width of item and user vectors; multiple of 32; <= 256 */
     int32_t dU;                    /* width of the raw user embeddings of eq. 1; multiple of 4 */
     int32_t L_max;                 /* longest behaviour sequence a user state can hold */
     int32_t F, B, dc;              /* cross fields, buckets per field, width of one cross embedding (multiple of 8) */
@@ -224,6 +224,14 @@ int aif_gather_rows(aif_ctx *ctx, const int32_t *ids, int64_t n, void *rows_out,
 int aif_poll_status(aif_ctx *ctx, uint32_t *bits);
 
 int aif_get_stats(aif_ctx *ctx, aif_stats *out);
+
+/* Per-kernel timing of scoring calls, for roofline measurements.  While on, every scoring call brackets each of
+ * its kernels with CUDA events on the call's stream (a few microseconds of overhead per kernel, so leave it off
+ * for throughput runs).  aif_get_kernel_timing synchronises on the last scoring call and returns, for that call,
+ * the number of kernels (<= 8), their names (static strings) and their durations in milliseconds.
+ * names / ms: host arrays of 8 entries. */
+int aif_set_kernel_timing(aif_ctx *ctx, int on);
+int aif_get_kernel_timing(aif_ctx *ctx, int32_t *n, const char **names, float *ms);
 
 /* Number of kernels this library has launched in this process (all contexts). */
 uint64_t aif_kernel_launches(void);

@@ -74,7 +74,7 @@ EXPORTS = [
     "aif_input_width", "aif_mix64", "aif_create", "aif_destroy", "aif_load_weights", "aif_item_nearline_refresh",
     "aif_user_precompute", "aif_user_release", "aif_user_request_key", "aif_user_state_export", "aif_score",
     "aif_score_batch", "aif_score_host", "aif_gather_rows", "aif_poll_status", "aif_get_stats",
-    "aif_kernel_launches", "aif_strerror", "aif_last_error",
+    "aif_set_kernel_timing", "aif_get_kernel_timing", "aif_kernel_launches", "aif_strerror", "aif_last_error",
 ]
 
 _lib = None
@@ -106,6 +106,8 @@ def load_library(path: Optional[str] = None):
     lib.aif_gather_rows.argtypes = [vp, vp, i64, vp, vp]
     lib.aif_poll_status.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.aif_get_stats.argtypes = [vp, C.POINTER(aif_stats)]
+    lib.aif_set_kernel_timing.argtypes = [vp, C.c_int]
+    lib.aif_get_kernel_timing.argtypes = [vp, C.POINTER(i32), C.POINTER(C.c_char_p), C.POINTER(C.c_float)]
     lib.aif_kernel_launches.argtypes, lib.aif_kernel_launches.restype = [], u64
     lib.aif_strerror.argtypes, lib.aif_strerror.restype = [C.c_int], C.c_char_p
     lib.aif_last_error.argtypes, lib.aif_last_error.restype = [], C.c_char_p
@@ -293,6 +295,17 @@ class Aif:
         bits = C.c_uint32()
         _check(self.lib.aif_poll_status(self.h, C.byref(bits)), "aif_poll_status")
         return int(bits.value)
+
+    def set_kernel_timing(self, on: bool):
+        _check(self.lib.aif_set_kernel_timing(self.h, 1 if on else 0), "aif_set_kernel_timing")
+
+    def get_kernel_timing(self) -> dict:
+        """{kernel name: milliseconds} of the last scoring call (timing must be on)."""
+        n = C.c_int32()
+        names = (C.c_char_p * 8)()
+        ms = (C.c_float * 8)()
+        _check(self.lib.aif_get_kernel_timing(self.h, C.byref(n), names, ms), "aif_get_kernel_timing")
+        return {names[i].decode(): float(ms[i]) for i in range(n.value)}
 
     def get_stats(self) -> aif_stats:
         s = aif_stats()

@@ -108,6 +108,23 @@ int run_score(aif_ctx *ctx, const ScoreLaunch &sl, int64_t total, cudaStream_t s
 
 namespace aif {
 
+void timing_begin(const aif_ctx *ctx, cudaStream_t st)
+{
+    KernelTiming &t = ctx->timing;
+    if (!t.on) return;
+    t.n = 0;
+    cudaEventRecord(t.ev[0], st);
+}
+
+void timing_mark(const aif_ctx *ctx, const char *name, cudaStream_t st)
+{
+    KernelTiming &t = ctx->timing;
+    if (!t.on || t.n >= KernelTiming::kMax) return;
+    t.names[t.n] = name;
+    t.n += 1;
+    cudaEventRecord(t.ev[t.n], st);
+}
+
 ModelDev make_model(const aif_ctx *ctx)
 {
     const aif_config &c = ctx->cfg;
@@ -275,6 +292,8 @@ int aif_destroy(aif_ctx *ctx)
     cudaDeviceSynchronize();
     for (auto &hs : ctx->slots)
         if (hs.ev) cudaEventDestroy(hs.ev);
+    for (int i = 0; i <= KernelTiming::kMax; ++i)
+        if (ctx->timing.ev[i]) cudaEventDestroy(ctx->timing.ev[i]);
     for (int i = 0; i < PinnedRing::kSlots; ++i) {
         if (ctx->ring.host[i]) cudaFreeHost(ctx->ring.host[i]);
         if (ctx->ring.ev[i]) cudaEventDestroy(ctx->ring.ev[i]);
@@ -511,6 +530,34 @@ int aif_get_stats(aif_ctx *ctx, aif_stats *out)
     ctx->stats.device_bytes = ctx->device_bytes;
     ctx->stats.tensor_path = ctx->tensor_path ? 1 : 0;
     *out = ctx->stats;
+    return AIF_OK;
+}
+
+int aif_set_kernel_timing(aif_ctx *ctx, int on)
+{
+    if (!ctx) return AIF_ERR_ARG;
+    DeviceGuard g(ctx->device);
+    KernelTiming &t = ctx->timing;
+    if (on && !t.ev[0])
+        for (int i = 0; i <= KernelTiming::kMax; ++i) AIF_CUDA(cudaEventCreate(&t.ev[i]));
+    t.on = on != 0;
+    t.n = 0;
+    return AIF_OK;
+}
+
+int aif_get_kernel_timing(aif_ctx *ctx, int32_t *n, const char **names, float *ms)
+{
+    if (!ctx || !n || !names || !ms) return AIF_ERR_ARG;
+    DeviceGuard g(ctx->device);
+    KernelTiming &t = ctx->timing;
+    *n = 0;
+    if (!t.on || t.n == 0) return AIF_OK;
+    AIF_CUDA(cudaEventSynchronize(t.ev[t.n]));
+    for (int i = 0; i < t.n; ++i) {
+        AIF_CUDA(cudaEventElapsedTime(&ms[i], t.ev[i], t.ev[i + 1]));
+        names[i] = t.names[i];
+    }
+    *n = t.n;
     return AIF_OK;
 }
 

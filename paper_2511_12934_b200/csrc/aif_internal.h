@@ -81,6 +81,15 @@ struct HostSlot {
 
 constexpr int kUserPartials = 1184;   // warps of the self-attention launch (148 SMs x 8)
 
+// Optional per-kernel timing of the last scoring call (events on the call's stream).
+struct KernelTiming {
+    static constexpr int kMax = 8;
+    bool on = false;
+    int n = 0;
+    cudaEvent_t ev[kMax + 1] = {};
+    const char *names[kMax] = {};
+};
+
 struct PinnedRing {
     static constexpr int kSlots = 8;
     ReqDev *host[kSlots] = {};
@@ -136,6 +145,7 @@ struct aif_ctx {
     aif::PinnedRing ring;
 
     aif_stats stats{};
+    mutable aif::KernelTiming timing;
     std::vector<void *> allocations;
 };
 
@@ -143,6 +153,10 @@ namespace aif {
 
 extern std::atomic<uint64_t> g_launches;
 inline void count_launch(int n = 1) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+// Timing marks: begin(st) before the first kernel of a scoring call, mark(name, st) after each kernel.
+void timing_begin(const aif_ctx *ctx, cudaStream_t st);
+void timing_mark(const aif_ctx *ctx, const char *name, cudaStream_t st);
 
 ModelDev make_model(const aif_ctx *ctx);
 

@@ -490,6 +490,7 @@ cudaError_t launch_score_simt(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStr
     const size_t smem = simt_smem_bytes(ctx, max_h);
     const ModelDev md = make_model(ctx);
     cudaError_t e;
+    timing_begin(ctx, st);
     if (ctx->cfg.dtype == AIF_F32) {
         e = cudaFuncSetAttribute(k_score_simt<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -500,6 +501,7 @@ cudaError_t launch_score_simt(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStr
         k_score_simt<__nv_bfloat16><<<sl.n_tiles, kSimtThreads, smem, st>>>(md, sl, max_h);
     }
     count_launch();
+    timing_mark(ctx, "score_simt", st);
     return cudaGetLastError();
 }
 
