@@ -266,7 +266,13 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     // scratch
     TRY(dev_alloc(ctx, (void **)&ctx->ids_stage, (size_t)c.max_batch_candidates * 4, false));
     TRY(dev_alloc(ctx, (void **)&ctx->logits_stage, (size_t)c.max_batch_candidates * 4, false));
-    if (ctx->tensor_path) TRY(dev_alloc(ctx, &ctx->att_scratch, (size_t)(c.max_batch_candidates + kTcTile) * c.d * 2, true));
+    if (ctx->tensor_path) {
+        cudaError_t e = tc_prepare_context(ctx);
+        if (e != cudaSuccess) {
+            aif_destroy(ctx);
+            return e == cudaErrorMemoryAllocation ? AIF_ERR_OOM : cuda_fail(e, "tensor-path setup");
+        }
+    }
 
     // pinned ring for the request table of aif_score_batch
     ctx->ring.capacity = c.max_user_states;
@@ -298,6 +304,7 @@ int aif_destroy(aif_ctx *ctx)
         if (ctx->ring.host[i]) cudaFreeHost(ctx->ring.host[i]);
         if (ctx->ring.ev[i]) cudaEventDestroy(ctx->ring.ev[i]);
     }
+    if (ctx->tc_plan) tc_destroy_context(ctx);
     for (void *p : ctx->allocations) cudaFree(p);
     cudaGetLastError();
     delete ctx;

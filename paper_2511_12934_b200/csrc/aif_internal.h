@@ -141,7 +141,7 @@ struct aif_ctx {
     // scratch owned by the context
     int32_t *ids_stage = nullptr;     // device staging of host ids (aif_score_host)
     float *logits_stage = nullptr;
-    void *att_scratch = nullptr;      // [max_batch_candidates x d] bf16: attention output between the two tensor kernels
+    void *tc_plan = nullptr;          // tensor-core path: packed weights, tensor maps, activation scratch
     aif::PinnedRing ring;
 
     aif_stats stats{};
@@ -172,6 +172,8 @@ int simt_tiles_for(const aif_ctx *ctx, int n);
 
 // tensor-core path (aif_tc.cu)
 bool tc_supported(const aif_config &cfg);
+cudaError_t tc_prepare_context(aif_ctx *ctx);
+void tc_destroy_context(aif_ctx *ctx);
 cudaError_t tc_prepare_weights(aif_ctx *ctx, const aif_weights *w, cudaStream_t st);
 cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t total_candidates, cudaStream_t st);
 int tc_tiles_for(const aif_ctx *ctx, int n);

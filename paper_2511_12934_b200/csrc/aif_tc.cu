@@ -1,12 +1,739 @@
-// Tensor-core (tcgen05) scoring kernels.  Placeholder until the kernels land: reports "unsupported" so that every
-// configuration runs on the CUDA-core kernels.
+// Tensor-core scoring path for sm_100a (bf16 storage): the scoring MLP as tcgen05 GEMMs with a fused gather
+// prologue and fused epilogues.
+//
+// One layer = one persistent kernel (k_layer_tc).  A work item is (128-candidate tile, 256-wide slice of the
+// layer's outputs).  Roles inside a CTA of 320 threads:
+//   warps 0-3  epilogue: read the fp32 accumulator from TMEM (tcgen05.ld), add the bias (for the first layer the
+//              request's cached user partial p_u), ReLU, then either store bf16 activations for the next layer or
+//              reduce against w_out and write the logit
+//   warp  4    allocates TMEM; one lane issues tcgen05.mma (M=128, N<=256, K=16, bf16 in, fp32 accumulate)
+//   warps 5-8  A producer: gathers the tile's input rows chunk by chunk (64 columns = 128 bytes per row) with
+//              16-byte cp.async into the 128B-swizzled K-major layout the MMA reads: item-table rows by candidate
+//              id, cross-feature rows by (field, bucket(id, field)) from the request's pre-cache, dense rows
+//              (attention output, previous activations) by candidate position
+//   warp  9    B producer: one lane streams the weight slice with TMA (cp.async.bulk.tensor, 128B swizzle)
+// A four-stage shared-memory ring (mbarriers) decouples producers from the MMA; two TMEM accumulators of 256
+// columns let the epilogue of one item overlap the main loop of the next.  Every wait is bounded: on expiry the
+// CTA raises AIF_STATUS_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel returns.
+#include <cuda.h>
+
+#include "aif_device.cuh"
 #include "aif_internal.h"
 
 namespace aif {
+namespace {
 
-bool tc_supported(const aif_config &) { return false; }
-cudaError_t tc_prepare_weights(aif_ctx *, const aif_weights *, cudaStream_t) { return cudaSuccess; }
-cudaError_t launch_score_tc(const aif_ctx *, const ScoreLaunch &, int64_t, cudaStream_t) { return cudaErrorNotSupported; }
-int tc_tiles_for(const aif_ctx *, int) { return 0; }
+constexpr int kStages = 4;
+constexpr int kABytes = kTcTile * 128;    // one A chunk: 128 rows x 64 bf16
+constexpr int kBBytes = 256 * 128;        // one B chunk: up to 256 weight rows x 64 bf16
+constexpr int kThreads = 320;
+constexpr int kLookahead = 2;             // A chunks a producer thread keeps in flight beyond the one it signals
+constexpr int kMaxChunks = 64;
+constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 1.9 GHz
+
+enum { SRC_ITEM = 0, SRC_DENSE = 1, SRC_CROSS = 2 };
+enum { EPI_STORE = 0, EPI_DOT = 1 };
+
+struct ChunkSrc {
+    int32_t kind;
+    int32_t off;   // ITEM / DENSE: byte offset inside the source row; CROSS: first cross column of the chunk
+};
+
+struct LayerParams {
+    ScoreLaunch sl;
+    int32_t n_nchunks, n_cols, n_k, mini_batch;
+    // A sources
+    const uint8_t *E;
+    int64_t M;
+    int32_t e_row_bytes;
+    int32_t x_row_bytes;
+    const uint8_t *X;             // dense rows, indexed by candidate position in the launch
+    int32_t B, dc, bucket_mode, b_mask;
+    int32_t check_ids;            // first layer: flag ids outside the table
+    // epilogue
+    int32_t epi, bias_from_slot, emit_sigmoid, out_stride;
+    const float *bias;
+    __nv_bfloat16 *out;           // EPI_STORE: [positions x out_stride]
+    const __nv_bfloat16 *w_out;
+    const float *b_out;
+    ChunkSrc src[kMaxChunks];
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.b32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false if the CTA is aborting or the wait ran out (and then raises the abort flag).
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitCycles) {
+                *abort_flag = 1u;
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(tm), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, 8-row groups 1024 bytes
+// apart.  Fields: start address >> 4 [0,14), leading byte offset >> 4 [16,30) (unused for this layout), stride byte
+// offset >> 4 [32,46), descriptor version 1 [46,48), layout type 2 = SWIZZLE_128B [61,64).
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(1024u >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor of tcgen05.mma.kind::f16: D fp32 [4,6)=1, A bf16 [7,10)=1, B bf16 [10,13)=1, both operands
+// K-major (bits 15, 16 = 0), N >> 3 at [17,23), M >> 4 at [24,29).
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Arrives on the mbarrier once every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread = lane (row), register j = column j.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void named_bar_sync(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+struct TileInfo {
+    ReqDev rq;
+    int start, cnt;
+    int64_t pos0;   // position of the tile's first candidate in the launch (ids / logits / dense rows)
+};
+
+__device__ __forceinline__ TileInfo decode_tile(const LayerParams &p, int tile)
+{
+    TileInfo t;
+    t.rq = find_request(p.sl, tile);
+    tile_range(tile - t.rq.tile_begin, t.rq.n, kTcTile, p.mini_batch, t.start, t.cnt);
+    t.pos0 = t.rq.off + t.start;
+    return t;
+}
+
+// ---- the layer kernel -----------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1) k_layer_tc(const __grid_constant__ CUtensorMap tmapB, const LayerParams p)
+{
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+    unsigned char *smA = base;                          // kStages x 16 KB
+    unsigned char *smB = base + kStages * kABytes;      // kStages x 32 KB
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smB + kStages * kBBytes);
+    uint64_t *full_a = bars, *full_b = bars + kStages, *empty = bars + 2 * kStages;
+    uint64_t *acc_full = bars + 3 * kStages, *acc_empty = acc_full + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+    float *bias_s = reinterpret_cast<float *>(tmem_slot + 4);   // [256]
+    float *wout_s = bias_s + 256;                                // [256]
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_items = p.sl.n_tiles * p.n_nchunks;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(full_a + s), 128);
+            mbar_init(smem_u32(full_b + s), 1);
+            mbar_init(smem_u32(empty + s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(acc_full + b), 1);
+            mbar_init(smem_u32(acc_empty + b), 4);
+        }
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 4) tmem_alloc(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < 4) {
+        // ===================== epilogue =====================
+        const int row = warp * 32 + lane;
+        int it = 0;
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
+            const int tile = item / p.n_nchunks, nc = item - tile * p.n_nchunks, n0 = nc * p.n_cols;
+            const TileInfo t = decode_tile(p, tile);
+            const int buf = it & 1;
+            const float *bias = p.bias_from_slot ? p.sl.slots[t.rq.slot].p_u : p.bias;
+            for (int j = row; j < p.n_cols; j += 128) {
+                bias_s[j] = bias[n0 + j];
+                if (p.epi == EPI_DOT) wout_s[j] = __bfloat162float(p.w_out[n0 + j]);
+            }
+            named_bar_sync(1, 128);
+            if (!mbar_wait(smem_u32(acc_full + buf), (uint32_t)((it >> 1) & 1), abort_flag)) break;
+            tc_fence_after();
+            const bool valid = row < t.cnt;
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * 256);
+            float dot = 0.f;
+            for (int c0 = 0; c0 < p.n_cols; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(taddr + (uint32_t)c0, r);
+                tmem_ld_wait();
+                if (p.epi == EPI_STORE) {
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float a = fmaxf(__uint_as_float(r[2 * j]) + bias_s[c0 + 2 * j], 0.f);
+                        const float b = fmaxf(__uint_as_float(r[2 * j + 1]) + bias_s[c0 + 2 * j + 1], 0.f);
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+                        packed[j] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                    if (valid) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(p.out + (size_t)(t.pos0 + row) * p.out_stride + n0 + c0);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        dot = fmaf(fmaxf(__uint_as_float(r[j]) + bias_s[c0 + j], 0.f), wout_s[c0 + j], dot);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(acc_empty + buf));
+            if (p.epi == EPI_DOT && valid) {
+                float logit = dot + p.b_out[0];
+                if (p.emit_sigmoid) logit = 1.0f / (1.0f + expf(-logit));
+                const int id = p.sl.ids[t.pos0 + row];
+                if (id < 0 || (int64_t)id >= p.M) logit = __int_as_float(0x7fc00000);
+                p.sl.logits[t.pos0 + row] = logit;
+            }
+            named_bar_sync(1, 128);
+        }
+    } else if (warp == 4) {
+        // ===================== MMA issuer =====================
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(kTcTile, p.n_cols);
+            int it = 0;
+            uint32_t fill = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
+                const int buf = it & 1;
+                if (!mbar_wait(smem_u32(acc_empty + buf), (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
+                for (int kc = 0; kc < p.n_k; ++kc, ++fill) {
+                    const int s = fill % kStages;
+                    const uint32_t ph = (fill / kStages) & 1u;
+                    if (!mbar_wait(smem_u32(full_a + s), ph, abort_flag) || !mbar_wait(smem_u32(full_b + s), ph, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint64_t adesc = umma_desc_sw128(smem_u32(smA + s * kABytes));
+                    const uint64_t bdesc = umma_desc_sw128(smem_u32(smB + s * kBBytes));
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)   // 4 x K=16 inside the 64-column chunk: +32 bytes per step
+                        umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kc | k) != 0 ? 1u : 0u);
+                    umma_commit(smem_u32(empty + s));
+                }
+                if (ok) umma_commit(smem_u32(acc_full + buf));
+            }
+        }
+        __syncwarp();
+    } else if (warp < 9) {
+        // ===================== A producer (128 threads) =====================
+        const int pt = tid - 160;
+        const int sub = pt & 7;              // 16-byte slot inside the 128-byte row chunk
+        const int r0 = pt >> 3;              // rows r0, r0+16, ...
+        const uint32_t sw = (uint32_t)((sub ^ (r0 & 7)) << 4);
+        uint32_t fill = 0, signalled = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+            const int tile = item / p.n_nchunks;
+            const TileInfo t = decode_tile(p, tile);
+            const SlotDev *slot = p.sl.slots + t.rq.slot;
+            const uint8_t *Tt = reinterpret_cast<const uint8_t *>(slot->T);
+            int ids[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int row = r0 + 16 * i;
+                int id = -1;
+                if (row < t.cnt) {
+                    id = p.sl.ids[t.pos0 + row];
+                    if (id < 0 || (int64_t)id >= p.M) {
+                        id = -1;
+                        if (p.check_ids && sub == 0) atomicOr(p.sl.status, AIF_STATUS_BAD_ID);
+                    }
+                }
+                ids[i] = id;
+            }
+            for (int kc = 0; kc < p.n_k; ++kc, ++fill) {
+                const int s = fill % kStages;
+                if (!mbar_wait(smem_u32(empty + s), ((fill / kStages) & 1u) ^ 1u, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                const ChunkSrc src = p.src[kc];
+                const uint32_t dst0 = smem_u32(smA + s * kABytes) + (uint32_t)(r0 * 128) + sw;
+                int f = 0, kin = 0;
+                if (src.kind == SRC_CROSS) {
+                    const int col = src.off + sub * 8;
+                    f = col / p.dc;
+                    kin = col - f * p.dc;
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int row = r0 + 16 * i;
+                    const uint8_t *g = p.E;
+                    uint32_t bytes = 0;
+                    if (src.kind == SRC_DENSE) {
+                        if (row < t.cnt) {
+                            g = p.X + (size_t)(t.pos0 + row) * p.x_row_bytes + src.off + sub * 16;
+                            bytes = 16;
+                        }
+                    } else if (ids[i] >= 0) {
+                        bytes = 16;
+                        if (src.kind == SRC_ITEM) {
+                            g = p.E + (size_t)ids[i] * p.e_row_bytes + src.off + sub * 16;
+                        } else {
+                            int bk;
+                            if (p.bucket_mode == AIF_BUCKET_MOD) bk = ids[i] % p.B;
+                            else {
+                                const uint64_t h = mix64((uint64_t)ids[i], (uint64_t)f);
+                                bk = p.b_mask >= 0 ? (int)(h & (uint64_t)p.b_mask) : (int)(h % (uint64_t)p.B);
+                            }
+                            g = Tt + (((size_t)f * p.B + bk) * p.dc + kin) * 2;
+                        }
+                    }
+                    cp_async16(dst0 + (uint32_t)(i * 16 * 128), g, bytes);
+                }
+                cp_async_commit();
+                if (fill >= (uint32_t)kLookahead) {
+                    cp_async_wait<kLookahead>();
+                    fence_proxy_async();
+                    mbar_arrive(smem_u32(full_a + (signalled % kStages)));
+                    ++signalled;
+                }
+            }
+        }
+        cp_async_wait<0>();
+        fence_proxy_async();
+        if (ok)
+            for (; signalled < fill; ++signalled) mbar_arrive(smem_u32(full_a + (signalled % kStages)));
+    } else {
+        // ===================== B producer (TMA) =====================
+        if (lane == 0) {
+            uint32_t fill = 0;
+            bool ok = true;
+            const uint32_t bytes = (uint32_t)p.n_cols * 128u;
+            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+                const int tile = item / p.n_nchunks, nc = item - tile * p.n_nchunks;
+                for (int kc = 0; kc < p.n_k; ++kc, ++fill) {
+                    const int s = fill % kStages;
+                    if (!mbar_wait(smem_u32(empty + s), ((fill / kStages) & 1u) ^ 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    mbar_expect_tx(smem_u32(full_b + s), bytes);
+                    tma_load_2d(smem_u32(smB + s * kBBytes), &tmapB, smem_u32(full_b + s), kc * 64, nc * p.n_cols);
+                }
+            }
+        }
+        __syncwarp();
+    }
+
+    // ---- teardown: everybody arrives here, also after an abort
+    if (*abort_flag) {
+        if (tid == 0) atomicOr(p.sl.status, AIF_STATUS_TIMEOUT);
+        // let copies and MMAs that are still in flight land before shared memory and TMEM go away
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem_base, 512);
+}
+
+constexpr size_t kLayerSmem = 1024 + (size_t)kStages * (kABytes + kBBytes) + (3 * kStages + 4) * 8 + 16 + 2 * 256 * 4;
+
+// ---- interaction blocks that feed dense columns (CUDA cores; one warp per candidate) ---------------------------
+// Writes, per candidate position, a bf16 row [ att (d) | v_bea (d) | lsh_din (d) | simtier (64, first n_tiers used) ]
+// holding only the enabled blocks.
+__global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl, __nv_bfloat16 *X, int x_stride)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *qv = reinterpret_cast<float *>(smem_raw);                         // [8][d]
+    uint32_t *sigq = reinterpret_cast<uint32_t *>(qv + 8 * md.d);            // [8][8]
+    int *tiers = reinterpret_cast<int *>(sigq + 64);                         // [8][16]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, d = md.d, dq = d >> 5;
+    const ReqDev rq = find_request(sl, blockIdx.x);
+    int start, cnt;
+    tile_range(blockIdx.x - rq.tile_begin, rq.n, kTcTile, md.mini_batch, start, cnt);
+    const SlotDev slot = sl.slots[rq.slot];
+    const bool do_att = md.blocks & AIF_BLK_ATT, do_bea = md.blocks & AIF_BLK_BEA, do_din = md.blocks & AIF_BLK_LSH_DIN,
+               do_tier = md.blocks & AIF_BLK_SIMTIER, do_lsh = do_din || do_tier;
+    using T = __nv_bfloat16;
+    for (int c = warp; c < cnt; c += 8) {
+        const int64_t pos = rq.off + start + c;
+        const int id = sl.ids[pos];
+        T *xrow = X + (size_t)pos * x_stride;
+        if (id < 0 || (int64_t)id >= md.M) {
+            for (int k = lane; k < x_stride; k += 32) xrow[k] = __float2bfloat16_rn(0.f);
+            continue;
+        }
+        const T *e = reinterpret_cast<const T *>(md.E) + (size_t)id * d;
+        for (int k = lane; k < d; k += 32) qv[warp * d + k] = to_f(e[k]);
+        if (do_lsh && lane < (md.lsh_bits >> 5))
+            sigq[warp * 8 + lane] = reinterpret_cast<const uint32_t *>(md.sig + (size_t)id * (md.lsh_bits >> 3))[lane];
+        if (lane < 16) tiers[warp * 16 + lane] = 0;
+        __syncwarp();
+        float att[8], din[8];
+        if (do_att || do_lsh)
+            warp_interact<T>(qv + warp * d, reinterpret_cast<const T *>(slot.S), slot.L, d, rsqrtf((float)d), do_att, do_lsh,
+                             do_tier, sigq + warp * 8, slot.sigS, md.lsh_bits, md.n_tiers, tiers + warp * 16, att, din);
+        int col = 0;
+        if (do_att) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (q < dq) xrow[col + lane + 32 * q] = __float2bfloat16_rn(att[q]);
+            col += d;
+        }
+        if (do_bea) {
+            const T *wh = reinterpret_cast<const T *>(md.bea_w) + (size_t)id * md.n_bridge;
+            const T *V = reinterpret_cast<const T *>(slot.V);
+            for (int k = lane; k < d; k += 32) {
+                float acc = 0.f;
+                for (int b = 0; b < md.n_bridge; ++b) acc = fmaf(to_f(wh[b]), to_f(V[(size_t)b * d + k]), acc);
+                xrow[col + k] = __float2bfloat16_rn(acc);
+            }
+            col += d;
+        }
+        if (do_din) {
+            const float nrm = md.lsh_din_norm == AIF_NORM_MEAN ? 1.0f / (float)slot.L : 1.0f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (q < dq) xrow[col + lane + 32 * q] = __float2bfloat16_rn(din[q] * nrm);
+            col += d;
+        }
+        if (do_tier) {
+            __syncwarp();
+            const float nrm = md.simtier_norm == AIF_NORM_MEAN ? 1.0f / (float)slot.L : 1.0f;
+            for (int k = lane; k < 64; k += 32)
+                xrow[col + k] = __float2bfloat16_rn(k < md.n_tiers ? (float)tiers[warp * 16 + k] * nrm : 0.f);
+        }
+        __syncwarp();
+    }
+}
+
+// W1 [H1 x Din] -> [H1 x k1pad]: user columns dropped, zero padding at the end.
+__global__ void k_pack_w1(const __nv_bfloat16 *W1, __nv_bfloat16 *out, int H1, int din, int d, int k1, int k1pad)
+{
+    const int64_t total = (int64_t)H1 * k1pad;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int j = (int)(i / k1pad), c = (int)(i - (int64_t)j * k1pad);
+        out[i] = c < k1 ? W1[(size_t)j * din + d + c] : __float2bfloat16_rn(0.f);
+    }
+}
+
+// ---- host side ------------------------------------------------------------------------------------------------
+using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                              const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn()
+{
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(p);
+    }
+    return fn;
+}
+
+struct TcPlan {
+    int n_layers = 0;
+    int k1 = 0, k1pad = 0, x_cols = 0;
+    int n_k[kMaxHidden] = {}, n_cols[kMaxHidden] = {}, n_nchunks[kMaxHidden] = {};
+    ChunkSrc src0[kMaxChunks] = {};
+    CUtensorMap tmap[kMaxHidden];
+    __nv_bfloat16 *W[kMaxHidden] = {};
+    __nv_bfloat16 *H[kMaxHidden] = {};   // activations after layer k (k < last)
+    __nv_bfloat16 *X = nullptr;
+    bool maps_ready = false;
+};
+
+int dense_cols(const aif_config &c)
+{
+    int x = 0;
+    if (c.blocks & AIF_BLK_ATT) x += c.d;
+    if (c.blocks & AIF_BLK_BEA) x += c.d;
+    if (c.blocks & AIF_BLK_LSH_DIN) x += c.d;
+    if (c.blocks & AIF_BLK_SIMTIER) x += 64;
+    return x;
+}
+
+}  // namespace
+
+bool tc_supported(const aif_config &c)
+{
+    if (c.dtype != AIF_BF16 || c.d % 64 != 0) return false;
+    if (c.blocks & AIF_BLK_CROSS) {
+        if ((c.F * c.dc) % 64 != 0 || c.dc % 8 != 0) return false;
+        if (64 % c.dc != 0 && c.dc % 64 != 0) return false;
+    }
+    for (int k = 0; k < c.n_hidden; ++k) {
+        const int H = c.hidden[k];
+        if (H <= 256 ? H % 16 != 0 : H % 256 != 0) return false;
+        if (k + 1 < c.n_hidden && H % 64 != 0) return false;
+    }
+    if (c.hidden[c.n_hidden - 1] > 256) return false;
+    aif_config tmp = c;
+    const int k1 = aif_input_width(&tmp) - c.d;
+    if ((k1 + 63) / 64 > kMaxChunks) return false;
+    return encode_fn() != nullptr;
+}
+
+int tc_tiles_for(const aif_ctx *ctx, int n) { return tiles_of(n, kTcTile, ctx->cfg.mini_batch); }
+
+static TcPlan *plan_of(const aif_ctx *ctx) { return reinterpret_cast<TcPlan *>(ctx->tc_plan); }
+
+// Allocates the tensor-path buffers (called from aif_create through tc_prepare_context).
+cudaError_t tc_prepare_context(aif_ctx *ctx)
+{
+    const aif_config &c = ctx->cfg;
+    TcPlan *pl = new TcPlan();
+    ctx->tc_plan = pl;
+    pl->n_layers = c.n_hidden;
+    pl->k1 = ctx->input_width - c.d;
+    pl->x_cols = dense_cols(c);
+    // chunk list of the first layer, in the column order [e | att | cross | bea | din | simtier]
+    int n = 0, xoff = 0;
+    auto add = [&](int kind, int off) { pl->src0[n].kind = kind, pl->src0[n].off = off, ++n; };
+    for (int o = 0; o < c.d; o += 64) add(SRC_ITEM, o * 2);
+    if (c.blocks & AIF_BLK_ATT) {
+        for (int o = 0; o < c.d; o += 64) add(SRC_DENSE, (xoff + o) * 2);
+        xoff += c.d;
+    }
+    if (c.blocks & AIF_BLK_CROSS)
+        for (int o = 0; o < c.F * c.dc; o += 64) add(SRC_CROSS, o);
+    if (c.blocks & AIF_BLK_BEA) {
+        for (int o = 0; o < c.d; o += 64) add(SRC_DENSE, (xoff + o) * 2);
+        xoff += c.d;
+    }
+    if (c.blocks & AIF_BLK_LSH_DIN) {
+        for (int o = 0; o < c.d; o += 64) add(SRC_DENSE, (xoff + o) * 2);
+        xoff += c.d;
+    }
+    if (c.blocks & AIF_BLK_SIMTIER) add(SRC_DENSE, xoff * 2);
+    pl->k1pad = n * 64;
+    const size_t cap = (size_t)c.max_batch_candidates + kTcTile;
+    auto alloc = [&](void **p, size_t bytes) -> cudaError_t {
+        bytes = (bytes + 255) / 256 * 256;
+        cudaError_t e = cudaMalloc(p, bytes);
+        if (e != cudaSuccess) return e;
+        ctx->allocations.push_back(*p);
+        ctx->device_bytes += (int64_t)bytes;
+        return cudaMemset(*p, 0, bytes);
+    };
+    cudaError_t e;
+    int in_w = pl->k1pad;
+    for (int k = 0; k < c.n_hidden; ++k) {
+        const int H = c.hidden[k];
+        pl->n_k[k] = in_w / 64;
+        pl->n_cols[k] = H <= 256 ? H : 256;
+        pl->n_nchunks[k] = H / pl->n_cols[k];
+        if ((e = alloc((void **)&pl->W[k], (size_t)H * in_w * 2)) != cudaSuccess) return e;
+        if (k + 1 < c.n_hidden && (e = alloc((void **)&pl->H[k], cap * H * 2)) != cudaSuccess) return e;
+        in_w = H;
+    }
+    if (pl->x_cols && (e = alloc((void **)&pl->X, cap * pl->x_cols * 2)) != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_layer_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLayerSmem);
+    if (e != cudaSuccess) return e;
+    // tensor maps over the packed weights: [H x in_w] bf16, box = 64 columns x n_cols rows, 128-byte swizzle
+    EncodeFn enc = encode_fn();
+    if (!enc) return cudaErrorNotSupported;
+    in_w = pl->k1pad;
+    for (int k = 0; k < c.n_hidden; ++k) {
+        const cuuint64_t dims[2] = {(cuuint64_t)in_w, (cuuint64_t)c.hidden[k]};
+        const cuuint64_t strides[1] = {(cuuint64_t)in_w * 2};
+        const cuuint32_t box[2] = {64, (cuuint32_t)pl->n_cols[k]};
+        const cuuint32_t estr[2] = {1, 1};
+        CUresult r = enc(&pl->tmap[k], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pl->W[k], dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+        in_w = c.hidden[k];
+    }
+    pl->maps_ready = true;
+    return cudaSuccess;
+}
+
+void tc_destroy_context(aif_ctx *ctx)
+{
+    delete plan_of(ctx);
+    ctx->tc_plan = nullptr;
+}
+
+cudaError_t tc_prepare_weights(aif_ctx *ctx, const aif_weights *w, cudaStream_t st)
+{
+    const aif_config &c = ctx->cfg;
+    TcPlan *pl = plan_of(ctx);
+    k_pack_w1<<<296, 256, 0, st>>>((const __nv_bfloat16 *)w->W[0], pl->W[0], c.hidden[0], ctx->input_width, c.d, pl->k1,
+                                   pl->k1pad);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    for (int k = 1; k < c.n_hidden; ++k) {
+        e = cudaMemcpyAsync(pl->W[k], w->W[k], (size_t)c.hidden[k] * c.hidden[k - 1] * 2, cudaMemcpyDeviceToDevice, st);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t, cudaStream_t st)
+{
+    if (sl.n_tiles <= 0) return cudaSuccess;
+    const aif_config &c = ctx->cfg;
+    TcPlan *pl = plan_of(ctx);
+    const ModelDev md = make_model(ctx);
+    timing_begin(ctx, st);
+    if (pl->x_cols) {
+        const size_t smem = (size_t)8 * c.d * 4 + 64 * 4 + 128 * 4;
+        k_interact_x<<<sl.n_tiles, 256, smem, st>>>(md, sl, pl->X, pl->x_cols);
+        count_launch();
+        timing_mark(ctx, "interact", st);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    static const char *names[kMaxHidden] = {"layer1", "layer2", "layer3", "layer4"};
+    for (int k = 0; k < c.n_hidden; ++k) {
+        LayerParams p{};
+        p.sl = sl;
+        p.n_nchunks = pl->n_nchunks[k], p.n_cols = pl->n_cols[k], p.n_k = pl->n_k[k], p.mini_batch = c.mini_batch;
+        p.E = (const uint8_t *)ctx->E, p.M = c.M, p.e_row_bytes = c.d * 2;
+        p.B = c.B > 0 ? c.B : 1, p.dc = c.dc > 0 ? c.dc : 8, p.bucket_mode = c.bucket_mode;
+        p.b_mask = (p.B & (p.B - 1)) == 0 ? p.B - 1 : -1;
+        p.check_ids = k == 0;
+        if (k == 0) {
+            p.X = (const uint8_t *)pl->X, p.x_row_bytes = pl->x_cols * 2;
+            for (int i = 0; i < p.n_k; ++i) p.src[i] = pl->src0[i];
+        } else {
+            p.X = (const uint8_t *)pl->H[k - 1], p.x_row_bytes = c.hidden[k - 1] * 2;
+            for (int i = 0; i < p.n_k; ++i) p.src[i].kind = SRC_DENSE, p.src[i].off = i * 128;
+        }
+        const bool last = k + 1 == c.n_hidden;
+        p.epi = last ? EPI_DOT : EPI_STORE;
+        p.bias_from_slot = k == 0, p.bias = ctx->b[k], p.emit_sigmoid = c.emit_sigmoid;
+        p.out = pl->H[k], p.out_stride = c.hidden[k];
+        p.w_out = (const __nv_bfloat16 *)ctx->w_out, p.b_out = ctx->b_out;
+        const int items = sl.n_tiles * p.n_nchunks;
+        const int grid = items < 148 ? items : 148;
+        k_layer_tc<<<grid, kThreads, kLayerSmem, st>>>(pl->tmap[k], p);
+        count_launch();
+        timing_mark(ctx, names[k], st);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
 
 }  // namespace aif
