@@ -215,6 +215,32 @@ int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *st
 int aif_score_host(aif_ctx *ctx, const aif_user_state *state, const int32_t *host_ids, int32_t n,
                    float *host_logits, aif_stream stream);
 
+/* Scoring for callers that cannot allocate device memory.  (The paper has no counterpart to this call; it exists
+ * for deployment reasons only.)  Some hosts of this library never get to call cudaMalloc after start-up: a plug-in
+ * inside a serving process whose memory pool has already claimed the whole GPU, or a request thread that is not
+ * allowed to enter the driver's allocator because an allocation can stall every stream of the device.  A context
+ * normally keeps the activations that pass between its scoring kernels in memory it allocated in aif_create, sized
+ * by max_batch_candidates.  This call runs the same tensor-core kernel chain as aif_score but keeps those
+ * activations in a fixed array that is part of the library image instead, so it allocates nothing and does not
+ * depend on max_batch_candidates.  It calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * Limits: n <= AIF_NOALLOC_MAX_CANDIDATES, and the model's activations (dense interaction columns plus all hidden
+ * layers but the last, 2 bytes each) must fit AIF_NOALLOC_ROW_BYTES per candidate; beyond either the call returns
+ * AIF_ERR_SHAPE and aif_last_error says which.  It also returns AIF_ERR_SHAPE on a context that runs the CUDA-core
+ * kernel (fp32 storage or unsupported shapes): that kernel has no scratch, use aif_score.  The array costs
+ * (AIF_NOALLOC_MAX_CANDIDATES + 128) * AIF_NOALLOC_ROW_BYTES = 4.5 MiB on every GPU that loads the library, until
+ * the process exits.
+ *
+ * The first call on each device looks up the array's device address (once, with that device current); make that
+ * first call before any stream capture begins.  All calls on a device share the one array, and it keeps whatever the
+ * previous call left there: every element a call reads it has written itself earlier in the same call, so nothing
+ * needs clearing, but two calls that overlap on the GPU (different streams, or different contexts) race on it.
+ * Order them on one stream or with events.  Arguments and results are those of aif_score. */
+#define AIF_NOALLOC_MAX_CANDIDATES 1024
+#define AIF_NOALLOC_ROW_BYTES 4096
+int aif_score_noalloc(aif_ctx *ctx, const aif_user_state *state, const int32_t *cand_ids, int32_t n, float *logits,
+                      aif_stream stream);
+
 /* The gather stage alone (Section 1, "indexing the model embedding matrices"): rows_out[i] = table[ids[i]].
  * ids: device int32 [n]; rows_out: device [n x d] storage type.  Bad ids give zero rows and the status bit.
  * Exists so that the gather can be measured against HBM bandwidth by itself. */

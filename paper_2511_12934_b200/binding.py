@@ -24,6 +24,7 @@ BUCKET_MOD, BUCKET_HASH = 0, 1
 NORM_NONE, NORM_MEAN = 0, 1
 PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 USER_RAW, USER_PROJECTED = 0, 1
+NOALLOC_MAX_CANDIDATES, NOALLOC_ROW_BYTES = 1024, 4096
 BLK_ATT, BLK_CROSS, BLK_BEA, BLK_LSH_DIN, BLK_SIMTIER = 1, 2, 4, 8, 16
 
 
@@ -73,7 +74,7 @@ class aif_stats(C.Structure):
 EXPORTS = [
     "aif_input_width", "aif_mix64", "aif_create", "aif_destroy", "aif_load_weights", "aif_item_nearline_refresh",
     "aif_user_precompute", "aif_user_release", "aif_user_request_key", "aif_user_state_export", "aif_score",
-    "aif_score_batch", "aif_score_host", "aif_gather_rows", "aif_poll_status", "aif_get_stats",
+    "aif_score_batch", "aif_score_host", "aif_score_noalloc", "aif_gather_rows", "aif_poll_status", "aif_get_stats",
     "aif_set_kernel_timing", "aif_get_kernel_timing", "aif_kernel_launches", "aif_strerror", "aif_last_error",
 ]
 
@@ -103,6 +104,7 @@ def load_library(path: Optional[str] = None):
     lib.aif_score.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.aif_score_batch.argtypes = [vp, i32, C.POINTER(vp), vp, C.POINTER(i64), vp, vp]
     lib.aif_score_host.argtypes = [vp, vp, vp, i32, vp, vp]
+    lib.aif_score_noalloc.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.aif_gather_rows.argtypes = [vp, vp, i64, vp, vp]
     lib.aif_poll_status.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.aif_get_stats.argtypes = [vp, C.POINTER(aif_stats)]
@@ -275,6 +277,11 @@ class Aif:
     def score(self, state: UserState, cand_ids: torch.Tensor, logits: torch.Tensor, stream=None):
         _check(self.lib.aif_score(self.h, state.handle, _ptr(cand_ids), cand_ids.numel(), _ptr(logits),
                                   _stream(stream)), "aif_score")
+
+    def score_noalloc(self, state: UserState, cand_ids: torch.Tensor, logits: torch.Tensor, stream=None):
+        """aif_score_noalloc: same arguments as score; activations live in the library's fixed device array."""
+        _check(self.lib.aif_score_noalloc(self.h, state.handle, _ptr(cand_ids), cand_ids.numel(), _ptr(logits),
+                                          _stream(stream)), "aif_score_noalloc")
 
     def score_batch(self, states: Sequence[UserState], cand_ids: torch.Tensor, offsets: Sequence[int],
                     logits: torch.Tensor, stream=None):

@@ -108,6 +108,10 @@ int run_score(aif_ctx *ctx, const ScoreLaunch &sl, int64_t total, cudaStream_t s
 
 namespace aif {
 
+int check_user_state(aif_ctx *ctx, const aif_user_state *st) { return state_check(ctx, st); }
+
+void set_last_error(const char *text) { snprintf(g_last_error, sizeof(g_last_error), "%s", text); }
+
 void timing_begin(const aif_ctx *ctx, cudaStream_t st)
 {
     KernelTiming &t = ctx->timing;

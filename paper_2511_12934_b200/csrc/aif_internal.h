@@ -176,6 +176,17 @@ cudaError_t tc_prepare_context(aif_ctx *ctx);
 void tc_destroy_context(aif_ctx *ctx);
 cudaError_t tc_prepare_weights(aif_ctx *ctx, const aif_weights *w, cudaStream_t st);
 cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t total_candidates, cudaStream_t st);
+// The same kernel chain with its intermediate activations in caller-chosen memory.
+struct TcScratch {
+    void *X;               // dense interaction columns, [rows x x_cols] bf16
+    void *H[kMaxHidden];   // activations after hidden layer k (k < last), [rows x hidden[k]] bf16
+};
+size_t tc_scratch_row_bytes(const aif_ctx *ctx);
+void tc_scratch_layout(const aif_ctx *ctx, void *base, size_t rows, TcScratch *out);
+cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, const TcScratch &sc);
+// host-side checks shared by the scoring entry points (aif_api.cu)
+int check_user_state(aif_ctx *ctx, const aif_user_state *st);
+void set_last_error(const char *text);
 int tc_tiles_for(const aif_ctx *ctx, int n);
 
 }  // namespace aif

@@ -689,7 +689,39 @@ cudaError_t tc_prepare_weights(aif_ctx *ctx, const aif_weights *w, cudaStream_t 
     return cudaSuccess;
 }
 
+size_t tc_scratch_row_bytes(const aif_ctx *ctx)
+{
+    const aif_config &c = ctx->cfg;
+    size_t cols = (size_t)plan_of(ctx)->x_cols;
+    for (int k = 0; k + 1 < c.n_hidden; ++k) cols += (size_t)c.hidden[k];
+    return cols * 2;
+}
+
+void tc_scratch_layout(const aif_ctx *ctx, void *base, size_t rows, TcScratch *out)
+{
+    const aif_config &c = ctx->cfg;
+    unsigned char *p = reinterpret_cast<unsigned char *>(base);
+    out->X = p;
+    p += rows * (size_t)plan_of(ctx)->x_cols * 2;
+    for (int k = 0; k < kMaxHidden; ++k) {
+        out->H[k] = nullptr;
+        if (k + 1 < c.n_hidden) {
+            out->H[k] = p;
+            p += rows * (size_t)c.hidden[k] * 2;
+        }
+    }
+}
+
 cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t, cudaStream_t st)
+{
+    TcPlan *pl = plan_of(ctx);
+    TcScratch sc;
+    sc.X = pl->X;
+    for (int k = 0; k < kMaxHidden; ++k) sc.H[k] = pl->H[k];
+    return launch_score_tc_scratch(ctx, sl, st, sc);
+}
+
+cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, const TcScratch &sc)
 {
     if (sl.n_tiles <= 0) return cudaSuccess;
     const aif_config &c = ctx->cfg;
@@ -698,7 +730,7 @@ cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t, 
     timing_begin(ctx, st);
     if (pl->x_cols) {
         const size_t smem = (size_t)8 * c.d * 4 + 64 * 4 + 128 * 4;
-        k_interact_x<<<sl.n_tiles, 256, smem, st>>>(md, sl, pl->X, pl->x_cols);
+        k_interact_x<<<sl.n_tiles, 256, smem, st>>>(md, sl, (__nv_bfloat16 *)sc.X, pl->x_cols);
         count_launch();
         timing_mark(ctx, "interact", st);
         cudaError_t e = cudaGetLastError();
@@ -714,16 +746,16 @@ cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t, 
         p.b_mask = (p.B & (p.B - 1)) == 0 ? p.B - 1 : -1;
         p.check_ids = k == 0;
         if (k == 0) {
-            p.X = (const uint8_t *)pl->X, p.x_row_bytes = pl->x_cols * 2;
+            p.X = (const uint8_t *)sc.X, p.x_row_bytes = pl->x_cols * 2;
             for (int i = 0; i < p.n_k; ++i) p.src[i] = pl->src0[i];
         } else {
-            p.X = (const uint8_t *)pl->H[k - 1], p.x_row_bytes = c.hidden[k - 1] * 2;
+            p.X = (const uint8_t *)sc.H[k - 1], p.x_row_bytes = c.hidden[k - 1] * 2;
             for (int i = 0; i < p.n_k; ++i) p.src[i].kind = SRC_DENSE, p.src[i].off = i * 128;
         }
         const bool last = k + 1 == c.n_hidden;
         p.epi = last ? EPI_DOT : EPI_STORE;
         p.bias_from_slot = k == 0, p.bias = ctx->b[k], p.emit_sigmoid = c.emit_sigmoid;
-        p.out = pl->H[k], p.out_stride = c.hidden[k];
+        p.out = (__nv_bfloat16 *)sc.H[k], p.out_stride = c.hidden[k];
         p.w_out = (const __nv_bfloat16 *)ctx->w_out, p.b_out = ctx->b_out;
         const int items = sl.n_tiles * p.n_nchunks;
         const int grid = items < 148 ? items : 148;
