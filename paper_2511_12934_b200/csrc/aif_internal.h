@@ -142,6 +142,7 @@ struct aif_ctx {
     int32_t *ids_stage = nullptr;     // device staging of host ids (aif_score_host)
     float *logits_stage = nullptr;
     void *tc_plan = nullptr;          // tensor-core path: packed weights, tensor maps, activation scratch
+    void *tc_att_plan = nullptr;      // tensor-core attention: tensor map over the arena's S regions
     aif::PinnedRing ring;
 
     aif_stats stats{};
@@ -174,6 +175,11 @@ int simt_tiles_for(const aif_ctx *ctx, int n);
 bool tc_supported(const aif_config &cfg);
 cudaError_t tc_prepare_context(aif_ctx *ctx);
 void tc_destroy_context(aif_ctx *ctx);
+// tensor-core attention (aif_tc_att.cu)
+bool tc_att_supported(const aif_config &cfg);
+cudaError_t tc_att_prepare(aif_ctx *ctx);
+void tc_att_destroy(aif_ctx *ctx);
+cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, void *X, int x_stride);
 cudaError_t tc_prepare_weights(aif_ctx *ctx, const aif_weights *w, cudaStream_t st);
 cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t total_candidates, cudaStream_t st);
 // The same kernel chain with its intermediate activations in caller-chosen memory.

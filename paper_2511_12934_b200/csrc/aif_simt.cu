@@ -477,6 +477,10 @@ static cudaError_t user_network_typed(const aif_ctx *ctx, HostSlot &hs, int slot
             cudaSuccess)
             return e;
     }
+    {   // zero the rows between L and the end of the last 128-key block, so that block-wise readers see no stale rows
+        const int L_pad = (L + 127) / 128 * 128 < c.L_max ? (L + 127) / 128 * 128 : c.L_max;
+        if (L_pad > L && (e = cudaMemsetAsync(S + (size_t)L * d, 0, (size_t)(L_pad - L) * d * sizeof(T), st)) != cudaSuccess) return e;
+    }
     k_user_finish<T><<<1, 256, 0, st>>>(raw ? 1 : 0, S, L, d, hs.prof_hat, hs.partial, kUserPartials,
                                         (const T *)in->profile, (T *)hs.dev.u, (float *)hs.dev.u32, (const T *)ctx->Wt[0],
                                         ctx->b[0], H1, (float *)hs.dev.p_u);

@@ -19,6 +19,7 @@
 
 #include "aif_device.cuh"
 #include "aif_internal.h"
+#include "aif_tc_ptx.cuh"
 
 namespace aif {
 namespace {
@@ -29,7 +30,6 @@ constexpr int kBBytes = 256 * 128;        // one B chunk: up to 256 weight rows 
 constexpr int kThreads = 320;
 constexpr int kLookahead = 2;             // A chunks a producer thread keeps in flight beyond the one it signals
 constexpr int kMaxChunks = 64;
-constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 1.9 GHz
 
 enum { SRC_ITEM = 0, SRC_DENSE = 1, SRC_CROSS = 2 };
 enum { EPI_STORE = 0, EPI_DOT = 1 };
@@ -58,144 +58,6 @@ struct LayerParams {
     const float *b_out;
     ChunkSrc src[kMaxChunks];
 };
-
-// ---- PTX wrappers ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.b32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
-// Bounded wait.  Returns false if the CTA is aborting or the wait ran out (and then raises the abort flag).
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 0u) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) {
-                *abort_flag = 1u;
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-        "l"(tm), "r"(bar), "r"(c0), "r"(c1)
-        : "memory");
-}
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait()
-{
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, 8-row groups 1024 bytes
-// apart.  Fields: start address >> 4 [0,14), leading byte offset >> 4 [16,30) (unused for this layout), stride byte
-// offset >> 4 [32,46), descriptor version 1 [46,48), layout type 2 = SWIZZLE_128B [61,64).
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)(1024u >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-
-// Instruction descriptor of tcgen05.mma.kind::f16: D fp32 [4,6)=1, A bf16 [7,10)=1, B bf16 [10,13)=1, both operands
-// K-major (bits 15, 16 = 0), N >> 3 at [17,23), M >> 4 at [24,29).
-__host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
-        "}\n" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-// Arrives on the mbarrier once every tcgen05.mma issued so far by this thread has completed.
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
-{
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
-{
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-
-// 32 lanes x 32 consecutive fp32 columns: thread = lane (row), register j = column j.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ void named_bar_sync(int id, int threads)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
 
 struct TileInfo {
     ReqDev rq;
@@ -455,7 +317,7 @@ constexpr size_t kLayerSmem = 1024 + (size_t)kStages * (kABytes + kBBytes) + (3 
 // ---- interaction blocks that feed dense columns (CUDA cores; one warp per candidate) ---------------------------
 // Writes, per candidate position, a bf16 row [ att (d) | v_bea (d) | lsh_din (d) | simtier (64, first n_tiers used) ]
 // holding only the enabled blocks.
-__global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl, __nv_bfloat16 *X, int x_stride)
+__global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl, __nv_bfloat16 *X, int x_stride, int att_done)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *qv = reinterpret_cast<float *>(smem_raw);                         // [8][d]
@@ -466,7 +328,8 @@ __global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl,
     int start, cnt;
     tile_range(blockIdx.x - rq.tile_begin, rq.n, kTcTile, md.mini_batch, start, cnt);
     const SlotDev slot = sl.slots[rq.slot];
-    const bool do_att = md.blocks & AIF_BLK_ATT, do_bea = md.blocks & AIF_BLK_BEA, do_din = md.blocks & AIF_BLK_LSH_DIN,
+    // att_done: the attention columns were already written by the tensor-core attention kernel
+    const bool has_att = md.blocks & AIF_BLK_ATT, do_att = has_att && !att_done, do_bea = md.blocks & AIF_BLK_BEA, do_din = md.blocks & AIF_BLK_LSH_DIN,
                do_tier = md.blocks & AIF_BLK_SIMTIER, do_lsh = do_din || do_tier;
     using T = __nv_bfloat16;
     for (int c = warp; c < cnt; c += 8) {
@@ -487,7 +350,7 @@ __global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl,
         if (do_att || do_lsh)
             warp_interact<T>(qv + warp * d, reinterpret_cast<const T *>(slot.S), slot.L, d, rsqrtf((float)d), do_att, do_lsh,
                              do_tier, sigq + warp * 8, slot.sigS, md.lsh_bits, md.n_tiers, tiers + warp * 16, att, din);
-        int col = 0;
+        int col = (has_att && att_done) ? d : 0;
         if (do_att) {
 #pragma unroll
             for (int q = 0; q < 8; ++q)
@@ -532,23 +395,6 @@ __global__ void k_pack_w1(const __nv_bfloat16 *W1, __nv_bfloat16 *out, int H1, i
 }
 
 // ---- host side ------------------------------------------------------------------------------------------------
-using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                              const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn encode_fn()
-{
-    static EncodeFn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeFn>(p);
-    }
-    return fn;
-}
-
 struct TcPlan {
     int n_layers = 0;
     int k1 = 0, k1pad = 0, x_cols = 0;
@@ -664,11 +510,13 @@ cudaError_t tc_prepare_context(aif_ctx *ctx)
         in_w = c.hidden[k];
     }
     pl->maps_ready = true;
+    if (tc_att_supported(c) && (e = tc_att_prepare(ctx)) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
 void tc_destroy_context(aif_ctx *ctx)
 {
+    if (ctx->tc_att_plan) tc_att_destroy(ctx);
     delete plan_of(ctx);
     ctx->tc_plan = nullptr;
 }
@@ -728,9 +576,16 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
     TcPlan *pl = plan_of(ctx);
     const ModelDev md = make_model(ctx);
     timing_begin(ctx, st);
-    if (pl->x_cols) {
+    const bool att_tc = ctx->tc_att_plan != nullptr;
+    if (att_tc) {
+        cudaError_t e = launch_att_tc(ctx, sl, st, sc.X, pl->x_cols);
+        timing_mark(ctx, "attention", st);
+        if (e != cudaSuccess) return e;
+    }
+    const int other_dense = c.blocks & (AIF_BLK_BEA | AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER);
+    if (pl->x_cols && (!att_tc || other_dense)) {
         const size_t smem = (size_t)8 * c.d * 4 + 64 * 4 + 128 * 4;
-        k_interact_x<<<sl.n_tiles, 256, smem, st>>>(md, sl, (__nv_bfloat16 *)sc.X, pl->x_cols);
+        k_interact_x<<<sl.n_tiles, 256, smem, st>>>(md, sl, (__nv_bfloat16 *)sc.X, pl->x_cols, att_tc ? 1 : 0);
         count_launch();
         timing_mark(ctx, "interact", st);
         cudaError_t e = cudaGetLastError();

@@ -1,0 +1,371 @@
+// Dense target attention on the tensor cores (sm_100a): att_i = softmax(e_i S^T / sqrt(d)) S for a tile of 128
+// candidates against the request's projected behaviour sequence S [L x d] (Section 4.2, first paragraph: similarity
+// of the target item with every historical item, then pooling; here in its dense softmax form).
+//
+// One CTA per 128-candidate tile, 192 threads:
+//   warps 0-3  gather the tile's item rows (the queries) into shared memory, then per key block: read the scores
+//              from TMEM, online softmax in fp32 (one thread per candidate row), write the probabilities as a bf16
+//              A operand into shared memory; finally normalise O and store the attention rows
+//   warp  4    allocates TMEM; one lane issues tcgen05.mma: scores = Q K^T (both K-major), O += P V with V read from
+//              the very same shared-memory tile as K, as an MN-major B operand
+//   warp  5    one lane streams key/value blocks of S with TMA (3-D tensor map over the user-state arena)
+// TMEM: two score buffers (so the softmax of block j overlaps Q K^T of block j+1) and the O accumulator.
+// The running maximum is only raised when a row's block maximum exceeds it by more than 8 (in the log2 domain);
+// then the warp rescales its 32 rows of O in TMEM.  Until then probabilities stay below 2^8, which fp32 sums and
+// bf16 operands hold without loss of accuracy.  Every wait is bounded.
+#include "aif_device.cuh"
+#include "aif_internal.h"
+#include "aif_tc_ptx.cuh"
+
+namespace aif {
+namespace {
+
+constexpr int kAttThreads = 192;
+constexpr int kKvStages = 3;
+
+struct AttParams {
+    ScoreLaunch sl;
+    const uint8_t *E;
+    int64_t M;
+    int32_t mini_batch;
+    int32_t x_stride;        // elements per row of X
+    __nv_bfloat16 *X;        // attention rows go to columns [0, d)
+    float scale_log2;        // log2(e) / sqrt(d)
+};
+
+template <int D, int BN>
+struct AttCfg {
+    static constexpr int kQChunks = D / 64;             // 64-column (128-byte) chunks of a row
+    static constexpr int kQBytes = kQChunks * 128 * 128;
+    static constexpr int kKvChunkBytes = BN * 128;      // one 64-column chunk of a key block
+    static constexpr int kKvBytes = kQChunks * kKvChunkBytes;
+    static constexpr int kPChunks = BN / 64;
+    static constexpr int kPBytes = kPChunks * 128 * 128;
+    static constexpr int kTmemO = 2 * BN;               // column of the O accumulator
+    static constexpr size_t kSmem = 1024 + kQBytes + kKvStages * kKvBytes + 2 * kPBytes + 256;
+};
+
+template <int D, int BN>
+__global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant__ CUtensorMap tmapS, const AttParams p)
+{
+    using C = AttCfg<D, BN>;
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+    unsigned char *smQ = base;
+    unsigned char *smKV = smQ + C::kQBytes;
+    unsigned char *smP = smKV + kKvStages * C::kKvBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smP + 2 * C::kPBytes);
+    uint64_t *kv_full = bars, *kv_empty = bars + kKvStages;
+    uint64_t *s_full = bars + 2 * kKvStages, *p_full = s_full + 2, *pv_done = p_full + 2;
+    uint64_t *q_full = pv_done + 2, *o_final = q_full + 1;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(o_final + 1);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const ReqDev rq = find_request(p.sl, blockIdx.x);
+    int start, cnt;
+    tile_range(blockIdx.x - rq.tile_begin, rq.n, kTcTile, p.mini_batch, start, cnt);
+    const int64_t pos0 = rq.off + start;
+    const int L = p.sl.slots[rq.slot].L;
+    const int nb = (L + BN - 1) / BN;
+
+    if (tid == 0) {
+        for (int s = 0; s < kKvStages; ++s) {
+            mbar_init(smem_u32(kv_full + s), 1);
+            mbar_init(smem_u32(kv_empty + s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(s_full + b), 1);
+            mbar_init(smem_u32(p_full + b), 128);
+            mbar_init(smem_u32(pv_done + b), 1);
+        }
+        mbar_init(smem_u32(q_full), 128);
+        mbar_init(smem_u32(o_final), 1);
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 4) tmem_alloc(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < 4) {
+        // ===================== queries, softmax, output =====================
+        const int row = warp * 32 + lane;
+        {   // gather the item rows of the tile: 8 threads per row, 16 bytes each, 128B-swizzled K-major chunks
+            const int sub = tid & 7, r0 = tid >> 3;
+            const uint32_t sw = (uint32_t)((sub ^ (r0 & 7)) << 4);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = r0 + 16 * i;
+                int id = -1;
+                if (r < cnt) {
+                    id = p.sl.ids[pos0 + r];
+                    if (id < 0 || (int64_t)id >= p.M) id = -1;
+                }
+                const uint8_t *g = p.E + (id >= 0 ? (size_t)id * (D * 2) + sub * 16 : 0);
+#pragma unroll
+                for (int c = 0; c < C::kQChunks; ++c)
+                    cp_async16(smem_u32(smQ + c * 16384) + (uint32_t)(r * 128) + sw, g + c * 128, id >= 0 ? 16u : 0u);
+            }
+            cp_async_commit();
+            cp_async_wait<0>();
+            fence_proxy_async();
+            mbar_arrive(smem_u32(q_full));
+        }
+        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        const float k2 = p.scale_log2;
+        float m_used = -INFINITY, l_sum = 0.f;
+        bool ok = true;
+        for (int j = 0; j < nb; ++j) {
+            const int b = j & 1;
+            const int valid_cols = min(BN, L - j * BN);
+            if (!mbar_wait(smem_u32(s_full + b), (uint32_t)((j >> 1) & 1), abort_flag)) {
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const uint32_t ts = lane_base + (uint32_t)(b * BN);
+            // pass 1: block maximum of the row
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(ts + (uint32_t)c0, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (c0 + i < valid_cols) mx = fmaxf(mx, __uint_as_float(r[i]));
+            }
+            const float mt = mx * k2;
+            if (j == 0) {
+                m_used = mt;
+            } else {
+                const bool need = mt > m_used + 8.0f;
+                if (__any_sync(0xffffffffu, need)) {
+                    // raise the running maximum and rescale this warp's rows of O (rare)
+                    const float m_new = need ? mt : m_used;
+                    const float f = fast_exp2(m_used - m_new);
+                    l_sum *= f;
+                    m_used = m_new;
+                    if (!mbar_wait(smem_u32(pv_done + ((j - 1) & 1)), (uint32_t)(((j - 1) >> 1) & 1), abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c0 = 0; c0 < D; c0 += 32) {
+                        uint32_t r[32];
+                        tmem_ld32(lane_base + (uint32_t)(C::kTmemO + c0), r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+                        tmem_st32(lane_base + (uint32_t)(C::kTmemO + c0), r);
+                    }
+                    tmem_st_wait();
+                }
+            }
+            // the P buffer of block j-2 must have been consumed
+            if (j >= 2 && !mbar_wait(smem_u32(pv_done + b), (uint32_t)(((j - 2) >> 1) & 1), abort_flag)) {
+                ok = false;
+                break;
+            }
+            // pass 2: probabilities -> bf16 A operand in shared memory
+            unsigned char *Pb = smP + b * C::kPBytes;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(ts + (uint32_t)c0, r);
+                tmem_ld_wait();
+                uint32_t packed[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float p0 = (c0 + 2 * i < valid_cols) ? fast_exp2(fmaf(__uint_as_float(r[2 * i]), k2, -m_used)) : 0.f;
+                    const float p1 =
+                        (c0 + 2 * i + 1 < valid_cols) ? fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), k2, -m_used)) : 0.f;
+                    l_sum += p0 + p1;
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                    packed[i] = *reinterpret_cast<const uint32_t *>(&h);
+                }
+                unsigned char *chunk = Pb + (c0 >> 6) * 16384 + row * 128;
+                const int slot0 = (c0 & 63) >> 3;     // first 16-byte slot of these 32 columns inside the 128-byte row
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    *reinterpret_cast<uint4 *>(chunk + (((slot0 + q) ^ (row & 7)) << 4)) =
+                        make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(smem_u32(p_full + b));
+        }
+        if (ok && mbar_wait(smem_u32(o_final), 0u, abort_flag)) {
+            tc_fence_after();
+            const float inv = 1.0f / l_sum;
+            bool good = false;
+            if (row < cnt) {
+                const int id = p.sl.ids[pos0 + row];
+                good = id >= 0 && (int64_t)id < p.M;
+            }
+#pragma unroll 1
+            for (int c0 = 0; c0 < D; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(lane_base + (uint32_t)(C::kTmemO + c0), r);
+                tmem_ld_wait();
+                if (row < cnt) {
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(good ? __uint_as_float(r[2 * i]) * inv : 0.f,
+                                                                       good ? __uint_as_float(r[2 * i + 1]) * inv : 0.f);
+                        packed[i] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.X + (size_t)(pos0 + row) * p.x_stride + c0);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                }
+            }
+        }
+    } else if (warp == 4) {
+        // ===================== MMA issuer =====================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = umma_idesc_bf16(kTcTile, BN);
+            constexpr uint32_t idesc_pv = umma_idesc_bf16_bmn(kTcTile, D);
+            bool ok = mbar_wait(smem_u32(q_full), 0u, abort_flag);
+            tc_fence_after();
+            auto issue_qk = [&](int j) -> bool {
+                const int s = j % kKvStages;
+                if (!mbar_wait(smem_u32(kv_full + s), (uint32_t)((j / kKvStages) & 1), abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)((j & 1) * BN);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint64_t adesc = umma_desc_sw128(smem_u32(smQ + (kk >> 2) * 16384)) + (uint64_t)(2 * (kk & 3));
+                    const uint64_t bdesc =
+                        umma_desc_sw128(smem_u32(smKV + s * C::kKvBytes + (kk >> 2) * C::kKvChunkBytes)) + (uint64_t)(2 * (kk & 3));
+                    umma_bf16(d_tmem, adesc, bdesc, idesc_qk, kk > 0 ? 1u : 0u);
+                }
+                umma_commit(smem_u32(s_full + (j & 1)));
+                return true;
+            };
+            if (ok) ok = issue_qk(0);
+            for (int j = 0; ok && j < nb; ++j) {
+                if (j + 1 < nb && !issue_qk(j + 1)) {
+                    ok = false;
+                    break;
+                }
+                if (!mbar_wait(smem_u32(p_full + (j & 1)), (uint32_t)((j >> 1) & 1), abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const int s = j % kKvStages;
+                const uint32_t o_tmem = tmem_base + (uint32_t)C::kTmemO;
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk) {
+                    const uint64_t adesc =
+                        umma_desc_sw128(smem_u32(smP + (j & 1) * C::kPBytes + (kk >> 2) * 16384)) + (uint64_t)(2 * (kk & 3));
+                    // V: 16 keys further = 16 rows x 128 bytes
+                    const uint64_t bdesc = umma_desc_mn_sw128(smem_u32(smKV + s * C::kKvBytes + kk * 2048), C::kKvChunkBytes);
+                    umma_bf16(o_tmem, adesc, bdesc, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(smem_u32(pv_done + (j & 1)));
+                umma_commit(smem_u32(kv_empty + s));
+            }
+            if (ok) umma_commit(smem_u32(o_final));
+        }
+        __syncwarp();
+    } else {
+        // ===================== key/value producer (TMA) =====================
+        if (lane == 0) {
+            for (int j = 0; j < nb; ++j) {
+                const int s = j % kKvStages;
+                if (!mbar_wait(smem_u32(kv_empty + s), (uint32_t)(((j / kKvStages) & 1) ^ 1), abort_flag)) break;
+                mbar_expect_tx(smem_u32(kv_full + s), (uint32_t)C::kKvBytes);
+#pragma unroll
+                for (int c = 0; c < C::kQChunks; ++c)
+                    tma_load_3d(smem_u32(smKV + s * C::kKvBytes + c * C::kKvChunkBytes), &tmapS, smem_u32(kv_full + s), c * 64,
+                                j * BN, rq.slot);
+            }
+        }
+        __syncwarp();
+    }
+
+    if (*abort_flag) {
+        if (tid == 0) atomicOr(p.sl.status, AIF_STATUS_TIMEOUT);
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem_base, 512);
+}
+
+struct AttPlan {
+    CUtensorMap tmap;
+    int bn = 0;
+};
+
+}  // namespace
+
+bool tc_att_supported(const aif_config &c)
+{
+    return c.dtype == AIF_BF16 && (c.blocks & AIF_BLK_ATT) && (c.d == 128 || c.d == 256) && encode_fn() != nullptr;
+}
+
+// Tensor map over the S regions of all user-state slots: [n_slots][L_max][d] with the slot stride of the arena.
+cudaError_t tc_att_prepare(aif_ctx *ctx)
+{
+    const aif_config &c = ctx->cfg;
+    AttPlan *pl = new AttPlan();
+    ctx->tc_att_plan = pl;
+    pl->bn = c.d == 128 ? 128 : 64;
+    EncodeFn enc = encode_fn();
+    if (!enc) return cudaErrorNotSupported;
+    const cuuint64_t dims[3] = {(cuuint64_t)c.d, (cuuint64_t)c.L_max, (cuuint64_t)c.max_user_states};
+    const cuuint64_t strides[2] = {(cuuint64_t)c.d * 2, (cuuint64_t)ctx->slot_bytes};
+    const cuuint32_t box[3] = {64, (cuuint32_t)pl->bn, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    void *base = const_cast<void *>(ctx->slots[0].dev.S);
+    CUresult r = enc(&pl->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    cudaError_t e;
+    if (c.d == 128)
+        e = cudaFuncSetAttribute(k_att_tc<128, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttCfg<128, 128>::kSmem);
+    else
+        e = cudaFuncSetAttribute(k_att_tc<256, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttCfg<256, 64>::kSmem);
+    return e;
+}
+
+void tc_att_destroy(aif_ctx *ctx)
+{
+    delete reinterpret_cast<AttPlan *>(ctx->tc_att_plan);
+    ctx->tc_att_plan = nullptr;
+}
+
+// Rows a user state's S must have zeroed beyond L so that the last key block reads no stale values.
+int tc_att_key_block(const aif_ctx *ctx)
+{
+    const AttPlan *pl = reinterpret_cast<const AttPlan *>(ctx->tc_att_plan);
+    return pl ? pl->bn : 0;
+}
+
+cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, void *X, int x_stride)
+{
+    const aif_config &c = ctx->cfg;
+    const AttPlan *pl = reinterpret_cast<const AttPlan *>(ctx->tc_att_plan);
+    AttParams p{};
+    p.sl = sl, p.E = (const uint8_t *)ctx->E, p.M = c.M, p.mini_batch = c.mini_batch;
+    p.x_stride = x_stride, p.X = (__nv_bfloat16 *)X;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.d);
+    if (c.d == 128)
+        k_att_tc<128, 128><<<sl.n_tiles, kAttThreads, AttCfg<128, 128>::kSmem, st>>>(pl->tmap, p);
+    else
+        k_att_tc<256, 64><<<sl.n_tiles, kAttThreads, AttCfg<256, 64>::kSmem, st>>>(pl->tmap, p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace aif

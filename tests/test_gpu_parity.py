@@ -221,3 +221,28 @@ def test_full_size_c1_and_sampled_c2():
         _check_logits(got[pick], want, TOL[wl.dtype])
         assert np.isfinite(got).all()
         srv.close()
+
+
+def test_sharp_softmax_exercises_the_running_max_rescaling():
+    """Item vectors x32 and sequence rows x64 (exact in bf16) give scores with a standard deviation of about 5:
+    the softmax is close to one-hot and the running maximum of the tensor-core attention jumps by more than its
+    rescaling threshold between key blocks.  Activations are O(1) here instead of O(0.05), so the bf16 budget is
+    scaled: bf16 intermediates of magnitude A carry about 2^-9 A of rounding error."""
+    wl = helpers.MINI["c4"].with_(name="sharp", R=1, N=300, L=700)
+    weights = synth.make_weights(wl, zero_bias=False)
+    table = synth.make_item_table(wl)
+    table["E"] = synth.to_bf16_bits(synth.bf16_bits_to_f32(table["E"]) * 32.0)
+    rq = synth.make_request(wl, 0)
+    rq["S"] = synth.to_bf16_bits(synth.bf16_bits_to_f32(rq["S"]) * 64.0)
+    srv = serving.Server(wl, weights, table)
+    oracle = helpers.make_oracle(wl, weights, M=table["E"].shape[0])
+    ids = synth.IdSampler(wl).request_ids(0)
+    st = srv.precompute(1, srv.upload_request(rq, B.USER_PROJECTED))
+    want, x = oracle.score(table, helpers.projected_request(wl, rq), ids, return_inputs=True)
+    att = x[:, 2 * wl.d:3 * wl.d]
+    assert np.abs(att).max() > 1.0                      # the attention really is sharp: outputs near single rows of S
+    got = srv.score_ids(st, ids)
+    scale = max(1.0, float(np.abs(want).max()))
+    _check_logits(got, want, 1e-2 * scale)
+    assert srv.ctx.poll_status() == 0
+    srv.close()
