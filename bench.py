@@ -356,8 +356,15 @@ def main():
     ap.add_argument("--workload", default="c2", choices=sorted(synth.SHORT))
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    # scaled copies of a workload, for profiler captures that must stay small (the defaults are the full sizes)
+    ap.add_argument("--requests", type=int, default=0, help="override the number of requests per step")
+    ap.add_argument("--rows", type=int, default=0, help="override the rows of the item table")
     args = ap.parse_args()
     wl = synth.SHORT[args.workload]
+    if args.requests:
+        wl = wl.with_(R=args.requests)
+    if args.rows:
+        wl = wl.with_(M=args.rows)
     if args.impl == "reference":
         run_reference(args, wl)
     else:
