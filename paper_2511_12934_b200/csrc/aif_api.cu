@@ -450,6 +450,7 @@ int aif_score(aif_ctx *ctx, const aif_user_state *state, const int32_t *cand_ids
     sl.slots = ctx->slots_dev, sl.reqs = nullptr, sl.n_req = 1;
     sl.single = ReqDev{state->index, n, 0, 0, 0};
     sl.n_tiles = tiles_for(ctx, n);
+    sl.total = n;
     sl.ids = cand_ids, sl.logits = logits, sl.status = ctx->status;
     return run_score(ctx, sl, n, st);
 }
@@ -486,7 +487,7 @@ int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *st
     }
     AIF_CUDA(cudaMemcpyAsync(ring.dev[slot], ring.host[slot], sizeof(ReqDev) * (size_t)n_req, cudaMemcpyHostToDevice, st));
     ScoreLaunch sl{};
-    sl.slots = ctx->slots_dev, sl.reqs = ring.dev[slot], sl.n_req = n_req, sl.n_tiles = tiles;
+    sl.slots = ctx->slots_dev, sl.reqs = ring.dev[slot], sl.n_req = n_req, sl.n_tiles = tiles, sl.total = total;
     sl.ids = cand_ids, sl.logits = logits, sl.status = ctx->status;
     int rc = run_score(ctx, sl, total, st);
     if (rc != AIF_OK) return rc;

@@ -61,6 +61,7 @@ struct ScoreLaunch {
     ReqDev single;
     int32_t n_req;
     int32_t n_tiles;
+    int64_t total;          // candidates of the launch
     const int32_t *ids;
     float *logits;
     uint32_t *status;
@@ -186,6 +187,7 @@ cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t t
 struct TcScratch {
     void *X;               // dense interaction columns, [rows x x_cols] bf16
     void *H[kMaxHidden];   // activations after hidden layer k (k < last), [rows x hidden[k]] bf16
+    void *xb;              // cross-feature buckets, [rows x F] uint16
 };
 size_t tc_scratch_row_bytes(const aif_ctx *ctx);
 void tc_scratch_layout(const aif_ctx *ctx, void *base, size_t rows, TcScratch *out);

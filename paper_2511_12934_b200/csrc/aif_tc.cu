@@ -1,20 +1,22 @@
 // Tensor-core scoring path for sm_100a (bf16 storage): the scoring MLP as tcgen05 GEMMs with a fused gather
 // prologue and fused epilogues.
 //
-// One layer = one persistent kernel (k_layer_tc).  A work item is (128-candidate tile, 256-wide slice of the
-// layer's outputs).  Roles inside a CTA of 320 threads:
-//   warps 0-3  epilogue: read the fp32 accumulator from TMEM (tcgen05.ld), add the bias (for the first layer the
-//              request's cached user partial p_u), ReLU, then either store bf16 activations for the next layer or
+// One layer = one persistent kernel (k_layer_tc<G>).  A work item is (group of G 128-candidate tiles, 256-wide slice
+// of the layer's outputs).  Roles inside a CTA (G = 1: 320 threads, G = 2: 576 threads):
+//   epilogue   4 warps per tile: read the fp32 accumulator from TMEM (tcgen05.ld), add the bias (for the first layer
+//              the request's cached user partial p_u), ReLU, then either store bf16 activations for the next layer or
 //              reduce against w_out and write the logit
-//   warp  4    allocates TMEM; one lane issues tcgen05.mma (M=128, N<=256, K=16, bf16 in, fp32 accumulate)
-//   warps 5-8  A producer: gathers the tile's input rows chunk by chunk (64 columns = 128 bytes per row) with
+//   MMA        one warp allocates TMEM; one lane issues tcgen05.mma (M=128, N<=256, K=16, bf16 in, fp32 accumulate)
+//   A producer 4 warps per tile: gather the tile's input rows chunk by chunk (64 columns = 128 bytes per row) with
 //              16-byte cp.async into the 128B-swizzled K-major layout the MMA reads: item-table rows by candidate
-//              id, cross-feature rows by (field, bucket(id, field)) from the request's pre-cache, dense rows
-//              (attention output, previous activations) by candidate position
-//   warp  9    B producer: one lane streams the weight slice with TMA (cp.async.bulk.tensor, 128B swizzle)
-// A four-stage shared-memory ring (mbarriers) decouples producers from the MMA; two TMEM accumulators of 256
-// columns let the epilogue of one item overlap the main loop of the next.  Every wait is bounded: on expiry the
-// CTA raises AIF_STATUS_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel returns.
+//              id, cross-feature rows by (field, bucket) from the request's pre-cache with the bucket looked up in
+//              the table k_cross_buckets wrote, dense rows (attention output, previous activations) by position.
+//              Ids of the next item and the sources of the next chunk are fetched ahead of their use.
+//   B producer one lane streams the weight slice with TMA (cp.async.bulk.tensor, 128B swizzle)
+// A shared-memory ring (mbarriers) decouples producers from the MMA.  Two TMEM accumulators of 256 columns: with
+// G = 1 they alternate so that the epilogue of one item overlaps the main loop of the next; with G = 2 each tile of
+// the group owns one and both are fed from the same weight chunk.  Every wait is bounded: on expiry the CTA raises
+// AIF_STATUS_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel returns.
 #include <cuda.h>
 
 #include "aif_device.cuh"
@@ -24,11 +26,8 @@
 namespace aif {
 namespace {
 
-constexpr int kStages = 4;
-constexpr int kABytes = kTcTile * 128;    // one A chunk: 128 rows x 64 bf16
+constexpr int kABytes = kTcTile * 128;    // one A chunk of one tile: 128 rows x 64 bf16
 constexpr int kBBytes = 256 * 128;        // one B chunk: up to 256 weight rows x 64 bf16
-constexpr int kThreads = 320;
-constexpr int kLookahead = 2;             // A chunks a producer thread keeps in flight beyond the one it signals
 constexpr int kMaxChunks = 64;
 
 enum { SRC_ITEM = 0, SRC_DENSE = 1, SRC_CROSS = 2 };
@@ -48,7 +47,8 @@ struct LayerParams {
     int32_t e_row_bytes;
     int32_t x_row_bytes;
     const uint8_t *X;             // dense rows, indexed by candidate position in the launch
-    int32_t B, dc, bucket_mode, b_mask;
+    const uint16_t *xb;           // cross-feature buckets [positions x F], written by k_cross_buckets
+    int32_t F, B, dc;
     int32_t check_ids;            // first layer: flag ids outside the table
     // epilogue
     int32_t epi, bias_from_slot, emit_sigmoid, out_stride;
@@ -57,6 +57,22 @@ struct LayerParams {
     const __nv_bfloat16 *w_out;
     const float *b_out;
     ChunkSrc src[kMaxChunks];
+};
+
+// Geometry of the layer kernel.  G = 128-candidate tiles per work item: with G = 2 one weight chunk in shared memory
+// feeds two tiles (two TMEM accumulators), which halves the weight traffic per candidate; with G = 1 the two
+// accumulators alternate between consecutive items so that the epilogue of one overlaps the main loop of the next.
+template <int G>
+struct LayerCfg {
+    static constexpr int kStages = G == 1 ? 4 : 3;
+    static constexpr int kStageBytes = G * kABytes + kBBytes;
+    static constexpr int kEpiWarps = 4 * G;
+    static constexpr int kMmaWarp = kEpiWarps;
+    static constexpr int kProdWarp0 = kEpiWarps + 1;
+    static constexpr int kProdThreads = 128 * G;
+    static constexpr int kBWarp = kProdWarp0 + 4 * G;
+    static constexpr int kThreads = (kBWarp + 1) * 32;
+    static constexpr size_t kSmem = 1024 + (size_t)kStages * kStageBytes + (3 * kStages + 4) * 8 + 32 + 2 * G * 256 * 4;
 };
 
 struct TileInfo {
@@ -68,33 +84,64 @@ struct TileInfo {
 __device__ __forceinline__ TileInfo decode_tile(const LayerParams &p, int tile)
 {
     TileInfo t;
+    if (tile >= p.sl.n_tiles) {   // the second tile of the last group may not exist
+        t.rq = ReqDev{0, 0, 0, 0, 0};
+        t.start = 0, t.cnt = 0, t.pos0 = 0;
+        return t;
+    }
     t.rq = find_request(p.sl, tile);
     tile_range(tile - t.rq.tile_begin, t.rq.n, kTcTile, p.mini_batch, t.start, t.cnt);
     t.pos0 = t.rq.off + t.start;
     return t;
 }
 
-// ---- the layer kernel -----------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads, 1) k_layer_tc(const __grid_constant__ CUtensorMap tmapB, const LayerParams p)
+// Cross-feature index generation for a whole launch (Section 3.3, "real-time generation" from the candidate's
+// attribute): xb[pos][f] = bucket of candidate pos in field f.  Done once per call so that the layer kernel's gather
+// threads only look the bucket up.
+__global__ void __launch_bounds__(256) k_cross_buckets(const int32_t *__restrict__ ids, int64_t total, int F, int B, int b_mask,
+                                                        int mode, uint16_t *__restrict__ xb)
 {
+    const int64_t n = total * F;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t pos = i / F;
+        const int f = (int)(i - pos * F);
+        const int id = ids[pos];
+        int bk = 0;
+        if (id >= 0) {
+            if (mode == AIF_BUCKET_MOD) bk = id % B;
+            else {
+                const uint64_t h = mix64((uint64_t)id, (uint64_t)f);
+                bk = b_mask >= 0 ? (int)(h & (uint64_t)b_mask) : (int)(h % (uint64_t)B);
+            }
+        }
+        xb[i] = (uint16_t)bk;
+    }
+}
+
+// ---- the layer kernel -----------------------------------------------------------------------------------------
+template <int G>
+__global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __grid_constant__ CUtensorMap tmapB, const LayerParams p)
+{
+    using C = LayerCfg<G>;
+    constexpr int kStages = C::kStages;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-    unsigned char *smA = base;                          // kStages x 16 KB
-    unsigned char *smB = base + kStages * kABytes;      // kStages x 32 KB
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smB + kStages * kBBytes);
+    // stage s: G A chunks (one per tile of the group), then the B chunk
+    uint64_t *bars = reinterpret_cast<uint64_t *>(base + kStages * C::kStageBytes);
     uint64_t *full_a = bars, *full_b = bars + kStages, *empty = bars + 2 * kStages;
     uint64_t *acc_full = bars + 3 * kStages, *acc_empty = acc_full + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
     volatile uint32_t *abort_flag = tmem_slot + 1;
-    float *bias_s = reinterpret_cast<float *>(tmem_slot + 4);   // [256]
-    float *wout_s = bias_s + 256;                                // [256]
+    float *bias_s = reinterpret_cast<float *>(((uintptr_t)(tmem_slot + 4) + 15) & ~(uintptr_t)15);   // [G][256]
+    float *wout_s = bias_s + G * 256;                            // [G][256]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n_items = p.sl.n_tiles * p.n_nchunks;
+    const int n_groups = (p.sl.n_tiles + G - 1) / G;
+    const int n_items = n_groups * p.n_nchunks;
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(full_a + s), 128);
+            mbar_init(smem_u32(full_a + s), C::kProdThreads);
             mbar_init(smem_u32(full_b + s), 1);
             mbar_init(smem_u32(empty + s), 1);
         }
@@ -105,54 +152,71 @@ __global__ void __launch_bounds__(kThreads, 1) k_layer_tc(const __grid_constant_
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4) tmem_alloc(smem_u32(tmem_slot), 512);
+    if (warp == C::kMmaWarp) tmem_alloc(smem_u32(tmem_slot), 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp < 4) {
+    if (warp < C::kEpiWarps) {
         // ===================== epilogue =====================
-        const int row = warp * 32 + lane;
+        const int g = warp >> 2;                     // tile of the group this warp quartet serves
+        const int row = (warp & 3) * 32 + lane;      // TMEM lane = candidate row of the tile
+        float *bs = bias_s + g * 256, *ws = wout_s + g * 256;
         int it = 0;
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
-            const int tile = item / p.n_nchunks, nc = item - tile * p.n_nchunks, n0 = nc * p.n_cols;
-            const TileInfo t = decode_tile(p, tile);
-            const int buf = it & 1;
-            const float *bias = p.bias_from_slot ? p.sl.slots[t.rq.slot].p_u : p.bias;
-            for (int j = row; j < p.n_cols; j += 128) {
-                bias_s[j] = bias[n0 + j];
-                if (p.epi == EPI_DOT) wout_s[j] = __bfloat162float(p.w_out[n0 + j]);
+            const int grp = item / p.n_nchunks, nc = item - grp * p.n_nchunks, n0 = nc * p.n_cols;
+            const int buf = G == 1 ? (it & 1) : g;
+            const uint32_t ph = G == 1 ? (uint32_t)((it >> 1) & 1) : (uint32_t)(it & 1);
+            const TileInfo t = decode_tile(p, grp * G + g);
+            if (t.cnt > 0) {
+                const float *bias = p.bias_from_slot ? p.sl.slots[t.rq.slot].p_u : p.bias;
+                for (int j = row; j < p.n_cols; j += 128) {
+                    bs[j] = bias[n0 + j];
+                    if (p.epi == EPI_DOT) ws[j] = __bfloat162float(p.w_out[n0 + j]);
+                }
             }
-            named_bar_sync(1, 128);
-            if (!mbar_wait(smem_u32(acc_full + buf), (uint32_t)((it >> 1) & 1), abort_flag)) break;
+            named_bar_sync(1 + g, 128);
+            if (!mbar_wait(smem_u32(acc_full + buf), ph, abort_flag)) break;
             tc_fence_after();
             const bool valid = row < t.cnt;
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * 256);
+            const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(buf * 256);
             float dot = 0.f;
-            for (int c0 = 0; c0 < p.n_cols; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(taddr + (uint32_t)c0, r);
-                tmem_ld_wait();
-                if (p.epi == EPI_STORE) {
-                    uint32_t packed[16];
+            if (t.cnt > 0) {
+                for (int c0 = 0; c0 < p.n_cols; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld32(taddr + (uint32_t)c0, r);
+                    tmem_ld_wait();
+                    const float4 *b4 = reinterpret_cast<const float4 *>(bs + c0);
+                    if (p.epi == EPI_STORE) {
+                        uint32_t packed[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float a = fmaxf(__uint_as_float(r[2 * j]) + bias_s[c0 + 2 * j], 0.f);
-                        const float b = fmaxf(__uint_as_float(r[2 * j + 1]) + bias_s[c0 + 2 * j + 1], 0.f);
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-                        packed[j] = *reinterpret_cast<const uint32_t *>(&h);
+                        for (int q = 0; q < 8; ++q) {
+                            const float4 bb = b4[q];
+                            const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q]) + bb.x, 0.f),
+                                                                            fmaxf(__uint_as_float(r[4 * q + 1]) + bb.y, 0.f));
+                            const __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q + 2]) + bb.z, 0.f),
+                                                                            fmaxf(__uint_as_float(r[4 * q + 3]) + bb.w, 0.f));
+                            packed[2 * q] = *reinterpret_cast<const uint32_t *>(&h0);
+                            packed[2 * q + 1] = *reinterpret_cast<const uint32_t *>(&h1);
+                        }
+                        if (valid) {
+                            uint4 *dst = reinterpret_cast<uint4 *>(p.out + (size_t)(t.pos0 + row) * p.out_stride + n0 + c0);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                        }
+                    } else {
+                        const float4 *w4 = reinterpret_cast<const float4 *>(ws + c0);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const float4 bb = b4[q], ww = w4[q];
+                            dot = fmaf(fmaxf(__uint_as_float(r[4 * q]) + bb.x, 0.f), ww.x, dot);
+                            dot = fmaf(fmaxf(__uint_as_float(r[4 * q + 1]) + bb.y, 0.f), ww.y, dot);
+                            dot = fmaf(fmaxf(__uint_as_float(r[4 * q + 2]) + bb.z, 0.f), ww.z, dot);
+                            dot = fmaf(fmaxf(__uint_as_float(r[4 * q + 3]) + bb.w, 0.f), ww.w, dot);
+                        }
                     }
-                    if (valid) {
-                        uint4 *dst = reinterpret_cast<uint4 *>(p.out + (size_t)(t.pos0 + row) * p.out_stride + n0 + c0);
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        dot = fmaf(fmaxf(__uint_as_float(r[j]) + bias_s[c0 + j], 0.f), wout_s[c0 + j], dot);
                 }
             }
             tc_fence_before();
@@ -165,53 +229,71 @@ __global__ void __launch_bounds__(kThreads, 1) k_layer_tc(const __grid_constant_
                 if (id < 0 || (int64_t)id >= p.M) logit = __int_as_float(0x7fc00000);
                 p.sl.logits[t.pos0 + row] = logit;
             }
-            named_bar_sync(1, 128);
+            named_bar_sync(1 + g, 128);
         }
-    } else if (warp == 4) {
+    } else if (warp == C::kMmaWarp) {
         // ===================== MMA issuer =====================
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(kTcTile, p.n_cols);
-            int it = 0;
-            uint32_t fill = 0;
+            int it = 0, s = 0;
+            uint32_t ph = 0;
             bool ok = true;
             for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
-                const int buf = it & 1;
-                if (!mbar_wait(smem_u32(acc_empty + buf), (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag)) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
-                for (int kc = 0; kc < p.n_k; ++kc, ++fill) {
-                    const int s = fill % kStages;
-                    const uint32_t ph = (fill / kStages) & 1u;
+                for (int kc = 0; ok && kc < p.n_k; ++kc) {
                     if (!mbar_wait(smem_u32(full_a + s), ph, abort_flag) || !mbar_wait(smem_u32(full_b + s), ph, abort_flag)) {
                         ok = false;
                         break;
                     }
+                    // the A chunk was written by cp.async (generic proxy) and is read by the MMA (async proxy)
+                    fence_proxy_async();
                     tc_fence_after();
-                    const uint64_t adesc = umma_desc_sw128(smem_u32(smA + s * kABytes));
-                    const uint64_t bdesc = umma_desc_sw128(smem_u32(smB + s * kBBytes));
+                    unsigned char *stage = base + s * C::kStageBytes;
+                    const uint64_t bdesc = umma_desc_sw128(smem_u32(stage + G * kABytes));
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)   // 4 x K=16 inside the 64-column chunk: +32 bytes per step
-                        umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kc | k) != 0 ? 1u : 0u);
+                    for (int g = 0; g < G; ++g) {
+                        const int buf = G == 1 ? (it & 1) : g;
+                        if (kc == 0) {   // the accumulator must have been drained by the epilogue of its previous use
+                            const uint32_t eph = (G == 1 ? (uint32_t)((it >> 1) & 1) : (uint32_t)(it & 1)) ^ 1u;
+                            if (!mbar_wait(smem_u32(acc_empty + buf), eph, abort_flag)) {
+                                ok = false;
+                                break;
+                            }
+                            tc_fence_after();
+                        }
+                        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
+                        const uint64_t adesc = umma_desc_sw128(smem_u32(stage + g * kABytes));
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)   // 4 x K=16 inside the 64-column chunk: +32 bytes per step
+                            umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kc | k) != 0 ? 1u : 0u);
+                        if (kc == p.n_k - 1) umma_commit(smem_u32(acc_full + buf));
+                    }
+                    if (!ok) break;
                     umma_commit(smem_u32(empty + s));
+                    if (++s == kStages) s = 0, ph ^= 1u;
                 }
-                if (ok) umma_commit(smem_u32(acc_full + buf));
             }
         }
         __syncwarp();
-    } else if (warp < 9) {
-        // ===================== A producer (128 threads) =====================
-        const int pt = tid - 160;
+    } else if (warp < C::kBWarp) {
+        // ===================== A producer (128 threads per tile of the group) =====================
+        const int pt = tid - C::kProdWarp0 * 32;
+        const int g = pt >> 7;
         const int sub = pt & 7;              // 16-byte slot inside the 128-byte row chunk
-        const int r0 = pt >> 3;              // rows r0, r0+16, ...
+        const int r0 = (pt & 127) >> 3;      // rows r0, r0+16, ...
         const uint32_t sw = (uint32_t)((sub ^ (r0 & 7)) << 4);
-        uint32_t fill = 0, signalled = 0;
-        bool ok = true;
-        for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-            const int tile = item / p.n_nchunks;
-            const TileInfo t = decode_tile(p, tile);
-            const SlotDev *slot = p.sl.slots + t.rq.slot;
-            const uint8_t *Tt = reinterpret_cast<const uint8_t *>(slot->T);
+        const uint32_t a_off = (uint32_t)(g * kABytes + r0 * 128) + sw;
+
+        struct Rows {
             int ids[8];
+            int cnt;
+            int64_t pos0;
+            const uint8_t *Tt;
+        };
+        auto load_rows = [&](int item, Rows &R) {
+            const int grp = item / p.n_nchunks;
+            const TileInfo t = decode_tile(p, grp * G + g);
+            R.cnt = t.cnt, R.pos0 = t.pos0;
+            R.Tt = t.cnt > 0 ? reinterpret_cast<const uint8_t *>(p.sl.slots[t.rq.slot].T) : nullptr;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int row = r0 + 16 * i;
@@ -223,77 +305,93 @@ __global__ void __launch_bounds__(kThreads, 1) k_layer_tc(const __grid_constant_
                         if (p.check_ids && sub == 0) atomicOr(p.sl.status, AIF_STATUS_BAD_ID);
                     }
                 }
-                ids[i] = id;
+                R.ids[i] = id;
             }
-            for (int kc = 0; kc < p.n_k; ++kc, ++fill) {
-                const int s = fill % kStages;
-                if (!mbar_wait(smem_u32(empty + s), ((fill / kStages) & 1u) ^ 1u, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-                const ChunkSrc src = p.src[kc];
-                const uint32_t dst0 = smem_u32(smA + s * kABytes) + (uint32_t)(r0 * 128) + sw;
-                int f = 0, kin = 0;
-                if (src.kind == SRC_CROSS) {
-                    const int col = src.off + sub * 8;
-                    f = col / p.dc;
-                    kin = col - f * p.dc;
-                }
+        };
+        // global source of this thread's 16 bytes of each of its 8 rows in chunk kc; rows outside `mask` are zero-filled
+        auto sources = [&](int kc, const Rows &R, const uint8_t *(&gp)[8], uint32_t &mask) {
+            const ChunkSrc src = p.src[kc];
+            mask = 0;
+            if (src.kind == SRC_DENSE) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int row = r0 + 16 * i;
-                    const uint8_t *g = p.E;
-                    uint32_t bytes = 0;
-                    if (src.kind == SRC_DENSE) {
-                        if (row < t.cnt) {
-                            g = p.X + (size_t)(t.pos0 + row) * p.x_row_bytes + src.off + sub * 16;
-                            bytes = 16;
-                        }
-                    } else if (ids[i] >= 0) {
-                        bytes = 16;
-                        if (src.kind == SRC_ITEM) {
-                            g = p.E + (size_t)ids[i] * p.e_row_bytes + src.off + sub * 16;
-                        } else {
-                            int bk;
-                            if (p.bucket_mode == AIF_BUCKET_MOD) bk = ids[i] % p.B;
-                            else {
-                                const uint64_t h = mix64((uint64_t)ids[i], (uint64_t)f);
-                                bk = p.b_mask >= 0 ? (int)(h & (uint64_t)p.b_mask) : (int)(h % (uint64_t)p.B);
-                            }
-                            g = Tt + (((size_t)f * p.B + bk) * p.dc + kin) * 2;
-                        }
-                    }
-                    cp_async16(dst0 + (uint32_t)(i * 16 * 128), g, bytes);
+                    gp[i] = p.X + (size_t)(R.pos0 + row) * p.x_row_bytes + src.off + sub * 16;
+                    if (row < R.cnt) mask |= 1u << i;
                 }
-                cp_async_commit();
-                if (fill >= (uint32_t)kLookahead) {
-                    cp_async_wait<kLookahead>();
-                    fence_proxy_async();
-                    mbar_arrive(smem_u32(full_a + (signalled % kStages)));
-                    ++signalled;
+            } else if (src.kind == SRC_ITEM) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    gp[i] = p.E + (size_t)(R.ids[i] >= 0 ? R.ids[i] : 0) * p.e_row_bytes + src.off + sub * 16;
+                    if (R.ids[i] >= 0) mask |= 1u << i;
+                }
+            } else {
+                const int col = src.off + sub * 8;
+                const int f = col / p.dc, kin = col - f * p.dc;
+                const uint16_t *xb = p.xb + (size_t)(R.pos0 + r0) * p.F + f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    int bk = 0;
+                    if (R.ids[i] >= 0) {
+                        bk = __ldg(xb + (size_t)(16 * i) * p.F);
+                        mask |= 1u << i;
+                    }
+                    gp[i] = R.Tt + (((size_t)f * p.B + bk) * p.dc + kin) * 2;
                 }
             }
+        };
+
+        int s = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        Rows cur;
+        const uint8_t *gp[8];
+        uint32_t mask = 0;
+        if ((int)blockIdx.x < n_items) {
+            load_rows(blockIdx.x, cur);
+            sources(0, cur, gp, mask);
         }
-        cp_async_wait<0>();
-        fence_proxy_async();
-        if (ok)
-            for (; signalled < fill; ++signalled) mbar_arrive(smem_u32(full_a + (signalled % kStages)));
+        for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+            const int next_item = item + gridDim.x;
+            Rows nxt = cur;
+            if (next_item < n_items) load_rows(next_item, nxt);   // global loads land while this item's chunks are copied
+            for (int kc = 0; kc < p.n_k; ++kc) {
+                if (!mbar_wait(smem_u32(empty + s), ph ^ 1u, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                const uint32_t dst0 = smem_u32(base + s * C::kStageBytes) + a_off;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    cp_async16(dst0 + (uint32_t)(i * 16 * 128), (mask >> i) & 1u ? gp[i] : p.E, (mask >> i) & 1u ? 16u : 0u);
+                // the stage's barrier receives this thread's arrival when its copies have landed: no thread waits for them
+                cp_async_arrive_noinc(smem_u32(full_a + s));
+                if (++s == kStages) s = 0, ph ^= 1u;
+                // sources of the next chunk: the bucket look-ups are in flight while this thread waits for the next stage
+                if (kc + 1 < p.n_k) sources(kc + 1, cur, gp, mask);
+                else if (next_item < n_items) sources(0, nxt, gp, mask);
+            }
+            cur = nxt;
+        }
+        cp_async_wait_all();
     } else {
         // ===================== B producer (TMA) =====================
         if (lane == 0) {
-            uint32_t fill = 0;
+            int s = 0;
+            uint32_t ph = 0;
             bool ok = true;
             const uint32_t bytes = (uint32_t)p.n_cols * 128u;
             for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-                const int tile = item / p.n_nchunks, nc = item - tile * p.n_nchunks;
-                for (int kc = 0; kc < p.n_k; ++kc, ++fill) {
-                    const int s = fill % kStages;
-                    if (!mbar_wait(smem_u32(empty + s), ((fill / kStages) & 1u) ^ 1u, abort_flag)) {
+                const int grp = item / p.n_nchunks, nc = item - grp * p.n_nchunks;
+                for (int kc = 0; kc < p.n_k; ++kc) {
+                    if (!mbar_wait(smem_u32(empty + s), ph ^ 1u, abort_flag)) {
                         ok = false;
                         break;
                     }
                     mbar_expect_tx(smem_u32(full_b + s), bytes);
-                    tma_load_2d(smem_u32(smB + s * kBBytes), &tmapB, smem_u32(full_b + s), kc * 64, nc * p.n_cols);
+                    tma_load_2d(smem_u32(base + s * C::kStageBytes + G * kABytes), &tmapB, smem_u32(full_b + s), kc * 64,
+                                nc * p.n_cols);
+                    if (++s == kStages) s = 0, ph ^= 1u;
                 }
             }
         }
@@ -309,10 +407,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_layer_tc(const __grid_constant_
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem_base, 512);
+    if (warp == C::kMmaWarp) tmem_dealloc(tmem_base, 512);
 }
-
-constexpr size_t kLayerSmem = 1024 + (size_t)kStages * (kABytes + kBBytes) + (3 * kStages + 4) * 8 + 16 + 2 * 256 * 4;
 
 // ---- interaction blocks that feed dense columns (CUDA cores; one warp per candidate) ---------------------------
 // Writes, per candidate position, a bf16 row [ att (d) | v_bea (d) | lsh_din (d) | simtier (64, first n_tiers used) ]
@@ -404,6 +500,7 @@ struct TcPlan {
     __nv_bfloat16 *W[kMaxHidden] = {};
     __nv_bfloat16 *H[kMaxHidden] = {};   // activations after layer k (k < last)
     __nv_bfloat16 *X = nullptr;
+    uint16_t *xb = nullptr;              // cross-feature buckets [positions x F]
     bool maps_ready = false;
 };
 
@@ -423,7 +520,7 @@ bool tc_supported(const aif_config &c)
 {
     if (c.dtype != AIF_BF16 || c.d % 64 != 0) return false;
     if (c.blocks & AIF_BLK_CROSS) {
-        if ((c.F * c.dc) % 64 != 0 || c.dc % 8 != 0) return false;
+        if ((c.F * c.dc) % 64 != 0 || c.dc % 8 != 0 || c.B > 65536) return false;
         if (64 % c.dc != 0 && c.dc % 64 != 0) return false;
     }
     for (int k = 0; k < c.n_hidden; ++k) {
@@ -492,7 +589,10 @@ cudaError_t tc_prepare_context(aif_ctx *ctx)
         in_w = H;
     }
     if (pl->x_cols && (e = alloc((void **)&pl->X, cap * pl->x_cols * 2)) != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_layer_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLayerSmem);
+    if ((c.blocks & AIF_BLK_CROSS) && (e = alloc((void **)&pl->xb, cap * c.F * 2)) != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_layer_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LayerCfg<1>::kSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_layer_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LayerCfg<2>::kSmem);
     if (e != cudaSuccess) return e;
     // tensor maps over the packed weights: [H x in_w] bf16, box = 64 columns x n_cols rows, 128-byte swizzle
     EncodeFn enc = encode_fn();
@@ -542,6 +642,7 @@ size_t tc_scratch_row_bytes(const aif_ctx *ctx)
     const aif_config &c = ctx->cfg;
     size_t cols = (size_t)plan_of(ctx)->x_cols;
     for (int k = 0; k + 1 < c.n_hidden; ++k) cols += (size_t)c.hidden[k];
+    if (c.blocks & AIF_BLK_CROSS) cols += (size_t)c.F;
     return cols * 2;
 }
 
@@ -558,6 +659,7 @@ void tc_scratch_layout(const aif_ctx *ctx, void *base, size_t rows, TcScratch *o
             p += rows * (size_t)c.hidden[k] * 2;
         }
     }
+    out->xb = (c.blocks & AIF_BLK_CROSS) ? p : nullptr;
 }
 
 cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t, cudaStream_t st)
@@ -565,6 +667,7 @@ cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t, 
     TcPlan *pl = plan_of(ctx);
     TcScratch sc;
     sc.X = pl->X;
+    sc.xb = pl->xb;
     for (int k = 0; k < kMaxHidden; ++k) sc.H[k] = pl->H[k];
     return launch_score_tc_scratch(ctx, sl, st, sc);
 }
@@ -576,6 +679,16 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
     TcPlan *pl = plan_of(ctx);
     const ModelDev md = make_model(ctx);
     timing_begin(ctx, st);
+    if (c.blocks & AIF_BLK_CROSS) {
+        const int64_t n = sl.total * c.F;
+        const int grid = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
+        k_cross_buckets<<<grid, 256, 0, st>>>(sl.ids, sl.total, c.F, c.B, (c.B & (c.B - 1)) == 0 ? c.B - 1 : -1, c.bucket_mode,
+                                              (uint16_t *)sc.xb);
+        count_launch();
+        timing_mark(ctx, "buckets", st);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     const bool att_tc = ctx->tc_att_plan != nullptr;
     if (att_tc) {
         cudaError_t e = launch_att_tc(ctx, sl, st, sc.X, pl->x_cols);
@@ -597,8 +710,7 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
         p.sl = sl;
         p.n_nchunks = pl->n_nchunks[k], p.n_cols = pl->n_cols[k], p.n_k = pl->n_k[k], p.mini_batch = c.mini_batch;
         p.E = (const uint8_t *)ctx->E, p.M = c.M, p.e_row_bytes = c.d * 2;
-        p.B = c.B > 0 ? c.B : 1, p.dc = c.dc > 0 ? c.dc : 8, p.bucket_mode = c.bucket_mode;
-        p.b_mask = (p.B & (p.B - 1)) == 0 ? p.B - 1 : -1;
+        p.B = c.B > 0 ? c.B : 1, p.dc = c.dc > 0 ? c.dc : 8, p.F = c.F, p.xb = (const uint16_t *)sc.xb;
         p.check_ids = k == 0;
         if (k == 0) {
             p.X = (const uint8_t *)sc.X, p.x_row_bytes = pl->x_cols * 2;
@@ -612,9 +724,12 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
         p.bias_from_slot = k == 0, p.bias = ctx->b[k], p.emit_sigmoid = c.emit_sigmoid;
         p.out = (__nv_bfloat16 *)sc.H[k], p.out_stride = c.hidden[k];
         p.w_out = (const __nv_bfloat16 *)ctx->w_out, p.b_out = ctx->b_out;
-        const int items = sl.n_tiles * p.n_nchunks;
+        // two tiles per item once that still leaves every SM at least two items
+        const bool pair = ((sl.n_tiles + 1) / 2) * p.n_nchunks >= 2 * 148;
+        const int items = pair ? ((sl.n_tiles + 1) / 2) * p.n_nchunks : sl.n_tiles * p.n_nchunks;
         const int grid = items < 148 ? items : 148;
-        k_layer_tc<<<grid, kThreads, kLayerSmem, st>>>(pl->tmap[k], p);
+        if (pair) k_layer_tc<2><<<grid, LayerCfg<2>::kThreads, LayerCfg<2>::kSmem, st>>>(pl->tmap[k], p);
+        else k_layer_tc<1><<<grid, LayerCfg<1>::kThreads, LayerCfg<1>::kSmem, st>>>(pl->tmap[k], p);
         count_launch();
         timing_mark(ctx, names[k], st);
         cudaError_t e = cudaGetLastError();
