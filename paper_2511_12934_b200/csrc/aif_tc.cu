@@ -72,7 +72,7 @@ struct LayerCfg {
     static constexpr int kProdThreads = 128 * G;
     static constexpr int kBWarp = kProdWarp0 + 4 * G;
     static constexpr int kThreads = (kBWarp + 1) * 32;
-    static constexpr size_t kSmem = 1024 + (size_t)kStages * kStageBytes + (3 * kStages + 4) * 8 + 32 + 2 * G * 256 * 4;
+    static constexpr size_t kSmem = 1024 + (size_t)kStages * kStageBytes + (3 * kStages + 4) * 8 + 32 + 2 * G * 256 * 4 + kEpiWarps * 2048;
 };
 
 struct TileInfo {
@@ -163,6 +163,7 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
         const int g = warp >> 2;                     // tile of the group this warp quartet serves
         const int row = (warp & 3) * 32 + lane;      // TMEM lane = candidate row of the tile
         float *bs = bias_s + g * 256, *ws = wout_s + g * 256;
+        unsigned char *stg = reinterpret_cast<unsigned char *>(wout_s + G * 256) + warp * 2048;   // 32 rows x 64 bytes
         int it = 0;
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
             const int grp = item / p.n_nchunks, nc = item - grp * p.n_nchunks, n0 = nc * p.n_cols;
@@ -200,12 +201,22 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
                             packed[2 * q] = *reinterpret_cast<const uint32_t *>(&h0);
                             packed[2 * q + 1] = *reinterpret_cast<const uint32_t *>(&h1);
                         }
-                        if (valid) {
-                            uint4 *dst = reinterpret_cast<uint4 *>(p.out + (size_t)(t.pos0 + row) * p.out_stride + n0 + c0);
+                        // through the warp's staging rows so that four lanes store one row's 64 bytes side by side
+                        const int swz = (lane >> 1) & 3;
 #pragma unroll
-                            for (int q = 0; q < 4; ++q)
-                                dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                        for (int q = 0; q < 4; ++q)
+                            *reinterpret_cast<uint4 *>(stg + lane * 64 + ((q ^ swz) << 4)) =
+                                make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int rr = 8 * j + (lane >> 2), q = lane & 3;
+                            const uint4 v = *reinterpret_cast<const uint4 *>(stg + rr * 64 + ((q ^ ((rr >> 1) & 3)) << 4));
+                            const int trow = (warp & 3) * 32 + rr;
+                            if (trow < t.cnt)
+                                *reinterpret_cast<uint4 *>(p.out + (size_t)(t.pos0 + trow) * p.out_stride + n0 + c0 + q * 8) = v;
                         }
+                        __syncwarp();
                     } else {
                         const float4 *w4 = reinterpret_cast<const float4 *>(ws + c0);
 #pragma unroll
@@ -235,11 +246,17 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
         // ===================== MMA issuer =====================
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(kTcTile, p.n_cols);
+            const int n_k = p.n_k;
+            // descriptors of stage 0; stage s lies s * kStageBytes further (the address field counts 16-byte units)
+            const uint64_t bdesc0 = umma_desc_sw128(smem_u32(base + G * kABytes));
+            uint64_t adesc0[G];
+#pragma unroll
+            for (int g = 0; g < G; ++g) adesc0[g] = umma_desc_sw128(smem_u32(base + g * kABytes));
             int it = 0, s = 0;
             uint32_t ph = 0;
             bool ok = true;
             for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
-                for (int kc = 0; ok && kc < p.n_k; ++kc) {
+                for (int kc = 0; kc < n_k; ++kc) {
                     if (!mbar_wait(smem_u32(full_a + s), ph, abort_flag) || !mbar_wait(smem_u32(full_b + s), ph, abort_flag)) {
                         ok = false;
                         break;
@@ -247,8 +264,8 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
                     // the A chunk was written by cp.async (generic proxy) and is read by the MMA (async proxy)
                     fence_proxy_async();
                     tc_fence_after();
-                    unsigned char *stage = base + s * C::kStageBytes;
-                    const uint64_t bdesc = umma_desc_sw128(smem_u32(stage + G * kABytes));
+                    const uint64_t soff = (uint64_t)(uint32_t)(s * (C::kStageBytes >> 4));
+                    const uint64_t bdesc = bdesc0 + soff;
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
                         const int buf = G == 1 ? (it & 1) : g;
@@ -261,11 +278,13 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
                             tc_fence_after();
                         }
                         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
-                        const uint64_t adesc = umma_desc_sw128(smem_u32(stage + g * kABytes));
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)   // 4 x K=16 inside the 64-column chunk: +32 bytes per step
-                            umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kc | k) != 0 ? 1u : 0u);
-                        if (kc == p.n_k - 1) umma_commit(smem_u32(acc_full + buf));
+                        const uint64_t adesc = adesc0[g] + soff;
+                        // 4 x K=16 inside the 64-column chunk: +32 bytes (2 units) per step
+                        umma_bf16(d_tmem, adesc, bdesc, idesc, kc != 0 ? 1u : 0u);
+                        umma_bf16_acc(d_tmem, adesc + 2, bdesc + 2, idesc);
+                        umma_bf16_acc(d_tmem, adesc + 4, bdesc + 4, idesc);
+                        umma_bf16_acc(d_tmem, adesc + 6, bdesc + 6, idesc);
+                        if (kc == n_k - 1) umma_commit(smem_u32(acc_full + buf));
                     }
                     if (!ok) break;
                     umma_commit(smem_u32(empty + s));
