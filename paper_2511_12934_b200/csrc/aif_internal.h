@@ -188,6 +188,7 @@ struct TcScratch {
     void *X;               // dense interaction columns, [rows x x_cols] bf16
     void *H[kMaxHidden];   // activations after hidden layer k (k < last), [rows x hidden[k]] bf16
     void *xb;              // cross-feature buckets, [rows x F] uint16
+    size_t rows;           // rows every array has room for
 };
 size_t tc_scratch_row_bytes(const aif_ctx *ctx);
 void tc_scratch_layout(const aif_ctx *ctx, void *base, size_t rows, TcScratch *out);

@@ -69,10 +69,11 @@ struct LayerCfg {
     static constexpr int kEpiWarps = 4 * G;
     static constexpr int kMmaWarp = kEpiWarps;
     static constexpr int kProdWarp0 = kEpiWarps + 1;
-    static constexpr int kProdThreads = 128 * G;
+    static constexpr int kProdThreads = 128 * G;    // 128 producer threads per tile of the group, 8 rows each
     static constexpr int kBWarp = kProdWarp0 + 4 * G;
     static constexpr int kThreads = (kBWarp + 1) * 32;
-    static constexpr size_t kSmem = 1024 + (size_t)kStages * kStageBytes + (3 * kStages + 4) * 8 + 32 + 2 * G * 256 * 4 + kEpiWarps * 2048;
+    static constexpr int kSlabs = G == 1 ? 2 : 1;    // output staging slabs (2 KB) per epilogue warp
+    static constexpr size_t kSmem = 1024 + (size_t)kStages * kStageBytes + (3 * kStages + 4) * 8 + 32 + 2 * G * 256 * 4 + kEpiWarps * kSlabs * 2048 + 2 * G * 128 * 4;
 };
 
 struct TileInfo {
@@ -120,20 +121,24 @@ __global__ void __launch_bounds__(256) k_cross_buckets(const int32_t *__restrict
 
 // ---- the layer kernel -----------------------------------------------------------------------------------------
 template <int G>
-__global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __grid_constant__ CUtensorMap tmapB, const LayerParams p)
+__global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __grid_constant__ CUtensorMap tmapB, const __grid_constant__ CUtensorMap tmapOut,
+                                                                       const LayerParams p)
 {
     using C = LayerCfg<G>;
     constexpr int kStages = C::kStages;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
     // stage s: G A chunks (one per tile of the group), then the B chunk
-    uint64_t *bars = reinterpret_cast<uint64_t *>(base + kStages * C::kStageBytes);
+    // then the output staging slabs (2 KB each) of the epilogue warps, then barriers and small arrays
+    unsigned char *out_stage = base + kStages * C::kStageBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(out_stage + C::kEpiWarps * C::kSlabs * 2048);
     uint64_t *full_a = bars, *full_b = bars + kStages, *empty = bars + 2 * kStages;
     uint64_t *acc_full = bars + 3 * kStages, *acc_empty = acc_full + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
     volatile uint32_t *abort_flag = tmem_slot + 1;
     float *bias_s = reinterpret_cast<float *>(((uintptr_t)(tmem_slot + 4) + 15) & ~(uintptr_t)15);   // [G][256]
     float *wout_s = bias_s + G * 256;                            // [G][256]
+    int *ids_s = reinterpret_cast<int *>(wout_s + G * 256);      // [2][G][128] validated ids of the current / next item
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_groups = (p.sl.n_tiles + G - 1) / G;
@@ -163,7 +168,9 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
         const int g = warp >> 2;                     // tile of the group this warp quartet serves
         const int row = (warp & 3) * 32 + lane;      // TMEM lane = candidate row of the tile
         float *bs = bias_s + g * 256, *ws = wout_s + g * 256;
-        unsigned char *stg = reinterpret_cast<unsigned char *>(wout_s + G * 256) + warp * 2048;   // 32 rows x 64 bytes
+        // staging slabs of 32 rows x 64 bytes, 64-byte swizzle (the layout tmapOut expects)
+        unsigned char *stg = out_stage + warp * (C::kSlabs * 2048);
+        uint32_t slab = 0;
         int it = 0;
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
             const int grp = item / p.n_nchunks, nc = item - grp * p.n_nchunks, n0 = nc * p.n_cols;
@@ -201,22 +208,36 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
                             packed[2 * q] = *reinterpret_cast<const uint32_t *>(&h0);
                             packed[2 * q + 1] = *reinterpret_cast<const uint32_t *>(&h1);
                         }
-                        // through the warp's staging rows so that four lanes store one row's 64 bytes side by side
+                        // through a staging slab: the rows of a full slab leave with one asynchronous tile store, a
+                        // ragged slab (last tile of a request or mini-batch) with guarded 16-byte stores
+                        unsigned char *sb = stg + slab * 2048;
+                        if (lane == 0) bulk_wait_read<C::kSlabs - 1>();   // the store that last read this slab is done with it
+                        __syncwarp();
                         const int swz = (lane >> 1) & 3;
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
-                            *reinterpret_cast<uint4 *>(stg + lane * 64 + ((q ^ swz) << 4)) =
+                            *reinterpret_cast<uint4 *>(sb + lane * 64 + ((q ^ swz) << 4)) =
                                 make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-                        __syncwarp();
+                        const int wrow0 = (warp & 3) * 32;
+                        if (wrow0 + 32 <= t.cnt) {
+                            fence_proxy_async();
+                            __syncwarp();
+                            if (lane == 0) {
+                                tma_store_2d(&tmapOut, smem_u32(sb), n0 + c0, (int)(t.pos0 + wrow0));
+                                bulk_commit();
+                            }
+                        } else {
+                            __syncwarp();
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int rr = 8 * j + (lane >> 2), q = lane & 3;
-                            const uint4 v = *reinterpret_cast<const uint4 *>(stg + rr * 64 + ((q ^ ((rr >> 1) & 3)) << 4));
-                            const int trow = (warp & 3) * 32 + rr;
-                            if (trow < t.cnt)
-                                *reinterpret_cast<uint4 *>(p.out + (size_t)(t.pos0 + trow) * p.out_stride + n0 + c0 + q * 8) = v;
+                            for (int j = 0; j < 4; ++j) {
+                                const int rr = 8 * j + (lane >> 2), q = lane & 3;
+                                const uint4 v = *reinterpret_cast<const uint4 *>(sb + rr * 64 + ((q ^ ((rr >> 1) & 3)) << 4));
+                                if (wrow0 + rr < t.cnt)
+                                    *reinterpret_cast<uint4 *>(p.out + (size_t)(t.pos0 + wrow0 + rr) * p.out_stride + n0 + c0 + q * 8) = v;
+                            }
+                            __syncwarp();
                         }
-                        __syncwarp();
+                        slab = (slab + 1u) % (uint32_t)C::kSlabs;
                     } else {
                         const float4 *w4 = reinterpret_cast<const float4 *>(ws + c0);
 #pragma unroll
@@ -242,6 +263,7 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
             }
             named_bar_sync(1 + g, 128);
         }
+        if (lane == 0) bulk_wait<0>();   // all tile stores of this warp have reached global memory
     } else if (warp == C::kMmaWarp) {
         // ===================== MMA issuer =====================
         if (lane == 0) {
@@ -296,84 +318,110 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
     } else if (warp < C::kBWarp) {
         // ===================== A producer (128 threads per tile of the group) =====================
         const int pt = tid - C::kProdWarp0 * 32;
-        const int g = pt >> 7;
-        const int sub = pt & 7;              // 16-byte slot inside the 128-byte row chunk
-        const int r0 = (pt & 127) >> 3;      // rows r0, r0+16, ...
-        const uint32_t sw = (uint32_t)((sub ^ (r0 & 7)) << 4);
-        const uint32_t a_off = (uint32_t)(g * kABytes + r0 * 128) + sw;
+        const int gt = pt >> 7, lp = pt & 127;   // tile of the group this thread serves; its index among that tile's threads
+        const int sub = lp & 7;                  // 16-byte slot inside the 128-byte row chunk
+        const int r0 = lp >> 3;                  // rows r0, r0+16, ...
+        const uint32_t a_off = (uint32_t)(gt * kABytes + r0 * 128) + (uint32_t)((sub ^ (r0 & 7)) << 4);
+        const bool deep = p.n_k >= 2;            // bucket look-ups run two chunks ahead (needs the next item at most)
 
+        // The tile of the current / next item: registers hold where it lies, shared memory its validated ids
+        // (ids_s[buffer][tile][row], -1 for rows beyond the tile and for ids outside the table).
         struct Rows {
-            int ids[8];
             int cnt;
-            int64_t pos0;
+            uint32_t pos0;
             const uint8_t *Tt;
         };
-        auto load_rows = [&](int item, Rows &R) {
-            const int grp = item / p.n_nchunks;
-            const TileInfo t = decode_tile(p, grp * G + g);
-            R.cnt = t.cnt, R.pos0 = t.pos0;
-            R.Tt = t.cnt > 0 ? reinterpret_cast<const uint8_t *>(p.sl.slots[t.rq.slot].T) : nullptr;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int row = r0 + 16 * i;
-                int id = -1;
-                if (row < t.cnt) {
-                    id = p.sl.ids[t.pos0 + row];
-                    if (id < 0 || (int64_t)id >= p.M) {
-                        id = -1;
-                        if (p.check_ids && sub == 0) atomicOr(p.sl.status, AIF_STATUS_BAD_ID);
-                    }
+        auto load_rows = [&](int item, Rows &R, int &pend) {
+            const TileInfo t = decode_tile(p, (item / p.n_nchunks) * G + gt);
+            R.cnt = t.cnt, R.pos0 = (uint32_t)t.pos0;
+            R.Tt = t.cnt > 0 ? reinterpret_cast<const uint8_t *>(p.sl.slots[t.rq.slot].T) : p.E;
+            int id = -1;
+            if (lp < t.cnt) {   // this thread fetches the id of row lp; the others read it from shared memory
+                id = p.sl.ids[t.pos0 + lp];
+                if (id < 0 || (int64_t)id >= p.M) {
+                    id = -1;
+                    if (p.check_ids) atomicOr(p.sl.status, AIF_STATUS_BAD_ID);
                 }
-                R.ids[i] = id;
             }
+            pend = id;
         };
-        // global source of this thread's 16 bytes of each of its 8 rows in chunk kc; rows outside `mask` are zero-filled
-        auto sources = [&](int kc, const Rows &R, const uint8_t *(&gp)[8], uint32_t &mask) {
+        auto publish = [&](int buf, int pend) {
+            named_bar_sync(9, C::kProdThreads);   // every producer thread is done reading what this buffer held
+            ids_s[(buf * G + gt) * 128 + lp] = pend;
+            named_bar_sync(9, C::kProdThreads);
+        };
+        // bucket of this thread's rows in the field its slot of chunk kc belongs to (cross chunks only)
+        auto fetch = [&](int kc, const Rows &R, const int *ids, uint32_t (&raw)[8]) {
+            const ChunkSrc src = p.src[kc];
+            if (src.kind != SRC_CROSS) return;
+            const int f = (src.off + sub * 8) / p.dc;
+            const uint16_t *xb = p.xb + (size_t)(R.pos0 + r0) * p.F + f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) raw[i] = ids[r0 + 16 * i] >= 0 ? (uint32_t)__ldg(xb + (size_t)(16 * i) * p.F) : 0u;
+        };
+        // global sources of chunk kc: a base pointer and, per row, an offset in 16-byte units; rows whose bit in `mask`
+        // is clear are zero-filled
+        auto resolve = [&](int kc, const Rows &R, const int *ids, const uint32_t (&raw)[8], bool have_raw, const uint8_t *&bp,
+                           uint32_t (&off)[8], uint32_t &mask) {
             const ChunkSrc src = p.src[kc];
             mask = 0;
             if (src.kind == SRC_DENSE) {
+                const uint32_t row16 = (uint32_t)(p.x_row_bytes >> 4), c16 = (uint32_t)(src.off >> 4) + sub;
+                bp = p.X;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int row = r0 + 16 * i;
-                    gp[i] = p.X + (size_t)(R.pos0 + row) * p.x_row_bytes + src.off + sub * 16;
+                    off[i] = (R.pos0 + row) * row16 + c16;
                     if (row < R.cnt) mask |= 1u << i;
                 }
             } else if (src.kind == SRC_ITEM) {
+                const uint32_t row16 = (uint32_t)(p.e_row_bytes >> 4), c16 = (uint32_t)(src.off >> 4) + sub;
+                bp = p.E;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    gp[i] = p.E + (size_t)(R.ids[i] >= 0 ? R.ids[i] : 0) * p.e_row_bytes + src.off + sub * 16;
-                    if (R.ids[i] >= 0) mask |= 1u << i;
+                    const int id = ids[r0 + 16 * i];
+                    off[i] = (uint32_t)(id >= 0 ? id : 0) * row16 + c16;
+                    if (id >= 0) mask |= 1u << i;
                 }
             } else {
                 const int col = src.off + sub * 8;
                 const int f = col / p.dc, kin = col - f * p.dc;
+                const uint32_t row16 = (uint32_t)(p.dc >> 3), c16 = (uint32_t)(kin >> 3), fB = (uint32_t)(f * p.B);
+                bp = R.Tt;
                 const uint16_t *xb = p.xb + (size_t)(R.pos0 + r0) * p.F + f;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    int bk = 0;
-                    if (R.ids[i] >= 0) {
-                        bk = __ldg(xb + (size_t)(16 * i) * p.F);
+                    uint32_t bk = 0;
+                    if (ids[r0 + 16 * i] >= 0) {
+                        bk = have_raw ? raw[i] : (uint32_t)__ldg(xb + (size_t)(16 * i) * p.F);
                         mask |= 1u << i;
                     }
-                    gp[i] = R.Tt + (((size_t)f * p.B + bk) * p.dc + kin) * 2;
+                    off[i] = (fB + bk) * row16 + c16;
                 }
             }
         };
 
-        int s = 0;
+        int s = 0, buf = 0;
         uint32_t ph = 0;
         bool ok = true;
-        Rows cur;
-        const uint8_t *gp[8];
-        uint32_t mask = 0;
+        Rows cur, nxt;
+        int pend = -1;
+        const uint8_t *bp = p.E;
+        uint32_t off[8], raw[8], mask = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) off[i] = 0, raw[i] = 0;
         if ((int)blockIdx.x < n_items) {
-            load_rows(blockIdx.x, cur);
-            sources(0, cur, gp, mask);
+            load_rows(blockIdx.x, cur, pend);
+            publish(0, pend);
+            resolve(0, cur, ids_s + gt * 128, raw, false, bp, off, mask);
+            if (deep) fetch(1, cur, ids_s + gt * 128, raw);
         }
-        for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+        nxt = cur;
+        for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, buf ^= 1) {
             const int next_item = item + gridDim.x;
-            Rows nxt = cur;
-            if (next_item < n_items) load_rows(next_item, nxt);   // global loads land while this item's chunks are copied
+            const bool has_next = next_item < n_items;
+            const int *ids_cur = ids_s + (buf * G + gt) * 128, *ids_nxt = ids_s + ((buf ^ 1) * G + gt) * 128;
+            if (has_next) load_rows(next_item, nxt, pend);   // the id load lands while chunk 0 is copied
             for (int kc = 0; kc < p.n_k; ++kc) {
                 if (!mbar_wait(smem_u32(empty + s), ph ^ 1u, abort_flag)) {
                     ok = false;
@@ -381,14 +429,22 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
                 }
                 const uint32_t dst0 = smem_u32(base + s * C::kStageBytes) + a_off;
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    cp_async16(dst0 + (uint32_t)(i * 16 * 128), (mask >> i) & 1u ? gp[i] : p.E, (mask >> i) & 1u ? 16u : 0u);
+                for (int i = 0; i < 8; ++i) {
+                    const bool on = (mask >> i) & 1u;
+                    cp_async16(dst0 + (uint32_t)(i * 16 * 128), on ? bp + ((size_t)off[i] << 4) : p.E, on ? 16u : 0u);
+                }
                 // the stage's barrier receives this thread's arrival when its copies have landed: no thread waits for them
                 cp_async_arrive_noinc(smem_u32(full_a + s));
                 if (++s == kStages) s = 0, ph ^= 1u;
-                // sources of the next chunk: the bucket look-ups are in flight while this thread waits for the next stage
-                if (kc + 1 < p.n_k) sources(kc + 1, cur, gp, mask);
-                else if (next_item < n_items) sources(0, nxt, gp, mask);
+                if (kc == 0 && has_next) publish(buf ^ 1, pend);
+                // sources of the next chunk from the buckets fetched one iteration ago; then start the fetch for the
+                // chunk after it, so that its latency is covered by a whole iteration
+                if (kc + 1 < p.n_k) resolve(kc + 1, cur, ids_cur, raw, deep, bp, off, mask);
+                else if (has_next) resolve(0, nxt, ids_nxt, raw, deep, bp, off, mask);
+                if (deep) {
+                    if (kc + 2 < p.n_k) fetch(kc + 2, cur, ids_cur, raw);
+                    else if (has_next) fetch(kc + 2 - p.n_k, nxt, ids_nxt, raw);
+                }
             }
             cur = nxt;
         }
@@ -516,6 +572,7 @@ struct TcPlan {
     int n_k[kMaxHidden] = {}, n_cols[kMaxHidden] = {}, n_nchunks[kMaxHidden] = {};
     ChunkSrc src0[kMaxChunks] = {};
     CUtensorMap tmap[kMaxHidden];
+    size_t cap_rows = 0;                 // rows of the context's own scratch arrays
     __nv_bfloat16 *W[kMaxHidden] = {};
     __nv_bfloat16 *H[kMaxHidden] = {};   // activations after layer k (k < last)
     __nv_bfloat16 *X = nullptr;
@@ -538,6 +595,8 @@ int dense_cols(const aif_config &c)
 bool tc_supported(const aif_config &c)
 {
     if (c.dtype != AIF_BF16 || c.d % 64 != 0) return false;
+    if ((uint64_t)c.M * (uint64_t)c.d * 2 / 16 >= (1ull << 32)) return false;        // row offsets are 32-bit, in 16-byte units
+    if ((uint64_t)(c.max_batch_candidates + kTcTile) * 4096 / 16 >= (1ull << 32)) return false;   // same for dense rows
     if (c.blocks & AIF_BLK_CROSS) {
         if ((c.F * c.dc) % 64 != 0 || c.dc % 8 != 0 || c.B > 65536) return false;
         if (64 % c.dc != 0 && c.dc % 64 != 0) return false;
@@ -588,6 +647,7 @@ cudaError_t tc_prepare_context(aif_ctx *ctx)
     if (c.blocks & AIF_BLK_SIMTIER) add(SRC_DENSE, xoff * 2);
     pl->k1pad = n * 64;
     const size_t cap = (size_t)c.max_batch_candidates + kTcTile;
+    pl->cap_rows = cap;
     auto alloc = [&](void **p, size_t bytes) -> cudaError_t {
         bytes = (bytes + 255) / 256 * 256;
         cudaError_t e = cudaMalloc(p, bytes);
@@ -679,6 +739,7 @@ void tc_scratch_layout(const aif_ctx *ctx, void *base, size_t rows, TcScratch *o
         }
     }
     out->xb = (c.blocks & AIF_BLK_CROSS) ? p : nullptr;
+    out->rows = rows;
 }
 
 cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t, cudaStream_t st)
@@ -687,6 +748,7 @@ cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t, 
     TcScratch sc;
     sc.X = pl->X;
     sc.xb = pl->xb;
+    sc.rows = pl->cap_rows;
     for (int k = 0; k < kMaxHidden; ++k) sc.H[k] = pl->H[k];
     return launch_score_tc_scratch(ctx, sl, st, sc);
 }
@@ -739,6 +801,18 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
             for (int i = 0; i < p.n_k; ++i) p.src[i].kind = SRC_DENSE, p.src[i].off = i * 128;
         }
         const bool last = k + 1 == c.n_hidden;
+        // store target of the epilogue: the activation array as a [rows x hidden[k]] tensor, 32 x 32 boxes, 64-byte swizzle
+        CUtensorMap tmap_out = pl->tmap[k];
+        if (!last) {
+            const cuuint64_t dims[2] = {(cuuint64_t)c.hidden[k], (cuuint64_t)sc.rows};
+            const cuuint64_t strides[1] = {(cuuint64_t)c.hidden[k] * 2};
+            const cuuint32_t box[2] = {32, 32};
+            const cuuint32_t estr[2] = {1, 1};
+            CUresult r = encode_fn()(&tmap_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, sc.H[k], dims, strides, box, estr,
+                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+        }
         p.epi = last ? EPI_DOT : EPI_STORE;
         p.bias_from_slot = k == 0, p.bias = ctx->b[k], p.emit_sigmoid = c.emit_sigmoid;
         p.out = (__nv_bfloat16 *)sc.H[k], p.out_stride = c.hidden[k];
@@ -747,8 +821,8 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
         const bool pair = ((sl.n_tiles + 1) / 2) * p.n_nchunks >= 2 * 148;
         const int items = pair ? ((sl.n_tiles + 1) / 2) * p.n_nchunks : sl.n_tiles * p.n_nchunks;
         const int grid = items < 148 ? items : 148;
-        if (pair) k_layer_tc<2><<<grid, LayerCfg<2>::kThreads, LayerCfg<2>::kSmem, st>>>(pl->tmap[k], p);
-        else k_layer_tc<1><<<grid, LayerCfg<1>::kThreads, LayerCfg<1>::kSmem, st>>>(pl->tmap[k], p);
+        if (pair) k_layer_tc<2><<<grid, LayerCfg<2>::kThreads, LayerCfg<2>::kSmem, st>>>(pl->tmap[k], tmap_out, p);
+        else k_layer_tc<1><<<grid, LayerCfg<1>::kThreads, LayerCfg<1>::kSmem, st>>>(pl->tmap[k], tmap_out, p);
         count_launch();
         timing_mark(ctx, names[k], st);
         cudaError_t e = cudaGetLastError();
