@@ -127,18 +127,27 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
             }
             tc_fence_after();
             const uint32_t ts = lane_base + (uint32_t)(b * BN);
-            // pass 1: block maximum of the row
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(ts + (uint32_t)c0, r);
-                tmem_ld_wait();
+            // the row's BN scores: all loads first, one wait
+            uint32_t sc[BN];
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (c0 + i < valid_cols) mx = fmaxf(mx, __uint_as_float(r[i]));
+            for (int c0 = 0; c0 < BN; c0 += 32) tmem_ld32(ts + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[32]>(&sc[c0]));
+            tmem_ld_wait();
+            // block maximum of the row (four independent chains)
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            if (valid_cols == BN) {
+#pragma unroll
+                for (int i = 0; i < BN; i += 4) {
+                    mx4[0] = fmaxf(mx4[0], __uint_as_float(sc[i]));
+                    mx4[1] = fmaxf(mx4[1], __uint_as_float(sc[i + 1]));
+                    mx4[2] = fmaxf(mx4[2], __uint_as_float(sc[i + 2]));
+                    mx4[3] = fmaxf(mx4[3], __uint_as_float(sc[i + 3]));
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < BN; ++i)
+                    if (i < valid_cols) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sc[i]));
             }
-            const float mt = mx * k2;
+            const float mt = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * k2;
             if (j == 0) {
                 m_used = mt;
             } else {
@@ -171,20 +180,21 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                 ok = false;
                 break;
             }
-            // pass 2: probabilities -> bf16 A operand in shared memory
+            // probabilities -> bf16 A operand in shared memory
             unsigned char *Pb = smP + b * C::kPBytes;
-#pragma unroll 1
+            float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
             for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(ts + (uint32_t)c0, r);
-                tmem_ld_wait();
                 uint32_t packed[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const float p0 = (c0 + 2 * i < valid_cols) ? fast_exp2(fmaf(__uint_as_float(r[2 * i]), k2, -m_used)) : 0.f;
-                    const float p1 =
-                        (c0 + 2 * i + 1 < valid_cols) ? fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), k2, -m_used)) : 0.f;
-                    l_sum += p0 + p1;
+                    float p0 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i]), k2, -m_used));
+                    float p1 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i + 1]), k2, -m_used));
+                    if (valid_cols != BN) {
+                        if (c0 + 2 * i >= valid_cols) p0 = 0.f;
+                        if (c0 + 2 * i + 1 >= valid_cols) p1 = 0.f;
+                    }
+                    ls4[i & 3] += p0 + p1;
                     const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                     packed[i] = *reinterpret_cast<const uint32_t *>(&h);
                 }
@@ -195,6 +205,7 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                     *reinterpret_cast<uint4 *>(chunk + (((slot0 + q) ^ (row & 7)) << 4)) =
                         make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
             }
+            l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(smem_u32(p_full + b));
