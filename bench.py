@@ -60,6 +60,8 @@ def kernel_flops(name: str, wl: synth.Workload, n: int) -> float:
         return f["total"] * n
     if name == "interact":
         return (f["attention"] + f["lsh_din"] + f["bea"]) * n
+    if name == "buckets":
+        return 0.0
     return f.get(name, 0.0) * n
 
 
@@ -302,7 +304,24 @@ def run_ours(args, wl):
     kavg = {k: v / kcount for k, v in ksum.items()}
     assert srv.ctx.poll_status() == 0, "device status word set during the benchmark"
 
+    # the gather stage alone (aif_gather_rows) on a long id stream drawn like the workload's candidates: HBM roofline
+    gn = 1 << 22
+    g_ids = torch.from_numpy(sampler._raw(np.random.default_rng(7), gn).astype(np.int32)).cuda()
+    g_out = torch.empty(gn, wl.d, dtype=torch.float32 if wl.dtype == "f32" else torch.bfloat16, device="cuda")
+    row_bytes = wl.d * (4 if wl.dtype == "f32" else 2)
+
+    def gather_step(i):
+        srv.ctx.gather_rows(g_ids, g_out)
+
+    gather_step(0)
+    g_ms = float(np.median(timed(10, gather_step)))
+    del g_out
+
     peaks, peak_kind = load_peaks()
+    gather = {"rows": gn, "row_bytes": row_bytes, "ms": g_ms, "achieved": gn * (2 * row_bytes + 4) / (g_ms * 1e-3) / 1e9,
+              "peak": float(peaks["hbm_gbs"]), "unit": "GB/s", "bound": "hbm", "peak_kind": f"copy bandwidth, {peak_kind}",
+              "ids": "drawn like the workload's candidates, repeats allowed"}
+    gather["frac"] = gather["achieved"] / gather["peak"]
     top = max(kavg, key=kavg.get)
     tensor = bool(srv.ctx.get_stats().tensor_path) and top != "interact"
     kf = kernel_flops(top, wl, cands)
@@ -336,6 +355,7 @@ def run_ours(args, wl):
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": roof,
+        "gather_stage": gather,
         "replica_plan": plan,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
