@@ -97,22 +97,23 @@ __device__ __forceinline__ TileInfo decode_tile(const LayerParams &p, int tile)
 }
 
 // Cross-feature index generation for a whole launch (Section 3.3, "real-time generation" from the candidate's
-// attribute): xb[pos][f] = bucket of candidate pos in field f.  Done once per call so that the layer kernel's gather
-// threads only look the bucket up.
-__global__ void __launch_bounds__(256) k_cross_buckets(const int32_t *__restrict__ ids, int64_t total, int F, int B, int b_mask,
-                                                        int mode, uint16_t *__restrict__ xb)
+// attribute): xb[pos][f] = bucket of candidate pos in field f, or kNoBucket for an id outside the item table.  Done
+// once per call so that the layer kernel's gather threads only look the bucket up.
+constexpr uint32_t kNoBucket = 0xFFFFu;
+__global__ void __launch_bounds__(256) k_cross_buckets(const int32_t *__restrict__ ids, int64_t total, int64_t M, int F, int B,
+                                                        int b_mask, int mode, uint16_t *__restrict__ xb)
 {
     const int64_t n = total * F;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t pos = i / F;
         const int f = (int)(i - pos * F);
         const int id = ids[pos];
-        int bk = 0;
-        if (id >= 0) {
-            if (mode == AIF_BUCKET_MOD) bk = id % B;
+        uint32_t bk = kNoBucket;
+        if (id >= 0 && (int64_t)id < M) {
+            if (mode == AIF_BUCKET_MOD) bk = (uint32_t)(id % B);
             else {
                 const uint64_t h = mix64((uint64_t)id, (uint64_t)f);
-                bk = b_mask >= 0 ? (int)(h & (uint64_t)b_mask) : (int)(h % (uint64_t)B);
+                bk = b_mask >= 0 ? (uint32_t)(h & (uint64_t)b_mask) : (uint32_t)(h % (uint64_t)B);
             }
         }
         xb[i] = (uint16_t)bk;
@@ -327,14 +328,18 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
         // The tile of the current / next item: registers hold where it lies, shared memory its validated ids
         // (ids_s[buffer][tile][row], -1 for rows beyond the tile and for ids outside the table).
         struct Rows {
-            int cnt;
+            uint32_t rowmask;        // bit i: row r0 + 16 i lies inside the tile
             uint32_t pos0;
             const uint8_t *Tt;
+            const uint16_t *xb;      // bucket row of this thread's first row
         };
+        const uint32_t xb_step = (uint32_t)(16 * p.F);   // elements between the bucket rows of rows r0 + 16 i and r0 + 16 (i + 1)
         auto load_rows = [&](int item, Rows &R, int &pend) {
             const TileInfo t = decode_tile(p, (item / p.n_nchunks) * G + gt);
-            R.cnt = t.cnt, R.pos0 = (uint32_t)t.pos0;
+            const int nrows = t.cnt > r0 ? (t.cnt - r0 + 15) >> 4 : 0;
+            R.rowmask = (1u << nrows) - 1u, R.pos0 = (uint32_t)t.pos0;
             R.Tt = t.cnt > 0 ? reinterpret_cast<const uint8_t *>(p.sl.slots[t.rq.slot].T) : p.E;
+            R.xb = p.xb + (size_t)(t.pos0 + r0) * p.F;
             int id = -1;
             if (lp < t.cnt) {   // this thread fetches the id of row lp; the others read it from shared memory
                 id = p.sl.ids[t.pos0 + lp];
@@ -350,33 +355,31 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
             ids_s[(buf * G + gt) * 128 + lp] = pend;
             named_bar_sync(9, C::kProdThreads);
         };
-        // bucket of this thread's rows in the field its slot of chunk kc belongs to (cross chunks only)
-        auto fetch = [&](int kc, const Rows &R, const int *ids, uint32_t (&raw)[8]) {
+        // bucket of this thread's rows in the field its slot of chunk kc belongs to (cross chunks only); rows outside
+        // the tile read other candidates' entries or stale scratch, which rowmask discards
+        auto fetch = [&](int kc, const Rows &R, uint32_t (&raw)[8]) {
             const ChunkSrc src = p.src[kc];
             if (src.kind != SRC_CROSS) return;
-            const int f = (src.off + sub * 8) / p.dc;
-            const uint16_t *xb = p.xb + (size_t)(R.pos0 + r0) * p.F + f;
+            const uint16_t *xb = R.xb + (src.off + sub * 8) / p.dc;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) raw[i] = ids[r0 + 16 * i] >= 0 ? (uint32_t)__ldg(xb + (size_t)(16 * i) * p.F) : 0u;
+            for (int i = 0; i < 8; ++i) raw[i] = (uint32_t)__ldg(xb + i * xb_step);
         };
         // global sources of chunk kc: a base pointer and, per row, an offset in 16-byte units; rows whose bit in `mask`
         // is clear are zero-filled
-        auto resolve = [&](int kc, const Rows &R, const int *ids, const uint32_t (&raw)[8], bool have_raw, const uint8_t *&bp,
+        auto resolve = [&](int kc, const Rows &R, const int *ids, uint32_t (&raw)[8], bool have_raw, const uint8_t *&bp,
                            uint32_t (&off)[8], uint32_t &mask) {
             const ChunkSrc src = p.src[kc];
-            mask = 0;
             if (src.kind == SRC_DENSE) {
-                const uint32_t row16 = (uint32_t)(p.x_row_bytes >> 4), c16 = (uint32_t)(src.off >> 4) + sub;
+                const uint32_t row16 = (uint32_t)(p.x_row_bytes >> 4);
+                const uint32_t first = (R.pos0 + r0) * row16 + (uint32_t)(src.off >> 4) + sub;
                 bp = p.X;
+                mask = R.rowmask;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int row = r0 + 16 * i;
-                    off[i] = (R.pos0 + row) * row16 + c16;
-                    if (row < R.cnt) mask |= 1u << i;
-                }
+                for (int i = 0; i < 8; ++i) off[i] = first + (uint32_t)(16 * i) * row16;
             } else if (src.kind == SRC_ITEM) {
                 const uint32_t row16 = (uint32_t)(p.e_row_bytes >> 4), c16 = (uint32_t)(src.off >> 4) + sub;
                 bp = p.E;
+                mask = 0;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int id = ids[r0 + 16 * i];
@@ -386,18 +389,20 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
             } else {
                 const int col = src.off + sub * 8;
                 const int f = col / p.dc, kin = col - f * p.dc;
-                const uint32_t row16 = (uint32_t)(p.dc >> 3), c16 = (uint32_t)(kin >> 3), fB = (uint32_t)(f * p.B);
+                const uint32_t row16 = (uint32_t)(p.dc >> 3), base16 = (uint32_t)(f * p.B) * row16 + (uint32_t)(kin >> 3);
                 bp = R.Tt;
-                const uint16_t *xb = p.xb + (size_t)(R.pos0 + r0) * p.F + f;
+                if (!have_raw) {
+                    const uint16_t *xb = R.xb + f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) raw[i] = (uint32_t)__ldg(xb + i * xb_step);
+                }
+                mask = 0;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    uint32_t bk = 0;
-                    if (ids[r0 + 16 * i] >= 0) {
-                        bk = have_raw ? raw[i] : (uint32_t)__ldg(xb + (size_t)(16 * i) * p.F);
-                        mask |= 1u << i;
-                    }
-                    off[i] = (fB + bk) * row16 + c16;
+                    if (raw[i] != kNoBucket) mask |= 1u << i;
+                    off[i] = raw[i] * row16 + base16;
                 }
+                mask &= R.rowmask;
             }
         };
 
@@ -414,7 +419,7 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
             load_rows(blockIdx.x, cur, pend);
             publish(0, pend);
             resolve(0, cur, ids_s + gt * 128, raw, false, bp, off, mask);
-            if (deep) fetch(1, cur, ids_s + gt * 128, raw);
+            if (deep) fetch(1, cur, raw);
         }
         nxt = cur;
         for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, buf ^= 1) {
@@ -442,8 +447,8 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
                 if (kc + 1 < p.n_k) resolve(kc + 1, cur, ids_cur, raw, deep, bp, off, mask);
                 else if (has_next) resolve(0, nxt, ids_nxt, raw, deep, bp, off, mask);
                 if (deep) {
-                    if (kc + 2 < p.n_k) fetch(kc + 2, cur, ids_cur, raw);
-                    else if (has_next) fetch(kc + 2 - p.n_k, nxt, ids_nxt, raw);
+                    if (kc + 2 < p.n_k) fetch(kc + 2, cur, raw);
+                    else if (has_next) fetch(kc + 2 - p.n_k, nxt, raw);
                 }
             }
             cur = nxt;
@@ -598,7 +603,7 @@ bool tc_supported(const aif_config &c)
     if ((uint64_t)c.M * (uint64_t)c.d * 2 / 16 >= (1ull << 32)) return false;        // row offsets are 32-bit, in 16-byte units
     if ((uint64_t)(c.max_batch_candidates + kTcTile) * 4096 / 16 >= (1ull << 32)) return false;   // same for dense rows
     if (c.blocks & AIF_BLK_CROSS) {
-        if ((c.F * c.dc) % 64 != 0 || c.dc % 8 != 0 || c.B > 65536) return false;
+        if ((c.F * c.dc) % 64 != 0 || c.dc % 8 != 0 || c.B >= 65535) return false;
         if (64 % c.dc != 0 && c.dc % 64 != 0) return false;
     }
     for (int k = 0; k < c.n_hidden; ++k) {
@@ -763,8 +768,8 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
     if (c.blocks & AIF_BLK_CROSS) {
         const int64_t n = sl.total * c.F;
         const int grid = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
-        k_cross_buckets<<<grid, 256, 0, st>>>(sl.ids, sl.total, c.F, c.B, (c.B & (c.B - 1)) == 0 ? c.B - 1 : -1, c.bucket_mode,
-                                              (uint16_t *)sc.xb);
+        k_cross_buckets<<<grid, 256, 0, st>>>(sl.ids, sl.total, c.M, c.F, c.B, (c.B & (c.B - 1)) == 0 ? c.B - 1 : -1,
+                                              c.bucket_mode, (uint16_t *)sc.xb);
         count_launch();
         timing_mark(ctx, "buckets", st);
         cudaError_t e = cudaGetLastError();
