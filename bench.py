@@ -35,7 +35,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # CUDA-core kernels: SMs x lanes x 2 x max clock
 
 # DRAM traffic per launch of the dominant kernel from the committed ncu summary (profiles/), bytes; None = not captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {("c2_paper_shaped", "layer1"): 7367680}      # profiles/scoring_step_c2.md
 
 
 # ----------------------------------------------------------------------------------------------------------------
@@ -138,12 +138,16 @@ def oracle_sample_size(wl, core_seconds=12.0):
 def cpu_baseline(wl, pre=None):
     oracle, table, req, ids, threads = pre or oracle_setup(wl)
     n = oracle_sample_size(wl)
-    t0 = time.perf_counter()
-    oracle.score(table, req, ids[:n])
-    dt = time.perf_counter() - t0
-    return {"value": n / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": f"first {n} candidates of request 0 of {wl.name}, scored once ({dt:.2f} s)",
-            "ms_per_1e4_candidates": 1e4 * dt / n * 1e3}
+    # repeat the sample until about 12 core-seconds of oracle work have been timed
+    passes, dt = 0, 0.0
+    while passes == 0 or (dt * threads < 12.0 and passes < 64):
+        t0 = time.perf_counter()
+        oracle.score(table, req, ids[:n])
+        dt += time.perf_counter() - t0
+        passes += 1
+    return {"value": n * passes / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"first {n} candidates of request 0 of {wl.name}, scored {passes} times ({dt:.2f} s wall)",
+            "ms_per_1e4_candidates": 1e4 * dt / (n * passes) * 1e3}
 
 
 def run_reference(args, wl):
@@ -198,9 +202,7 @@ def reduce_max(value: float, dist=None) -> float:
 
 def run_ours(args, wl):
     import torch
-    from paper_2511_12934_b200 import binding as B
     from paper_2511_12934_b200 import build as libbuild
-    from paper_2511_12934_b200 import serving
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -212,9 +214,31 @@ def run_ours(args, wl):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     else:
         torch.cuda.set_device(0)
-    plan = replica_plan(world, rank)
     libbuild.build()
+    line = measure(args, wl, args.steps, args.warmup, dist, world, rank, full=True)
+    if world == 1 and args.also:
+        # the other bf16 shapes of the benchmark definition, briefly, so that one run shows every roofline fraction
+        others = {}
+        for name in args.also.split(","):
+            o = measure(args, synth.SHORT[name], 20, 3, None, 1, 0, full=False)
+            others[name] = {k: o[k] for k in ("value", "unit", "ms_per_step", "p50_ms_per_request", "p99_ms_per_request",
+                                              "flops_per_candidate", "config", "roofline", "step_tflops")}
+        line["other_workloads"] = others
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl)
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
 
+
+def measure(args, wl, steps, warmup, dist, world, rank, full):
+    """Times `steps` scoring steps of one workload on this rank's GPU; returns the JSON line as a dict."""
+    import torch
+    from paper_2511_12934_b200 import binding as B
+    from paper_2511_12934_b200 import serving
+
+    plan = replica_plan(world, rank)
     path = {"auto": B.PATH_AUTO, "simt": B.PATH_SIMT, "tensor": B.PATH_TENSOR}[args.path]
     weights = synth.make_weights(wl)
     table = synth.make_item_table(wl)
@@ -257,7 +281,7 @@ def run_ours(args, wl):
         torch.cuda.synchronize()
         return [a.elapsed_time(b) for a, b in ev]
 
-    for i in range(max(3, args.warmup)):
+    for i in range(max(3, warmup)):
         flush.zero_()
         step(i)
     torch.cuda.synchronize()
@@ -267,7 +291,7 @@ def run_ours(args, wl):
         dist.barrier()
     torch.cuda.synchronize()
     launches0 = B.kernel_launches()
-    times = timed(args.steps, step)
+    times = timed(steps, step)
     launches = B.kernel_launches() - launches0
     if dist is not None:
         dist.barrier()
@@ -285,7 +309,7 @@ def run_ours(args, wl):
         else:
             srv.ctx.score_host(states[i % pool], host_ids[i % pool], host_out[i % pool])
 
-    e2e_steps = max(3, min(args.steps, 50))
+    e2e_steps = max(3, min(steps, 50)) if full else 3
     step_e2e(0)
     e2e_times = timed(e2e_steps, step_e2e)
     e2e_ms = reduce_max(sum(e2e_times), dist)
@@ -294,7 +318,7 @@ def run_ours(args, wl):
     # per-kernel durations (events inside the library), for the roofline of the dominant kernel
     srv.ctx.set_kernel_timing(True)
     ksum, kcount = {}, 0
-    for i in range(min(args.steps, 50)):
+    for i in range(min(steps, 50)):
         flush.zero_()
         step(i)
         for k, v in srv.ctx.get_kernel_timing().items():
@@ -336,11 +360,11 @@ def run_ours(args, wl):
     roof["traffic"] = NCU_TRAFFIC_BYTES.get((wl.name, top))
     roof["kernel_ms"] = kavg
 
-    value = world * cands * args.steps / (total_ms * 1e-3)
+    value = world * cands * steps / (total_ms * 1e-3)
     per_request_ms = [t / (wl.R if batch else 1) for t in times]
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
-        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": max(3, warmup),
+        "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": wl.name, "requests_per_step": wl.R, "candidates_per_step": cands, "M": wl.M, "d": wl.d,
                    "L": wl.L, "F": wl.F, "hidden": list(wl.hidden), "mini_batch": wl.mini_batch,
@@ -350,6 +374,7 @@ def run_ours(args, wl):
         "p50_ms_per_request": float(np.percentile(per_request_ms, 50)),
         "p99_ms_per_request": float(np.percentile(per_request_ms, 99)),
         "flops_per_candidate": flops_per_candidate(wl)["total"],
+        "step_tflops": flops_per_candidate(wl)["total"] * cands * steps / (total_ms * 1e-3) / 1e12,
         "e2e": {"value": world * cands * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * cands,
                 "d2h_bytes_per_step": 4 * cands, "steps": e2e_steps},
         "gpu_launches": int(launches),
@@ -358,13 +383,10 @@ def run_ours(args, wl):
         "gather_stage": gather,
         "replica_plan": plan,
     }
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(wl)
-    if rank == 0:
-        print(json.dumps(line))
     srv.close()
-    if dist is not None:
-        dist.destroy_process_group()
+    del srv, flush, logits, ids_dev, g_ids
+    torch.cuda.empty_cache()
+    return line
 
 
 def main():
@@ -376,6 +398,7 @@ def main():
     ap.add_argument("--workload", default="c2", choices=sorted(synth.SHORT))
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--also", default="c3,c4,c5", help="other workloads measured briefly after the main one ('' = none)")
     # scaled copies of a workload, for profiler captures that must stay small (the defaults are the full sizes)
     ap.add_argument("--requests", type=int, default=0, help="override the number of requests per step")
     ap.add_argument("--rows", type=int, default=0, help="override the rows of the item table")
