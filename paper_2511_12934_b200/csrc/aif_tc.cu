@@ -59,21 +59,31 @@ struct LayerParams {
     ChunkSrc src[kMaxChunks];
 };
 
-// Geometry of the layer kernel.  G = 128-candidate tiles per work item: with G = 2 one weight chunk in shared memory
-// feeds two tiles (two TMEM accumulators), which halves the weight traffic per candidate; with G = 1 the two
-// accumulators alternate between consecutive items so that the epilogue of one overlaps the main loop of the next.
-template <int G>
+// Geometry of the layer kernel.  A work item fills one or two 256-column TMEM accumulators:
+//   MODE 0  one tile, one 256-wide output slice; the two accumulators alternate between consecutive items so that the
+//           epilogue of one overlaps the main loop of the next (small launches, every item on its own SM)
+//   MODE 1  two tiles, one slice: one weight chunk in shared memory feeds both tiles, which halves the weight traffic
+//           per candidate (large launches)
+//   MODE 2  one tile, two slices: one gathered A chunk feeds both slices, so the tile's rows are gathered once instead
+//           of once per slice (launches that would otherwise need a second round of items)
+// A and B have rings of their own: gathered rows have the longer latency and the smaller chunks.
+template <int MODE>
 struct LayerCfg {
-    static constexpr int kStages = G == 1 ? 4 : 3;
-    static constexpr int kStageBytes = G * kABytes + kBBytes;
-    static constexpr int kEpiWarps = 4 * G;
+    static constexpr int G = MODE == 1 ? 2 : 1;          // tiles per work item
+    static constexpr int NB = MODE == 2 ? 2 : 1;         // output slices per work item
+    static constexpr int kAcc = G * NB;                  // accumulators a work item fills
+    static constexpr int kStagesA = MODE == 1 ? 3 : 4;
+    static constexpr int kStagesB = MODE == 0 ? 4 : (MODE == 1 ? 3 : 2);
+    static constexpr int kAStage = G * kABytes, kBStage = NB * kBBytes;
+    static constexpr int kEpiWarps = 4 * kAcc;
     static constexpr int kMmaWarp = kEpiWarps;
     static constexpr int kProdWarp0 = kEpiWarps + 1;
     static constexpr int kProdThreads = 128 * G;    // 128 producer threads per tile of the group, 8 rows each
     static constexpr int kBWarp = kProdWarp0 + 4 * G;
     static constexpr int kThreads = (kBWarp + 1) * 32;
-    static constexpr int kSlabs = G == 1 ? 2 : 1;    // output staging slabs (2 KB) per epilogue warp
-    static constexpr size_t kSmem = 1024 + (size_t)kStages * kStageBytes + (3 * kStages + 4) * 8 + 32 + 2 * G * 256 * 4 + kEpiWarps * kSlabs * 2048 + 2 * G * 128 * 4;
+    static constexpr int kSlabs = MODE == 0 ? 2 : 1;    // output staging slabs (2 KB) per epilogue warp
+    static constexpr size_t kSmem = 1024 + (size_t)kStagesA * kAStage + (size_t)kStagesB * kBStage + (2 * kStagesA + 2 * kStagesB + 4) * 8 +
+                                    32 + 2 * kAcc * 256 * 4 + kEpiWarps * kSlabs * 2048 + 2 * G * 128 * 4;
 };
 
 struct TileInfo {
@@ -121,35 +131,40 @@ __global__ void __launch_bounds__(256) k_cross_buckets(const int32_t *__restrict
 }
 
 // ---- the layer kernel -----------------------------------------------------------------------------------------
-template <int G>
-__global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __grid_constant__ CUtensorMap tmapB, const __grid_constant__ CUtensorMap tmapOut,
-                                                                       const LayerParams p)
+template <int MODE>
+__global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const __grid_constant__ CUtensorMap tmapB,
+                                                                          const __grid_constant__ CUtensorMap tmapOut, const LayerParams p)
 {
-    using C = LayerCfg<G>;
-    constexpr int kStages = C::kStages;
+    using C = LayerCfg<MODE>;
+    constexpr int G = C::G, NB = C::NB, kAcc = C::kAcc, kSA = C::kStagesA, kSB = C::kStagesB;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-    // stage s: G A chunks (one per tile of the group), then the B chunk
-    // then the output staging slabs (2 KB each) of the epilogue warps, then barriers and small arrays
-    unsigned char *out_stage = base + kStages * C::kStageBytes;
+    // A ring (per stage: one chunk per tile of the group), B ring (per stage: one chunk per output slice), the output
+    // staging slabs (2 KB each) of the epilogue warps, then barriers and small arrays
+    unsigned char *smA = base, *smB = base + kSA * C::kAStage;
+    unsigned char *out_stage = smB + kSB * C::kBStage;
     uint64_t *bars = reinterpret_cast<uint64_t *>(out_stage + C::kEpiWarps * C::kSlabs * 2048);
-    uint64_t *full_a = bars, *full_b = bars + kStages, *empty = bars + 2 * kStages;
-    uint64_t *acc_full = bars + 3 * kStages, *acc_empty = acc_full + 2;
+    uint64_t *full_a = bars, *empty_a = full_a + kSA, *full_b = empty_a + kSA, *empty_b = full_b + kSB;
+    uint64_t *acc_full = empty_b + kSB, *acc_empty = acc_full + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
     volatile uint32_t *abort_flag = tmem_slot + 1;
-    float *bias_s = reinterpret_cast<float *>(((uintptr_t)(tmem_slot + 4) + 15) & ~(uintptr_t)15);   // [G][256]
-    float *wout_s = bias_s + G * 256;                            // [G][256]
-    int *ids_s = reinterpret_cast<int *>(wout_s + G * 256);      // [2][G][128] validated ids of the current / next item
+    float *bias_s = reinterpret_cast<float *>(((uintptr_t)(tmem_slot + 4) + 15) & ~(uintptr_t)15);   // [kAcc][256]
+    float *wout_s = bias_s + kAcc * 256;                         // [kAcc][256]
+    int *ids_s = reinterpret_cast<int *>(wout_s + kAcc * 256);   // [2][G][128] validated ids of the current / next item
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_groups = (p.sl.n_tiles + G - 1) / G;
-    const int n_items = n_groups * p.n_nchunks;
+    const int n_ncg = p.n_nchunks / NB;             // groups of output slices
+    const int n_items = n_groups * n_ncg;
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kSA; ++s) {
             mbar_init(smem_u32(full_a + s), C::kProdThreads);
+            mbar_init(smem_u32(empty_a + s), 1);
+        }
+        for (int s = 0; s < kSB; ++s) {
             mbar_init(smem_u32(full_b + s), 1);
-            mbar_init(smem_u32(empty + s), 1);
+            mbar_init(smem_u32(empty_b + s), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(acc_full + b), 1);
@@ -166,17 +181,18 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
 
     if (warp < C::kEpiWarps) {
         // ===================== epilogue =====================
-        const int g = warp >> 2;                     // tile of the group this warp quartet serves
+        const int a = warp >> 2;                     // accumulator this warp quartet serves
+        const int g = G == 2 ? a : 0;                // its tile of the group
         const int row = (warp & 3) * 32 + lane;      // TMEM lane = candidate row of the tile
-        float *bs = bias_s + g * 256, *ws = wout_s + g * 256;
+        float *bs = bias_s + a * 256, *ws = wout_s + a * 256;
         // staging slabs of 32 rows x 64 bytes, 64-byte swizzle (the layout tmapOut expects)
         unsigned char *stg = out_stage + warp * (C::kSlabs * 2048);
         uint32_t slab = 0;
         int it = 0;
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
-            const int grp = item / p.n_nchunks, nc = item - grp * p.n_nchunks, n0 = nc * p.n_cols;
-            const int buf = G == 1 ? (it & 1) : g;
-            const uint32_t ph = G == 1 ? (uint32_t)((it >> 1) & 1) : (uint32_t)(it & 1);
+            const int grp = item / n_ncg, nc = (item - grp * n_ncg) * NB + (NB == 2 ? a : 0), n0 = nc * p.n_cols;
+            const int buf = kAcc == 1 ? (it & 1) : a;
+            const uint32_t ph = kAcc == 1 ? (uint32_t)((it >> 1) & 1) : (uint32_t)(it & 1);
             const TileInfo t = decode_tile(p, grp * G + g);
             if (t.cnt > 0) {
                 const float *bias = p.bias_from_slot ? p.sl.slots[t.rq.slot].p_u : p.bias;
@@ -185,7 +201,7 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
                     if (p.epi == EPI_DOT) ws[j] = __bfloat162float(p.w_out[n0 + j]);
                 }
             }
-            named_bar_sync(1 + g, 128);
+            named_bar_sync(1 + a, 128);
             if (!mbar_wait(smem_u32(acc_full + buf), ph, abort_flag)) break;
             tc_fence_after();
             const bool valid = row < t.cnt;
@@ -262,7 +278,7 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
                 if (id < 0 || (int64_t)id >= p.M) logit = __int_as_float(0x7fc00000);
                 p.sl.logits[t.pos0 + row] = logit;
             }
-            named_bar_sync(1 + g, 128);
+            named_bar_sync(1 + a, 128);
         }
         if (lane == 0) bulk_wait<0>();   // all tile stores of this warp have reached global memory
     } else if (warp == C::kMmaWarp) {
@@ -270,30 +286,29 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(kTcTile, p.n_cols);
             const int n_k = p.n_k;
-            // descriptors of stage 0; stage s lies s * kStageBytes further (the address field counts 16-byte units)
-            const uint64_t bdesc0 = umma_desc_sw128(smem_u32(base + G * kABytes));
+            // descriptors of stage 0 of each ring; stage s lies s stage sizes further (the address field counts 16 bytes)
+            const uint64_t bdesc0 = umma_desc_sw128(smem_u32(smB));
             uint64_t adesc0[G];
 #pragma unroll
-            for (int g = 0; g < G; ++g) adesc0[g] = umma_desc_sw128(smem_u32(base + g * kABytes));
-            int it = 0, s = 0;
-            uint32_t ph = 0;
+            for (int g = 0; g < G; ++g) adesc0[g] = umma_desc_sw128(smem_u32(smA + g * kABytes));
+            int it = 0, sa = 0, sb = 0;
+            uint32_t pha = 0, phb = 0;
             bool ok = true;
             for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
                 for (int kc = 0; kc < n_k; ++kc) {
-                    if (!mbar_wait(smem_u32(full_a + s), ph, abort_flag) || !mbar_wait(smem_u32(full_b + s), ph, abort_flag)) {
+                    if (!mbar_wait(smem_u32(full_a + sa), pha, abort_flag) || !mbar_wait(smem_u32(full_b + sb), phb, abort_flag)) {
                         ok = false;
                         break;
                     }
                     // the A chunk was written by cp.async (generic proxy) and is read by the MMA (async proxy)
                     fence_proxy_async();
                     tc_fence_after();
-                    const uint64_t soff = (uint64_t)(uint32_t)(s * (C::kStageBytes >> 4));
-                    const uint64_t bdesc = bdesc0 + soff;
+                    const uint64_t aoff = (uint64_t)(uint32_t)(sa * (C::kAStage >> 4)), boff = (uint64_t)(uint32_t)(sb * (C::kBStage >> 4));
 #pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        const int buf = G == 1 ? (it & 1) : g;
+                    for (int a = 0; a < kAcc; ++a) {
+                        const int buf = kAcc == 1 ? (it & 1) : a;
                         if (kc == 0) {   // the accumulator must have been drained by the epilogue of its previous use
-                            const uint32_t eph = (G == 1 ? (uint32_t)((it >> 1) & 1) : (uint32_t)(it & 1)) ^ 1u;
+                            const uint32_t eph = (kAcc == 1 ? (uint32_t)((it >> 1) & 1) : (uint32_t)(it & 1)) ^ 1u;
                             if (!mbar_wait(smem_u32(acc_empty + buf), eph, abort_flag)) {
                                 ok = false;
                                 break;
@@ -301,7 +316,8 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
                             tc_fence_after();
                         }
                         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
-                        const uint64_t adesc = adesc0[g] + soff;
+                        const uint64_t adesc = adesc0[G == 2 ? a : 0] + aoff;
+                        const uint64_t bdesc = bdesc0 + boff + (uint64_t)(NB == 2 ? a * (kBBytes >> 4) : 0);
                         // 4 x K=16 inside the 64-column chunk: +32 bytes (2 units) per step
                         umma_bf16(d_tmem, adesc, bdesc, idesc, kc != 0 ? 1u : 0u);
                         umma_bf16_acc(d_tmem, adesc + 2, bdesc + 2, idesc);
@@ -310,8 +326,10 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
                         if (kc == n_k - 1) umma_commit(smem_u32(acc_full + buf));
                     }
                     if (!ok) break;
-                    umma_commit(smem_u32(empty + s));
-                    if (++s == kStages) s = 0, ph ^= 1u;
+                    umma_commit(smem_u32(empty_a + sa));
+                    umma_commit(smem_u32(empty_b + sb));
+                    if (++sa == kSA) sa = 0, pha ^= 1u;
+                    if (++sb == kSB) sb = 0, phb ^= 1u;
                 }
             }
         }
@@ -335,7 +353,7 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
         };
         const uint32_t xb_step = (uint32_t)(16 * p.F);   // elements between the bucket rows of rows r0 + 16 i and r0 + 16 (i + 1)
         auto load_rows = [&](int item, Rows &R, int &pend) {
-            const TileInfo t = decode_tile(p, (item / p.n_nchunks) * G + gt);
+            const TileInfo t = decode_tile(p, (item / n_ncg) * G + gt);
             const int nrows = t.cnt > r0 ? (t.cnt - r0 + 15) >> 4 : 0;
             R.rowmask = (1u << nrows) - 1u, R.pos0 = (uint32_t)t.pos0;
             R.Tt = t.cnt > 0 ? reinterpret_cast<const uint8_t *>(p.sl.slots[t.rq.slot].T) : p.E;
@@ -428,11 +446,11 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
             const int *ids_cur = ids_s + (buf * G + gt) * 128, *ids_nxt = ids_s + ((buf ^ 1) * G + gt) * 128;
             if (has_next) load_rows(next_item, nxt, pend);   // the id load lands while chunk 0 is copied
             for (int kc = 0; kc < p.n_k; ++kc) {
-                if (!mbar_wait(smem_u32(empty + s), ph ^ 1u, abort_flag)) {
+                if (!mbar_wait(smem_u32(empty_a + s), ph ^ 1u, abort_flag)) {
                     ok = false;
                     break;
                 }
-                const uint32_t dst0 = smem_u32(base + s * C::kStageBytes) + a_off;
+                const uint32_t dst0 = smem_u32(smA + s * C::kAStage) + a_off;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const bool on = (mask >> i) & 1u;
@@ -440,7 +458,7 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
                 }
                 // the stage's barrier receives this thread's arrival when its copies have landed: no thread waits for them
                 cp_async_arrive_noinc(smem_u32(full_a + s));
-                if (++s == kStages) s = 0, ph ^= 1u;
+                if (++s == kSA) s = 0, ph ^= 1u;
                 if (kc == 0 && has_next) publish(buf ^ 1, pend);
                 // sources of the next chunk from the buckets fetched one iteration ago; then start the fetch for the
                 // chunk after it, so that its latency is covered by a whole iteration
@@ -462,16 +480,18 @@ __global__ void __launch_bounds__(LayerCfg<G>::kThreads, 1) k_layer_tc(const __g
             bool ok = true;
             const uint32_t bytes = (uint32_t)p.n_cols * 128u;
             for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-                const int grp = item / p.n_nchunks, nc = item - grp * p.n_nchunks;
+                const int grp = item / n_ncg, nc0 = (item - grp * n_ncg) * NB;
                 for (int kc = 0; kc < p.n_k; ++kc) {
-                    if (!mbar_wait(smem_u32(empty + s), ph ^ 1u, abort_flag)) {
+                    if (!mbar_wait(smem_u32(empty_b + s), ph ^ 1u, abort_flag)) {
                         ok = false;
                         break;
                     }
-                    mbar_expect_tx(smem_u32(full_b + s), bytes);
-                    tma_load_2d(smem_u32(base + s * C::kStageBytes + G * kABytes), &tmapB, smem_u32(full_b + s), kc * 64,
-                                nc * p.n_cols);
-                    if (++s == kStages) s = 0, ph ^= 1u;
+                    mbar_expect_tx(smem_u32(full_b + s), NB * bytes);
+#pragma unroll
+                    for (int nb = 0; nb < NB; ++nb)
+                        tma_load_2d(smem_u32(smB + s * C::kBStage + nb * kBBytes), &tmapB, smem_u32(full_b + s), kc * 64,
+                                    (nc0 + nb) * p.n_cols);
+                    if (++s == kSB) s = 0, ph ^= 1u;
                 }
             }
         }
@@ -674,6 +694,8 @@ cudaError_t tc_prepare_context(aif_ctx *ctx)
     }
     if (pl->x_cols && (e = alloc((void **)&pl->X, cap * pl->x_cols * 2)) != cudaSuccess) return e;
     if ((c.blocks & AIF_BLK_CROSS) && (e = alloc((void **)&pl->xb, cap * c.F * 2)) != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_layer_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LayerCfg<0>::kSmem);
+    if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_layer_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LayerCfg<1>::kSmem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_layer_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LayerCfg<2>::kSmem);
@@ -822,12 +844,16 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
         p.bias_from_slot = k == 0, p.bias = ctx->b[k], p.emit_sigmoid = c.emit_sigmoid;
         p.out = (__nv_bfloat16 *)sc.H[k], p.out_stride = c.hidden[k];
         p.w_out = (const __nv_bfloat16 *)ctx->w_out, p.b_out = ctx->b_out;
-        // two tiles per item once that still leaves every SM at least two items
+        // two tiles per item once that still leaves every SM at least two items; else, if single items would need a
+        // second round on some SMs, one tile with two output slices per item
+        const int single = sl.n_tiles * p.n_nchunks;
         const bool pair = ((sl.n_tiles + 1) / 2) * p.n_nchunks >= 2 * 148;
-        const int items = pair ? ((sl.n_tiles + 1) / 2) * p.n_nchunks : sl.n_tiles * p.n_nchunks;
+        const bool wide = !pair && p.n_nchunks % 2 == 0 && single > 148;
+        const int items = pair ? ((sl.n_tiles + 1) / 2) * p.n_nchunks : wide ? single / 2 : single;
         const int grid = items < 148 ? items : 148;
-        if (pair) k_layer_tc<2><<<grid, LayerCfg<2>::kThreads, LayerCfg<2>::kSmem, st>>>(pl->tmap[k], tmap_out, p);
-        else k_layer_tc<1><<<grid, LayerCfg<1>::kThreads, LayerCfg<1>::kSmem, st>>>(pl->tmap[k], tmap_out, p);
+        if (pair) k_layer_tc<1><<<grid, LayerCfg<1>::kThreads, LayerCfg<1>::kSmem, st>>>(pl->tmap[k], tmap_out, p);
+        else if (wide) k_layer_tc<2><<<grid, LayerCfg<2>::kThreads, LayerCfg<2>::kSmem, st>>>(pl->tmap[k], tmap_out, p);
+        else k_layer_tc<0><<<grid, LayerCfg<0>::kThreads, LayerCfg<0>::kSmem, st>>>(pl->tmap[k], tmap_out, p);
         count_launch();
         timing_mark(ctx, names[k], st);
         cudaError_t e = cudaGetLastError();
