@@ -113,6 +113,8 @@ constexpr uint32_t kNoBucket = 0xFFFFu;
 __global__ void __launch_bounds__(256) k_cross_buckets(const int32_t *__restrict__ ids, int64_t total, int64_t M, int F, int B,
                                                         int b_mask, int mode, uint16_t *__restrict__ xb)
 {
+    grid_dep_launch();
+    grid_dep_wait();
     const int64_t n = total * F;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t pos = i / F;
@@ -178,6 +180,8 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    grid_dep_launch();
+    grid_dep_wait();   // everything above overlapped the tail of the previous kernel; from here on its results are read
 
     if (warp < C::kEpiWarps) {
         // ===================== epilogue =====================
@@ -520,6 +524,8 @@ __global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl,
     uint32_t *sigq = reinterpret_cast<uint32_t *>(qv + 8 * md.d);            // [8][8]
     int *tiers = reinterpret_cast<int *>(sigq + 64);                         // [8][16]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, d = md.d, dq = d >> 5;
+    grid_dep_launch();
+    grid_dep_wait();
     const ReqDev rq = find_request(sl, blockIdx.x);
     int start, cnt;
     tile_range(blockIdx.x - rq.tile_begin, rq.n, kTcTile, md.mini_batch, start, cnt);
@@ -790,11 +796,10 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
     if (c.blocks & AIF_BLK_CROSS) {
         const int64_t n = sl.total * c.F;
         const int grid = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
-        k_cross_buckets<<<grid, 256, 0, st>>>(sl.ids, sl.total, c.M, c.F, c.B, (c.B & (c.B - 1)) == 0 ? c.B - 1 : -1,
-                                              c.bucket_mode, (uint16_t *)sc.xb);
+        cudaError_t e = launch_pdl(k_cross_buckets, dim3(grid), dim3(256), 0, st, sl.ids, sl.total, c.M, c.F, c.B,
+                                   (c.B & (c.B - 1)) == 0 ? c.B - 1 : -1, c.bucket_mode, (uint16_t *)sc.xb);
         count_launch();
         timing_mark(ctx, "buckets", st);
-        cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     const bool att_tc = ctx->tc_att_plan != nullptr;
@@ -806,10 +811,10 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
     const int other_dense = c.blocks & (AIF_BLK_BEA | AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER);
     if (pl->x_cols && (!att_tc || other_dense)) {
         const size_t smem = (size_t)8 * c.d * 4 + 64 * 4 + 128 * 4;
-        k_interact_x<<<sl.n_tiles, 256, smem, st>>>(md, sl, (__nv_bfloat16 *)sc.X, pl->x_cols, att_tc ? 1 : 0);
+        cudaError_t e = launch_pdl(k_interact_x, dim3(sl.n_tiles), dim3(256), smem, st, md, sl, (__nv_bfloat16 *)sc.X, pl->x_cols,
+                                   att_tc ? 1 : 0);
         count_launch();
         timing_mark(ctx, "interact", st);
-        cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     static const char *names[kMaxHidden] = {"layer1", "layer2", "layer3", "layer4"};
@@ -851,12 +856,12 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
         const bool wide = !pair && p.n_nchunks % 2 == 0 && single > 148;
         const int items = pair ? ((sl.n_tiles + 1) / 2) * p.n_nchunks : wide ? single / 2 : single;
         const int grid = items < 148 ? items : 148;
-        if (pair) k_layer_tc<1><<<grid, LayerCfg<1>::kThreads, LayerCfg<1>::kSmem, st>>>(pl->tmap[k], tmap_out, p);
-        else if (wide) k_layer_tc<2><<<grid, LayerCfg<2>::kThreads, LayerCfg<2>::kSmem, st>>>(pl->tmap[k], tmap_out, p);
-        else k_layer_tc<0><<<grid, LayerCfg<0>::kThreads, LayerCfg<0>::kSmem, st>>>(pl->tmap[k], tmap_out, p);
+        cudaError_t e;
+        if (pair) e = launch_pdl(k_layer_tc<1>, dim3(grid), dim3(LayerCfg<1>::kThreads), LayerCfg<1>::kSmem, st, pl->tmap[k], tmap_out, p);
+        else if (wide) e = launch_pdl(k_layer_tc<2>, dim3(grid), dim3(LayerCfg<2>::kThreads), LayerCfg<2>::kSmem, st, pl->tmap[k], tmap_out, p);
+        else e = launch_pdl(k_layer_tc<0>, dim3(grid), dim3(LayerCfg<0>::kThreads), LayerCfg<0>::kSmem, st, pl->tmap[k], tmap_out, p);
         count_launch();
         timing_mark(ctx, names[k], st);
-        cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;

@@ -62,12 +62,6 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const ReqDev rq = find_request(p.sl, blockIdx.x);
-    int start, cnt;
-    tile_range(blockIdx.x - rq.tile_begin, rq.n, kTcTile, p.mini_batch, start, cnt);
-    const int64_t pos0 = rq.off + start;
-    const int L = p.sl.slots[rq.slot].L;
-    const int nb = (L + BN - 1) / BN;
 
     if (tid == 0) {
         for (int s = 0; s < kKvStages; ++s) {
@@ -89,6 +83,14 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    grid_dep_launch();
+    grid_dep_wait();   // the set-up above overlapped the previous kernel; the request table and slots are read from here on
+    const ReqDev rq = find_request(p.sl, blockIdx.x);
+    int start, cnt;
+    tile_range(blockIdx.x - rq.tile_begin, rq.n, kTcTile, p.mini_batch, start, cnt);
+    const int64_t pos0 = rq.off + start;
+    const int L = p.sl.slots[rq.slot].L;
+    const int nb = (L + BN - 1) / BN;
 
     if (warp < 4) {
         // ===================== queries, softmax, output =====================
@@ -371,12 +373,13 @@ cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
     p.sl = sl, p.E = (const uint8_t *)ctx->E, p.M = c.M, p.mini_batch = c.mini_batch;
     p.x_stride = x_stride, p.X = (__nv_bfloat16 *)X;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.d);
+    cudaError_t e;
     if (c.d == 128)
-        k_att_tc<128, 128><<<sl.n_tiles, kAttThreads, AttCfg<128, 128>::kSmem, st>>>(pl->tmap, p);
+        e = launch_pdl(k_att_tc<128, 128>, dim3(sl.n_tiles), dim3(kAttThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, p);
     else
-        k_att_tc<256, 64><<<sl.n_tiles, kAttThreads, AttCfg<256, 64>::kSmem, st>>>(pl->tmap, p);
+        e = launch_pdl(k_att_tc<256, 64>, dim3(sl.n_tiles), dim3(kAttThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, p);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace aif
