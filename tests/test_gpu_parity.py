@@ -246,3 +246,34 @@ def test_sharp_softmax_exercises_the_running_max_rescaling():
     _check_logits(got, want, 1e-2 * scale)
     assert srv.ctx.poll_status() == 0
     srv.close()
+
+
+@pytest.mark.parametrize("name", ["c3", "c4", "c5", "c5b"])
+def test_full_size_batches_on_sampled_candidates(name):
+    """The multi-request shapes at their full sizes, scored in one aif_score_batch call exactly as the benchmark
+    launches them; the oracle checks a seeded sample of candidates of a few requests (first, middle, last)."""
+    wl = synth.SHORT[name]
+    weights, table, srv, oracle = _setup(wl, zero_bias=False)
+    sampler = synth.IdSampler(wl)
+    states, id_lists, reqs = [], [], {}
+    check = sorted({0, wl.R // 2, wl.R - 1})
+    for r in range(wl.R):
+        rq = synth.make_request(wl, r)
+        states.append(srv.precompute(r, srv.upload_request(rq, B.USER_PROJECTED)))
+        id_lists.append(sampler.request_ids(r))
+        if r in check:
+            reqs[r] = helpers.projected_request(wl, rq)
+    outs = srv.score_many(states, id_lists)
+    assert srv.ctx.get_stats().tensor_path == 1
+    g = np.random.default_rng(11)
+    worst = 0.0
+    for r in check:
+        ids = id_lists[r]
+        # the sample always contains the request's first and last candidate (tile edges)
+        pick = np.unique(np.concatenate([[0, len(ids) - 1], g.choice(len(ids), 48, replace=False)]))
+        want = oracle.score(table, reqs[r], ids[pick])
+        worst = max(worst, _check_logits(outs[r][pick], want, TOL["bf16"]))
+    for o in outs:
+        assert np.isfinite(o).all()
+    assert srv.ctx.poll_status() == 0
+    srv.close()
