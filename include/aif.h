@@ -259,6 +259,14 @@ int aif_get_stats(aif_ctx *ctx, aif_stats *out);
 int aif_set_kernel_timing(aif_ctx *ctx, int on);
 int aif_get_kernel_timing(aif_ctx *ctx, int32_t *n, const char **names, float *ms);
 
+/* Self-test of the failure path of the device-side waits (Section 3.4's consistency requirement is enforced on the
+ * host; this is its device-side companion).  Every wait inside the tensor-core kernels is bounded: when a producer
+ * never delivers, the waiting thread gives up after a fixed number of clock cycles, the kernel sets AIF_STATUS_TIMEOUT
+ * and returns normally.  This call launches one tiny kernel on `stream` whose single wait can never be satisfied and
+ * whose bound is limit_cycles (1 .. 2e9 SM clock cycles); afterwards aif_poll_status reports AIF_STATUS_TIMEOUT and the
+ * context remains fully usable.  Nothing faults, traps or hangs. */
+int aif_selftest_bounded_wait(aif_ctx *ctx, int64_t limit_cycles, aif_stream stream);
+
 /* Number of kernels this library has launched in this process (all contexts). */
 uint64_t aif_kernel_launches(void);
 

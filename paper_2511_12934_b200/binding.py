@@ -75,7 +75,7 @@ EXPORTS = [
     "aif_input_width", "aif_mix64", "aif_create", "aif_destroy", "aif_load_weights", "aif_item_nearline_refresh",
     "aif_user_precompute", "aif_user_release", "aif_user_request_key", "aif_user_state_export", "aif_score",
     "aif_score_batch", "aif_score_host", "aif_score_noalloc", "aif_gather_rows", "aif_poll_status", "aif_get_stats",
-    "aif_set_kernel_timing", "aif_get_kernel_timing", "aif_kernel_launches", "aif_strerror", "aif_last_error",
+    "aif_set_kernel_timing", "aif_get_kernel_timing", "aif_kernel_launches", "aif_selftest_bounded_wait", "aif_strerror", "aif_last_error",
 ]
 
 _lib = None
@@ -111,6 +111,7 @@ def load_library(path: Optional[str] = None):
     lib.aif_set_kernel_timing.argtypes = [vp, C.c_int]
     lib.aif_get_kernel_timing.argtypes = [vp, C.POINTER(i32), C.POINTER(C.c_char_p), C.POINTER(C.c_float)]
     lib.aif_kernel_launches.argtypes, lib.aif_kernel_launches.restype = [], u64
+    lib.aif_selftest_bounded_wait.argtypes = [vp, i64, vp]
     lib.aif_strerror.argtypes, lib.aif_strerror.restype = [C.c_int], C.c_char_p
     lib.aif_last_error.argtypes, lib.aif_last_error.restype = [], C.c_char_p
     if path is None:
@@ -302,6 +303,10 @@ class Aif:
         bits = C.c_uint32()
         _check(self.lib.aif_poll_status(self.h, C.byref(bits)), "aif_poll_status")
         return int(bits.value)
+
+    def selftest_bounded_wait(self, limit_cycles: int, stream=None):
+        """Launches the kernel whose only wait runs out after limit_cycles; poll_status then shows STATUS_TIMEOUT."""
+        _check(self.lib.aif_selftest_bounded_wait(self.h, int(limit_cycles), _stream(stream)), "aif_selftest_bounded_wait")
 
     def set_kernel_timing(self, on: bool):
         _check(self.lib.aif_set_kernel_timing(self.h, 1 if on else 0), "aif_set_kernel_timing")

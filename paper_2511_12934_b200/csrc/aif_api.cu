@@ -575,6 +575,14 @@ int aif_get_kernel_timing(aif_ctx *ctx, int32_t *n, const char **names, float *m
 
 uint64_t aif_kernel_launches(void) { return g_launches.load(); }
 
+int aif_selftest_bounded_wait(aif_ctx *ctx, int64_t limit_cycles, aif_stream stream)
+{
+    if (!ctx || limit_cycles < 1 || limit_cycles > 2000000000ll) return AIF_ERR_ARG;
+    DeviceGuard g(ctx->device);
+    AIF_CUDA(launch_wait_selftest(ctx, (long long)limit_cycles, as_stream(stream)));
+    return AIF_OK;
+}
+
 const char *aif_strerror(int code)
 {
     switch (code) {

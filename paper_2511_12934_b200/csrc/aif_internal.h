@@ -197,5 +197,6 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
 int check_user_state(aif_ctx *ctx, const aif_user_state *st);
 void set_last_error(const char *text);
 int tc_tiles_for(const aif_ctx *ctx, int n);
+cudaError_t launch_wait_selftest(const aif_ctx *ctx, long long limit_cycles, cudaStream_t st);
 
 }  // namespace aif

@@ -586,6 +586,22 @@ __global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl,
     }
 }
 
+// Self-test of the bounded wait: one thread waits, with a short limit, on an mbarrier that nobody arrives on.  The wait
+// gives up, raises the status bit and the kernel returns normally: this is the path a scoring kernel takes when a
+// producer never delivers, exercised without any fault.
+__global__ void k_wait_selftest(uint32_t *status, long long limit_cycles)
+{
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const bool done = mbar_try_wait(smem_u32(&bar), 0u, 1000u) || mbar_wait_slow(smem_u32(&bar), 0u, &abort_flag, limit_cycles);
+        if (!done && abort_flag) atomicOr(status, AIF_STATUS_TIMEOUT);
+    }
+}
+
 // W1 [H1 x Din] -> [H1 x k1pad]: user columns dropped, zero padding at the end.
 __global__ void k_pack_w1(const __nv_bfloat16 *W1, __nv_bfloat16 *out, int H1, int din, int d, int k1, int k1pad)
 {
@@ -747,6 +763,13 @@ cudaError_t tc_prepare_weights(aif_ctx *ctx, const aif_weights *w, cudaStream_t 
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
+}
+
+cudaError_t launch_wait_selftest(const aif_ctx *ctx, long long limit_cycles, cudaStream_t st)
+{
+    k_wait_selftest<<<1, 32, 0, st>>>(ctx->status, limit_cycles);
+    count_launch();
+    return cudaGetLastError();
 }
 
 size_t tc_scratch_row_bytes(const aif_ctx *ctx)

@@ -277,3 +277,25 @@ def test_full_size_batches_on_sampled_candidates(name):
         assert np.isfinite(o).all()
     assert srv.ctx.poll_status() == 0
     srv.close()
+
+
+def test_a_wait_that_runs_out_sets_the_timeout_bit_and_leaves_the_context_usable():
+    """Failure detection without a fault: the device-side waits are bounded.  A kernel whose wait nobody satisfies gives
+    up after its limit, reports AIF_STATUS_TIMEOUT through the status word and returns; scoring afterwards is intact."""
+    wl = helpers.MINI["c2"].with_(name="timeout", N=300)
+    weights, table, srv, oracle = _setup(wl)
+    rq = synth.make_request(wl, 0)
+    ids = synth.IdSampler(wl).request_ids(0)
+    st = srv.precompute(1, srv.upload_request(rq, B.USER_PROJECTED))
+    want = oracle.score(table, helpers.projected_request(wl, rq), ids)
+    _check_logits(srv.score_ids(st, ids), want, TOL["bf16"])
+    assert srv.ctx.poll_status() == 0
+    srv.ctx.selftest_bounded_wait(2_000_000)            # about a millisecond
+    assert srv.ctx.poll_status() == B.STATUS_TIMEOUT
+    assert srv.ctx.get_stats().timeout_events == 1
+    assert srv.ctx.poll_status() == 0                   # read and cleared
+    _check_logits(srv.score_ids(st, ids), want, TOL["bf16"])
+    with pytest.raises(B.AifError) as e:
+        srv.ctx.selftest_bounded_wait(0)
+    assert e.value.code == B.ERR_ARG
+    srv.close()
