@@ -1,14 +1,17 @@
-// Dense target attention on the tensor cores (sm_100a): att_i = softmax(e_i S^T / sqrt(d)) S for a tile of 128
+// Dense target attention on the tensor cores (sm_100a): att_i = softmax(e_i S^T / sqrt(d)) S for tiles of 128
 // candidates against the request's projected behaviour sequence S [L x d] (Section 4.2, first paragraph: similarity
 // of the target item with every historical item, then pooling; here in its dense softmax form).
 //
-// One CTA per 128-candidate tile, 192 threads:
-//   warps 0-3  gather the tile's item rows (the queries) into shared memory, then per key block: read the scores
-//              from TMEM, online softmax in fp32 (one thread per candidate row), write the probabilities as a bf16
-//              A operand into shared memory; finally normalise O and store the attention rows
-//   warp  4    allocates TMEM; one lane issues tcgen05.mma: scores = Q K^T (both K-major), O += P V with V read from
-//              the very same shared-memory tile as K, as an MN-major B operand
+// Persistent kernel: one CTA per SM walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  224 threads:
+//   warps 0-3  per key block: read the score row from TMEM into registers, online softmax in fp32 (one thread per
+//              candidate row), write the probabilities as a bf16 A operand into shared memory; at the end of a tile
+//              normalise O and store the attention rows
+//   warp  4    allocates TMEM; one lane issues tcgen05.mma over the flat sequence of key blocks of all its tiles:
+//              scores = Q K^T (both K-major) one block ahead of O += P V, with V read from the very same shared-memory
+//              tile as K, as an MN-major B operand
 //   warp  5    one lane streams key/value blocks of S with TMA (3-D tensor map over the user-state arena)
+//   warp  6    gathers the item rows of the next tile (the queries) with cp.async while the current tile is processed
+//              (two query buffers where shared memory allows, d = 128)
 // TMEM: two score buffers (so the softmax of block j overlaps Q K^T of block j+1) and the O accumulator.
 // The running maximum is only raised when a row's block maximum exceeds it by more than 8 (in the log2 domain);
 // then the warp rescales its 32 rows of O in TMEM.  Until then probabilities stay below 2^8, which fp32 sums and
@@ -20,8 +23,8 @@
 namespace aif {
 namespace {
 
-constexpr int kAttThreads = 192;
-constexpr int kKvStages = 3;
+constexpr int kAttThreads = 224;
+constexpr int kAttMmaWarp = 4, kAttTmaWarp = 5, kAttQWarp = 6;
 
 struct AttParams {
     ScoreLaunch sl;
@@ -37,34 +40,55 @@ template <int D, int BN>
 struct AttCfg {
     static constexpr int kQChunks = D / 64;             // 64-column (128-byte) chunks of a row
     static constexpr int kQBytes = kQChunks * 128 * 128;
+    static constexpr int kQBufs = D <= 128 ? 2 : 1;     // query buffers
+    static constexpr int kKvStages = 3;
     static constexpr int kKvChunkBytes = BN * 128;      // one 64-column chunk of a key block
     static constexpr int kKvBytes = kQChunks * kKvChunkBytes;
     static constexpr int kPChunks = BN / 64;
     static constexpr int kPBytes = kPChunks * 128 * 128;
     static constexpr int kTmemO = 2 * BN;               // column of the O accumulator
-    static constexpr size_t kSmem = 1024 + kQBytes + kKvStages * kKvBytes + 2 * kPBytes + 256;
+    static constexpr size_t kSmem = 1024 + kQBufs * kQBytes + kKvStages * kKvBytes + 2 * kPBytes + 512;
 };
+
+// One tile of the launch as every role needs it.
+struct AttTile {
+    int slot, cnt, nb;
+    int64_t pos0;
+};
+
+template <int BN>
+__device__ __forceinline__ AttTile att_tile(const AttParams &p, int tile)
+{
+    const ReqDev rq = find_request(p.sl, tile);
+    int start, cnt;
+    tile_range(tile - rq.tile_begin, rq.n, kTcTile, p.mini_batch, start, cnt);
+    AttTile t;
+    t.slot = rq.slot, t.cnt = cnt, t.pos0 = rq.off + start;
+    t.nb = (p.sl.slots[rq.slot].L + BN - 1) / BN;
+    return t;
+}
 
 template <int D, int BN>
 __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant__ CUtensorMap tmapS, const AttParams p)
 {
     using C = AttCfg<D, BN>;
+    constexpr int kS = C::kKvStages, kQB = C::kQBufs;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
     unsigned char *smQ = base;
-    unsigned char *smKV = smQ + C::kQBytes;
-    unsigned char *smP = smKV + kKvStages * C::kKvBytes;
+    unsigned char *smKV = smQ + kQB * C::kQBytes;
+    unsigned char *smP = smKV + kS * C::kKvBytes;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smP + 2 * C::kPBytes);
-    uint64_t *kv_full = bars, *kv_empty = bars + kKvStages;
-    uint64_t *s_full = bars + 2 * kKvStages, *p_full = s_full + 2, *pv_done = p_full + 2;
-    uint64_t *q_full = pv_done + 2, *o_final = q_full + 1;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(o_final + 1);
+    uint64_t *kv_full = bars, *kv_empty = bars + kS;
+    uint64_t *s_full = bars + 2 * kS, *p_full = s_full + 2, *pv_done = p_full + 2;
+    uint64_t *q_full = pv_done + 2, *q_empty = q_full + 2, *o_final = q_empty + 2, *o_free = o_final + 1, *q_first = o_free + 1;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_first + 1);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
-        for (int s = 0; s < kKvStages; ++s) {
+        for (int s = 0; s < kS; ++s) {
             mbar_init(smem_u32(kv_full + s), 1);
             mbar_init(smem_u32(kv_empty + s), 1);
         }
@@ -72,152 +96,158 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
             mbar_init(smem_u32(s_full + b), 1);
             mbar_init(smem_u32(p_full + b), 128);
             mbar_init(smem_u32(pv_done + b), 1);
+            mbar_init(smem_u32(q_full + b), 32);
+            mbar_init(smem_u32(q_empty + b), 1);
         }
-        mbar_init(smem_u32(q_full), 128);
         mbar_init(smem_u32(o_final), 1);
+        mbar_init(smem_u32(o_free), 128);
+        mbar_init(smem_u32(q_first), 128);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4) tmem_alloc(smem_u32(tmem_slot), 512);
+    if (warp == kAttMmaWarp) tmem_alloc(smem_u32(tmem_slot), 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     grid_dep_launch();
     grid_dep_wait();   // the set-up above overlapped the previous kernel; the request table and slots are read from here on
-    const ReqDev rq = find_request(p.sl, blockIdx.x);
-    int start, cnt;
-    tile_range(blockIdx.x - rq.tile_begin, rq.n, kTcTile, p.mini_batch, start, cnt);
-    const int64_t pos0 = rq.off + start;
-    const int L = p.sl.slots[rq.slot].L;
-    const int nb = (L + BN - 1) / BN;
+
+    const int n_tiles = p.sl.n_tiles;
 
     if (warp < 4) {
-        // ===================== queries, softmax, output =====================
+        // ===================== softmax, output =====================
         const int row = warp * 32 + lane;
-        {   // gather the item rows of the tile: 8 threads per row, 16 bytes each, 128B-swizzled K-major chunks
+        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        const float k2 = p.scale_log2;
+        bool ok = true;
+        uint32_t gb = 0;     // key blocks processed so far by this CTA (all tiles): selects score / P buffers and phases
+        int k = 0;           // tiles processed so far
+        if ((int)blockIdx.x < n_tiles) {
+            // The CTA's first tile has nobody to prefetch it: these four warps, idle until the first scores arrive, gather
+            // its queries (8 threads per row, 16 bytes each per 128-byte chunk); later tiles come from the gather warp.
+            const AttTile t = att_tile<BN>(p, blockIdx.x);
             const int sub = tid & 7, r0 = tid >> 3;
-            const uint32_t sw = (uint32_t)((sub ^ (r0 & 7)) << 4);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int r = r0 + 16 * i;
                 int id = -1;
-                if (r < cnt) {
-                    id = p.sl.ids[pos0 + r];
+                if (r < t.cnt) {
+                    id = p.sl.ids[t.pos0 + r];
                     if (id < 0 || (int64_t)id >= p.M) id = -1;
                 }
                 const uint8_t *g = p.E + (id >= 0 ? (size_t)id * (D * 2) + sub * 16 : 0);
+                const uint32_t dst = smem_u32(smQ) + (uint32_t)(r * 128) + (uint32_t)((sub ^ (r & 7)) << 4);
 #pragma unroll
-                for (int c = 0; c < C::kQChunks; ++c)
-                    cp_async16(smem_u32(smQ + c * 16384) + (uint32_t)(r * 128) + sw, g + c * 128, id >= 0 ? 16u : 0u);
+                for (int c = 0; c < C::kQChunks; ++c) cp_async16(dst + c * 16384, g + c * 128, id >= 0 ? 16u : 0u);
             }
-            cp_async_commit();
-            cp_async_wait<0>();
-            fence_proxy_async();
-            mbar_arrive(smem_u32(q_full));
+            cp_async_arrive_noinc(smem_u32(q_first));
         }
-        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
-        const float k2 = p.scale_log2;
-        float m_used = -INFINITY, l_sum = 0.f;
-        bool ok = true;
-        for (int j = 0; j < nb; ++j) {
-            const int b = j & 1;
-            const int valid_cols = min(BN, L - j * BN);
-            if (!mbar_wait(smem_u32(s_full + b), (uint32_t)((j >> 1) & 1), abort_flag)) {
-                ok = false;
-                break;
-            }
-            tc_fence_after();
-            const uint32_t ts = lane_base + (uint32_t)(b * BN);
-            // the row's BN scores: all loads first, one wait
-            uint32_t sc[BN];
-#pragma unroll
-            for (int c0 = 0; c0 < BN; c0 += 32) tmem_ld32(ts + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[32]>(&sc[c0]));
-            tmem_ld_wait();
-            // block maximum of the row (four independent chains)
-            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            if (valid_cols == BN) {
-#pragma unroll
-                for (int i = 0; i < BN; i += 4) {
-                    mx4[0] = fmaxf(mx4[0], __uint_as_float(sc[i]));
-                    mx4[1] = fmaxf(mx4[1], __uint_as_float(sc[i + 1]));
-                    mx4[2] = fmaxf(mx4[2], __uint_as_float(sc[i + 2]));
-                    mx4[3] = fmaxf(mx4[3], __uint_as_float(sc[i + 3]));
+        for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++k) {
+            const AttTile t = att_tile<BN>(p, tile);
+            const int L = p.sl.slots[t.slot].L;
+            float m_used = -INFINITY, l_sum = 0.f;
+            for (int j = 0; j < t.nb; ++j, ++gb) {
+                const int b = (int)(gb & 1u);
+                const int valid_cols = min(BN, L - j * BN);
+                if (!mbar_wait(smem_u32(s_full + b), (gb >> 1) & 1u, abort_flag)) {
+                    ok = false;
+                    break;
                 }
-            } else {
+                tc_fence_after();
+                const uint32_t ts = lane_base + (uint32_t)(b * BN);
+                // the row's BN scores: all loads first, one wait
+                uint32_t sc[BN];
 #pragma unroll
-                for (int i = 0; i < BN; ++i)
-                    if (i < valid_cols) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sc[i]));
-            }
-            const float mt = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * k2;
-            if (j == 0) {
-                m_used = mt;
-            } else {
-                const bool need = mt > m_used + 8.0f;
-                if (__any_sync(0xffffffffu, need)) {
-                    // raise the running maximum and rescale this warp's rows of O (rare)
-                    const float m_new = need ? mt : m_used;
-                    const float f = fast_exp2(m_used - m_new);
-                    l_sum *= f;
-                    m_used = m_new;
-                    if (!mbar_wait(smem_u32(pv_done + ((j - 1) & 1)), (uint32_t)(((j - 1) >> 1) & 1), abort_flag)) {
-                        ok = false;
-                        break;
+                for (int c0 = 0; c0 < BN; c0 += 32) tmem_ld32(ts + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[32]>(&sc[c0]));
+                tmem_ld_wait();
+                // block maximum of the row (four independent chains)
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                if (valid_cols == BN) {
+#pragma unroll
+                    for (int i = 0; i < BN; i += 4) {
+                        mx4[0] = fmaxf(mx4[0], __uint_as_float(sc[i]));
+                        mx4[1] = fmaxf(mx4[1], __uint_as_float(sc[i + 1]));
+                        mx4[2] = fmaxf(mx4[2], __uint_as_float(sc[i + 2]));
+                        mx4[3] = fmaxf(mx4[3], __uint_as_float(sc[i + 3]));
                     }
-                    tc_fence_after();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < BN; ++i)
+                        if (i < valid_cols) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sc[i]));
+                }
+                const float mt = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * k2;
+                if (j == 0) {
+                    m_used = mt;
+                } else {
+                    const bool need = mt > m_used + 8.0f;
+                    if (__any_sync(0xffffffffu, need)) {
+                        // raise the running maximum and rescale this warp's rows of O (rare)
+                        const float m_new = need ? mt : m_used;
+                        const float f = fast_exp2(m_used - m_new);
+                        l_sum *= f;
+                        m_used = m_new;
+                        if (!mbar_wait(smem_u32(pv_done + ((gb - 1) & 1u)), ((gb - 1) >> 1) & 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
 #pragma unroll 1
-                    for (int c0 = 0; c0 < D; c0 += 32) {
-                        uint32_t r[32];
-                        tmem_ld32(lane_base + (uint32_t)(C::kTmemO + c0), r);
-                        tmem_ld_wait();
+                        for (int c0 = 0; c0 < D; c0 += 32) {
+                            uint32_t r[32];
+                            tmem_ld32(lane_base + (uint32_t)(C::kTmemO + c0), r);
+                            tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
-                        tmem_st32(lane_base + (uint32_t)(C::kTmemO + c0), r);
+                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+                            tmem_st32(lane_base + (uint32_t)(C::kTmemO + c0), r);
+                        }
+                        tmem_st_wait();
                     }
-                    tmem_st_wait();
                 }
+                // the P buffer was last read by the P V product two blocks ago
+                if (gb >= 2 && !mbar_wait(smem_u32(pv_done + b), ((gb - 2) >> 1) & 1u, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                // probabilities -> bf16 A operand in shared memory
+                unsigned char *Pb = smP + b * C::kPBytes;
+                float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        float p0 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i]), k2, -m_used));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i + 1]), k2, -m_used));
+                        if (valid_cols != BN) {
+                            if (c0 + 2 * i >= valid_cols) p0 = 0.f;
+                            if (c0 + 2 * i + 1 >= valid_cols) p1 = 0.f;
+                        }
+                        ls4[i & 3] += p0 + p1;
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                        packed[i] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                    unsigned char *chunk = Pb + (c0 >> 6) * 16384 + row * 128;
+                    const int slot0 = (c0 & 63) >> 3;     // first 16-byte slot of these 32 columns inside the 128-byte row
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        *reinterpret_cast<uint4 *>(chunk + (((slot0 + q) ^ (row & 7)) << 4)) =
+                            make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                }
+                l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+                fence_proxy_async();
+                tc_fence_before();
+                mbar_arrive(smem_u32(p_full + b));
             }
-            // the P buffer of block j-2 must have been consumed
-            if (j >= 2 && !mbar_wait(smem_u32(pv_done + b), (uint32_t)(((j - 2) >> 1) & 1), abort_flag)) {
+            if (!ok || !mbar_wait(smem_u32(o_final), (uint32_t)(k & 1), abort_flag)) {
                 ok = false;
                 break;
             }
-            // probabilities -> bf16 A operand in shared memory
-            unsigned char *Pb = smP + b * C::kPBytes;
-            float ls4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t packed[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float p0 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i]), k2, -m_used));
-                    float p1 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i + 1]), k2, -m_used));
-                    if (valid_cols != BN) {
-                        if (c0 + 2 * i >= valid_cols) p0 = 0.f;
-                        if (c0 + 2 * i + 1 >= valid_cols) p1 = 0.f;
-                    }
-                    ls4[i & 3] += p0 + p1;
-                    const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                    packed[i] = *reinterpret_cast<const uint32_t *>(&h);
-                }
-                unsigned char *chunk = Pb + (c0 >> 6) * 16384 + row * 128;
-                const int slot0 = (c0 & 63) >> 3;     // first 16-byte slot of these 32 columns inside the 128-byte row
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    *reinterpret_cast<uint4 *>(chunk + (((slot0 + q) ^ (row & 7)) << 4)) =
-                        make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-            }
-            l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-            fence_proxy_async();
-            tc_fence_before();
-            mbar_arrive(smem_u32(p_full + b));
-        }
-        if (ok && mbar_wait(smem_u32(o_final), 0u, abort_flag)) {
             tc_fence_after();
             const float inv = 1.0f / l_sum;
             bool good = false;
-            if (row < cnt) {
-                const int id = p.sl.ids[pos0 + row];
+            if (row < t.cnt) {
+                const int id = p.sl.ids[t.pos0 + row];
                 good = id >= 0 && (int64_t)id < p.M;
             }
 #pragma unroll 1
@@ -225,7 +255,11 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                 uint32_t r[32];
                 tmem_ld32(lane_base + (uint32_t)(C::kTmemO + c0), r);
                 tmem_ld_wait();
-                if (row < cnt) {
+                if (c0 + 32 == D) {   // O is in registers: the next tile's first P V may overwrite the accumulator
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(o_free));
+                }
+                if (row < t.cnt) {
                     uint32_t packed[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
@@ -233,76 +267,154 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                                                                        good ? __uint_as_float(r[2 * i + 1]) * inv : 0.f);
                         packed[i] = *reinterpret_cast<const uint32_t *>(&h);
                     }
-                    uint4 *dst = reinterpret_cast<uint4 *>(p.X + (size_t)(pos0 + row) * p.x_stride + c0);
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.X + (size_t)(t.pos0 + row) * p.x_stride + c0);
 #pragma unroll
                     for (int q = 0; q < 4; ++q)
                         dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
                 }
             }
         }
-    } else if (warp == 4) {
+    } else if (warp == kAttMmaWarp) {
         // ===================== MMA issuer =====================
         if (lane == 0) {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(kTcTile, BN);
             constexpr uint32_t idesc_pv = umma_idesc_bf16_bmn(kTcTile, D);
-            bool ok = mbar_wait(smem_u32(q_full), 0u, abort_flag);
-            tc_fence_after();
-            auto issue_qk = [&](int j) -> bool {
-                const int s = j % kKvStages;
-                if (!mbar_wait(smem_u32(kv_full + s), (uint32_t)((j / kKvStages) & 1), abort_flag)) return false;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)((j & 1) * BN);
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint64_t adesc = umma_desc_sw128(smem_u32(smQ + (kk >> 2) * 16384)) + (uint64_t)(2 * (kk & 3));
-                    const uint64_t bdesc =
-                        umma_desc_sw128(smem_u32(smKV + s * C::kKvBytes + (kk >> 2) * C::kKvChunkBytes)) + (uint64_t)(2 * (kk & 3));
-                    umma_bf16(d_tmem, adesc, bdesc, idesc_qk, kk > 0 ? 1u : 0u);
+            bool ok = true;
+            // two cursors over the flat sequence of key blocks of this CTA's tiles: Q K^T runs one block ahead of P V
+            struct Cursor {
+                int tile, k, j, nb;
+                uint32_t gb;
+            };
+            auto open_tile = [&](Cursor &c) {
+                if (c.tile < n_tiles) c.nb = att_tile<BN>(p, c.tile).nb;
+            };
+            auto advance = [&](Cursor &c) {
+                ++c.gb;
+                if (++c.j == c.nb) {
+                    c.j = 0, c.tile += gridDim.x, ++c.k;
+                    open_tile(c);
                 }
-                umma_commit(smem_u32(s_full + (j & 1)));
+            };
+            // operand descriptors of buffer / stage 0; the others lie a fixed number of 16-byte units further
+            const uint64_t qdesc0 = umma_desc_sw128(smem_u32(smQ)), kdesc0 = umma_desc_sw128(smem_u32(smKV));
+            const uint64_t pdesc0 = umma_desc_sw128(smem_u32(smP));
+            const uint64_t vdesc0 = umma_desc_mn_sw128(smem_u32(smKV), C::kKvChunkBytes);
+            Cursor cq{(int)blockIdx.x, 0, 0, 0, 0u}, cp{(int)blockIdx.x, 0, 0, 0, 0u};
+            open_tile(cq);
+            cp.nb = cq.nb;
+            auto issue_qk = [&]() -> bool {
+                const int qb = cq.k % kQB;
+                if (cq.j == 0) {   // first block of a tile: its queries must have landed (cp.async, generic proxy)
+                    const bool got = cq.k == 0 ? mbar_wait(smem_u32(q_first), 0u, abort_flag)
+                                               : mbar_wait(smem_u32(q_full + qb), (uint32_t)(((cq.k - 1) / kQB) & 1), abort_flag);
+                    if (!got) return false;
+                    fence_proxy_async();
+                }
+                const int s = (int)(cq.gb % kS);
+                if (!mbar_wait(smem_u32(kv_full + s), (cq.gb / kS) & 1u, abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)((cq.gb & 1u) * BN);
+                const uint64_t qd = qdesc0 + (uint64_t)(uint32_t)(qb * (C::kQBytes >> 4));
+                const uint64_t kd = kdesc0 + (uint64_t)(uint32_t)(s * (C::kKvBytes >> 4));
+                umma_bf16(d_tmem, qd, kd, idesc_qk, 0u);
+#pragma unroll
+                for (int kk = 1; kk < D / 16; ++kk)
+                    umma_bf16_acc(d_tmem, qd + (uint64_t)((kk >> 2) * (16384 >> 4) + 2 * (kk & 3)),
+                                  kd + (uint64_t)((kk >> 2) * (C::kKvChunkBytes >> 4) + 2 * (kk & 3)), idesc_qk);
+                umma_commit(smem_u32(s_full + (cq.gb & 1u)));
+                if (cq.j == cq.nb - 1) umma_commit(smem_u32(q_empty + qb));   // the tile's queries are no longer needed
+                advance(cq);
                 return true;
             };
-            if (ok) ok = issue_qk(0);
-            for (int j = 0; ok && j < nb; ++j) {
-                if (j + 1 < nb && !issue_qk(j + 1)) {
+            if (cq.tile < n_tiles) ok = issue_qk();
+            while (ok && cp.tile < n_tiles) {
+                if (cq.tile < n_tiles && !issue_qk()) {
                     ok = false;
                     break;
                 }
-                if (!mbar_wait(smem_u32(p_full + (j & 1)), (uint32_t)((j >> 1) & 1), abort_flag)) {
+                if (!mbar_wait(smem_u32(p_full + (cp.gb & 1u)), (cp.gb >> 1) & 1u, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                // the first P V of a tile overwrites O: the previous tile's output must have been read
+                if (cp.j == 0 && cp.k > 0 && !mbar_wait(smem_u32(o_free), (uint32_t)((cp.k - 1) & 1), abort_flag)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                const int s = j % kKvStages;
+                const int s = (int)(cp.gb % kS);
                 const uint32_t o_tmem = tmem_base + (uint32_t)C::kTmemO;
+                const uint64_t pd = pdesc0 + (uint64_t)((cp.gb & 1u) * (uint32_t)(C::kPBytes >> 4));
+                const uint64_t vd = vdesc0 + (uint64_t)(uint32_t)(s * (C::kKvBytes >> 4));
+                umma_bf16(o_tmem, pd, vd, idesc_pv, cp.j > 0 ? 1u : 0u);
 #pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk) {
-                    const uint64_t adesc =
-                        umma_desc_sw128(smem_u32(smP + (j & 1) * C::kPBytes + (kk >> 2) * 16384)) + (uint64_t)(2 * (kk & 3));
-                    // V: 16 keys further = 16 rows x 128 bytes
-                    const uint64_t bdesc = umma_desc_mn_sw128(smem_u32(smKV + s * C::kKvBytes + kk * 2048), C::kKvChunkBytes);
-                    umma_bf16(o_tmem, adesc, bdesc, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
-                }
-                umma_commit(smem_u32(pv_done + (j & 1)));
+                for (int kk = 1; kk < BN / 16; ++kk)   // V: 16 keys further = 16 rows x 128 bytes
+                    umma_bf16_acc(o_tmem, pd + (uint64_t)((kk >> 2) * (16384 >> 4) + 2 * (kk & 3)), vd + (uint64_t)(kk * (2048 >> 4)),
+                                  idesc_pv);
+                umma_commit(smem_u32(pv_done + (cp.gb & 1u)));
                 umma_commit(smem_u32(kv_empty + s));
+                if (cp.j == cp.nb - 1) umma_commit(smem_u32(o_final));
+                advance(cp);
             }
-            if (ok) umma_commit(smem_u32(o_final));
+        }
+        __syncwarp();
+    } else if (warp == kAttTmaWarp) {
+        // ===================== key/value producer (TMA) =====================
+        if (lane == 0) {
+            uint32_t gb = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+                const AttTile t = att_tile<BN>(p, tile);
+                for (int j = 0; j < t.nb; ++j, ++gb) {
+                    const int s = (int)(gb % kS);
+                    if (!mbar_wait(smem_u32(kv_empty + s), ((gb / kS) & 1u) ^ 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    mbar_expect_tx(smem_u32(kv_full + s), (uint32_t)C::kKvBytes);
+#pragma unroll
+                    for (int c = 0; c < C::kQChunks; ++c)
+                        tma_load_3d(smem_u32(smKV + s * C::kKvBytes + c * C::kKvChunkBytes), &tmapS, smem_u32(kv_full + s), c * 64,
+                                    j * BN, t.slot);
+                }
+            }
         }
         __syncwarp();
     } else {
-        // ===================== key/value producer (TMA) =====================
-        if (lane == 0) {
-            for (int j = 0; j < nb; ++j) {
-                const int s = j % kKvStages;
-                if (!mbar_wait(smem_u32(kv_empty + s), (uint32_t)(((j / kKvStages) & 1) ^ 1), abort_flag)) break;
-                mbar_expect_tx(smem_u32(kv_full + s), (uint32_t)C::kKvBytes);
+        // ===================== query gather (32 threads) =====================
+        // 8 threads per row (16 bytes each per 128-byte chunk), rows lane / 8 + 4 i, 128B-swizzled K-major chunks
+        const int sub = lane & 7, r0 = lane >> 3;
+        int k = 1;
+        for (int tile = blockIdx.x + gridDim.x; tile < n_tiles; tile += gridDim.x, ++k) {
+            const int qb = k % kQB;
+            // the buffer's previous tenant is tile k - kQB (the first tile, tenant of buffer 0, included)
+            if (k >= kQB && !mbar_wait(smem_u32(q_empty + qb), (uint32_t)(((k - kQB) / kQB) & 1), abort_flag)) break;
+            const AttTile t = att_tile<BN>(p, tile);
+            unsigned char *q = smQ + qb * C::kQBytes;
+            // the tile's 128 ids with four coalesced loads per lane (rows lane, lane + 32, ...); -1 = zero row
+            int idv[4];
 #pragma unroll
-                for (int c = 0; c < C::kQChunks; ++c)
-                    tma_load_3d(smem_u32(smKV + s * C::kKvBytes + c * C::kKvChunkBytes), &tmapS, smem_u32(kv_full + s), c * 64,
-                                j * BN, rq.slot);
+            for (int u = 0; u < 4; ++u) {
+                const int r = lane + 32 * u;
+                int id = -1;
+                if (r < t.cnt) {
+                    id = p.sl.ids[t.pos0 + r];
+                    if (id < 0 || (int64_t)id >= p.M) id = -1;
+                }
+                idv[u] = id;
             }
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int r = r0 + 4 * i;                                   // row r: register r / 32 of lane r % 32
+                const int id = __shfl_sync(0xffffffffu, idv[i >> 3], r0 + 4 * (i & 7));
+                const uint8_t *g = p.E + (id >= 0 ? (size_t)id * (D * 2) + sub * 16 : 0);
+                const uint32_t dst = smem_u32(q) + (uint32_t)(r * 128) + (uint32_t)((sub ^ (r & 7)) << 4);
+#pragma unroll
+                for (int c = 0; c < C::kQChunks; ++c) cp_async16(dst + c * 16384, g + c * 128, id >= 0 ? 16u : 0u);
+            }
+            cp_async_arrive_noinc(smem_u32(q_full + qb));
         }
-        __syncwarp();
+        cp_async_wait_all();
     }
 
     if (*abort_flag) {
@@ -312,7 +424,7 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem_base, 512);
+    if (warp == kAttMmaWarp) tmem_dealloc(tmem_base, 512);
 }
 
 struct AttPlan {
@@ -373,11 +485,15 @@ cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
     p.sl = sl, p.E = (const uint8_t *)ctx->E, p.M = c.M, p.mini_batch = c.mini_batch;
     p.x_stride = x_stride, p.X = (__nv_bfloat16 *)X;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.d);
+    // One CTA per SM walking over many tiles saves the per-tile set-up and prefetches the next tile's queries, but its
+    // static tile assignment loses to the hardware's dynamic CTA scheduling when an SM gets only a few tiles (8.4 tiles
+    // per SM cost 9 tile times everywhere): below 16 tiles per SM every tile gets a CTA of its own.
+    const int grid = sl.n_tiles >= 148 * 16 ? 148 : sl.n_tiles;
     cudaError_t e;
     if (c.d == 128)
-        e = launch_pdl(k_att_tc<128, 128>, dim3(sl.n_tiles), dim3(kAttThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, p);
+        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(kAttThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, p);
     else
-        e = launch_pdl(k_att_tc<256, 64>, dim3(sl.n_tiles), dim3(kAttThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, p);
+        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(kAttThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, p);
     count_launch();
     return e;
 }
