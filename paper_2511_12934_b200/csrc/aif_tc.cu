@@ -135,7 +135,8 @@ __global__ void __launch_bounds__(256) k_cross_buckets(const int32_t *__restrict
 // ---- the layer kernel -----------------------------------------------------------------------------------------
 template <int MODE>
 __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const __grid_constant__ CUtensorMap tmapB,
-                                                                          const __grid_constant__ CUtensorMap tmapOut, const LayerParams p)
+                                                                          const __grid_constant__ CUtensorMap tmapOut,
+                                                                          const __grid_constant__ CUtensorMap tmapA, const LayerParams p)
 {
     using C = LayerCfg<MODE>;
     constexpr int G = C::G, NB = C::NB, kAcc = C::kAcc, kSA = C::kStagesA, kSB = C::kStagesB;
@@ -388,16 +389,17 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
         };
         // global sources of chunk kc: a base pointer and, per row, an offset in 16-byte units; rows whose bit in `mask`
         // is clear are zero-filled
+        // (dense chunks: consecutive rows of X / the previous activations, fetched as one TMA tile by the tile's first
+        // producer thread; tma_x < 0 marks every other kind)
         auto resolve = [&](int kc, const Rows &R, const int *ids, uint32_t (&raw)[8], bool have_raw, const uint8_t *&bp,
-                           uint32_t (&off)[8], uint32_t &mask) {
+                           uint32_t (&off)[8], uint32_t &mask, int &tma_x, int &tma_y) {
             const ChunkSrc src = p.src[kc];
+            tma_x = -1;
             if (src.kind == SRC_DENSE) {
-                const uint32_t row16 = (uint32_t)(p.x_row_bytes >> 4);
-                const uint32_t first = (R.pos0 + r0) * row16 + (uint32_t)(src.off >> 4) + sub;
-                bp = p.X;
-                mask = R.rowmask;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) off[i] = first + (uint32_t)(16 * i) * row16;
+                // rows beyond the tile bring other candidates' values along; their results are never stored
+                tma_x = R.rowmask != 0u || lp != 0 ? src.off >> 1 : -2;   // -2: the tile does not exist, nothing to fetch
+                tma_y = (int)R.pos0;
+                mask = 0;
             } else if (src.kind == SRC_ITEM) {
                 const uint32_t row16 = (uint32_t)(p.e_row_bytes >> 4), c16 = (uint32_t)(src.off >> 4) + sub;
                 bp = p.E;
@@ -435,12 +437,13 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
         int pend = -1;
         const uint8_t *bp = p.E;
         uint32_t off[8], raw[8], mask = 0;
+        int tma_x = -1, tma_y = 0;
 #pragma unroll
         for (int i = 0; i < 8; ++i) off[i] = 0, raw[i] = 0;
         if ((int)blockIdx.x < n_items) {
             load_rows(blockIdx.x, cur, pend);
             publish(0, pend);
-            resolve(0, cur, ids_s + gt * 128, raw, false, bp, off, mask);
+            resolve(0, cur, ids_s + gt * 128, raw, false, bp, off, mask, tma_x, tma_y);
             if (deep) fetch(1, cur, raw);
         }
         nxt = cur;
@@ -454,11 +457,16 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
                     ok = false;
                     break;
                 }
-                const uint32_t dst0 = smem_u32(smA + s * C::kAStage) + a_off;
+                if (tma_x == -1) {
+                    const uint32_t dst0 = smem_u32(smA + s * C::kAStage) + a_off;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const bool on = (mask >> i) & 1u;
-                    cp_async16(dst0 + (uint32_t)(i * 16 * 128), on ? bp + ((size_t)off[i] << 4) : p.E, on ? 16u : 0u);
+                    for (int i = 0; i < 8; ++i) {
+                        const bool on = (mask >> i) & 1u;
+                        cp_async16(dst0 + (uint32_t)(i * 16 * 128), on ? bp + ((size_t)off[i] << 4) : p.E, on ? 16u : 0u);
+                    }
+                } else if (lp == 0 && tma_x >= 0) {
+                    mbar_expect_tx_only(smem_u32(full_a + s), (uint32_t)kABytes);
+                    tma_load_2d(smem_u32(smA + s * C::kAStage + gt * kABytes), &tmapA, smem_u32(full_a + s), tma_x, tma_y);
                 }
                 // the stage's barrier receives this thread's arrival when its copies have landed: no thread waits for them
                 cp_async_arrive_noinc(smem_u32(full_a + s));
@@ -466,8 +474,8 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
                 if (kc == 0 && has_next) publish(buf ^ 1, pend);
                 // sources of the next chunk from the buckets fetched one iteration ago; then start the fetch for the
                 // chunk after it, so that its latency is covered by a whole iteration
-                if (kc + 1 < p.n_k) resolve(kc + 1, cur, ids_cur, raw, deep, bp, off, mask);
-                else if (has_next) resolve(0, nxt, ids_nxt, raw, deep, bp, off, mask);
+                if (kc + 1 < p.n_k) resolve(kc + 1, cur, ids_cur, raw, deep, bp, off, mask, tma_x, tma_y);
+                else if (has_next) resolve(0, nxt, ids_nxt, raw, deep, bp, off, mask, tma_x, tma_y);
                 if (deep) {
                     if (kc + 2 < p.n_k) fetch(kc + 2, cur, raw);
                     else if (has_next) fetch(kc + 2 - p.n_k, nxt, raw);
@@ -879,10 +887,23 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
         const bool wide = !pair && p.n_nchunks % 2 == 0 && single > 148;
         const int items = pair ? ((sl.n_tiles + 1) / 2) * p.n_nchunks : wide ? single / 2 : single;
         const int grid = items < 148 ? items : 148;
+        // load source of the dense chunks: X (layer 1) or the previous activations, 64-column x 128-row tiles
+        CUtensorMap tmap_a = pl->tmap[k];
+        const int dense_w = k == 0 ? pl->x_cols : c.hidden[k - 1];
+        if (dense_w > 0) {
+            const cuuint64_t dims[2] = {(cuuint64_t)dense_w, (cuuint64_t)sc.rows};
+            const cuuint64_t strides[1] = {(cuuint64_t)dense_w * 2};
+            const cuuint32_t box[2] = {64, 128};
+            const cuuint32_t estr[2] = {1, 1};
+            CUresult r = encode_fn()(&tmap_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint8_t *>(p.X), dims, strides, box, estr,
+                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+        }
         cudaError_t e;
-        if (pair) e = launch_pdl(k_layer_tc<1>, dim3(grid), dim3(LayerCfg<1>::kThreads), LayerCfg<1>::kSmem, st, pl->tmap[k], tmap_out, p);
-        else if (wide) e = launch_pdl(k_layer_tc<2>, dim3(grid), dim3(LayerCfg<2>::kThreads), LayerCfg<2>::kSmem, st, pl->tmap[k], tmap_out, p);
-        else e = launch_pdl(k_layer_tc<0>, dim3(grid), dim3(LayerCfg<0>::kThreads), LayerCfg<0>::kSmem, st, pl->tmap[k], tmap_out, p);
+        if (pair) e = launch_pdl(k_layer_tc<1>, dim3(grid), dim3(LayerCfg<1>::kThreads), LayerCfg<1>::kSmem, st, pl->tmap[k], tmap_out, tmap_a, p);
+        else if (wide) e = launch_pdl(k_layer_tc<2>, dim3(grid), dim3(LayerCfg<2>::kThreads), LayerCfg<2>::kSmem, st, pl->tmap[k], tmap_out, tmap_a, p);
+        else e = launch_pdl(k_layer_tc<0>, dim3(grid), dim3(LayerCfg<0>::kThreads), LayerCfg<0>::kSmem, st, pl->tmap[k], tmap_out, tmap_a, p);
         count_launch();
         timing_mark(ctx, names[k], st);
         if (e != cudaSuccess) return e;

@@ -28,6 +28,11 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 }
 // One try: returns at once when the phase is complete.  Otherwise the hardware may suspend the thread (it then
 // occupies no issue slot) until the phase completes or `suspend_ns` have passed, whichever comes first.
+// Announces `bytes` more asynchronous-copy bytes for the current phase without arriving.
+__device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t suspend_ns = 20000u)
 {
     uint32_t ok;
