@@ -66,10 +66,12 @@ struct LayerParams {
 //           per candidate (large launches)
 //   MODE 2  one tile, two slices: one gathered A chunk feeds both slices, so the tile's rows are gathered once instead
 //           of once per slice (launches that would otherwise need a second round of items)
+//   MODE 3  as MODE 1 with a deeper A ring and a shallower B ring, for the first layer: its cross-feature rows come
+//           from per-request tables that may live in HBM, the weights from L2
 // A and B have rings of their own: gathered rows have the longer latency and the smaller chunks.
 template <int MODE>
 struct LayerCfg {
-    static constexpr int G = MODE == 1 ? 2 : 1;          // tiles per work item
+    static constexpr int G = (MODE == 1 || MODE == 3) ? 2 : 1;   // tiles per work item
     static constexpr int NB = MODE == 2 ? 2 : 1;         // output slices per work item
     static constexpr int kAcc = G * NB;                  // accumulators a work item fills
     static constexpr int kStagesA = MODE == 1 ? 3 : 4;
@@ -82,6 +84,7 @@ struct LayerCfg {
     static constexpr int kBWarp = kProdWarp0 + 4 * G;
     static constexpr int kThreads = (kBWarp + 1) * 32;
     static constexpr int kSlabs = MODE == 0 ? 2 : 1;    // output staging slabs (2 KB) per epilogue warp
+    static_assert(1024 + kStagesA * kAStage + kStagesB * kBStage + kEpiWarps * kSlabs * 2048 + 8192 <= 227 * 1024, "shared memory");
     static constexpr size_t kSmem = 1024 + (size_t)kStagesA * kAStage + (size_t)kStagesB * kBStage + (2 * kStagesA + 2 * kStagesB + 4) * 8 +
                                     32 + 2 * kAcc * 256 * 4 + kEpiWarps * kSlabs * 2048 + 2 * G * 128 * 4;
 };
@@ -730,6 +733,8 @@ cudaError_t tc_prepare_context(aif_ctx *ctx)
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_layer_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LayerCfg<2>::kSmem);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_layer_tc<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LayerCfg<3>::kSmem);
+    if (e != cudaSuccess) return e;
     // tensor maps over the packed weights: [H x in_w] bf16, box = 64 columns x n_cols rows, 128-byte swizzle
     EncodeFn enc = encode_fn();
     if (!enc) return cudaErrorNotSupported;
@@ -901,7 +906,9 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
             if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
         }
         cudaError_t e;
-        if (pair) e = launch_pdl(k_layer_tc<1>, dim3(grid), dim3(LayerCfg<1>::kThreads), LayerCfg<1>::kSmem, st, pl->tmap[k], tmap_out, tmap_a, p);
+        if (pair && k == 0 && (c.blocks & AIF_BLK_CROSS))
+            e = launch_pdl(k_layer_tc<3>, dim3(grid), dim3(LayerCfg<3>::kThreads), LayerCfg<3>::kSmem, st, pl->tmap[k], tmap_out, tmap_a, p);
+        else if (pair) e = launch_pdl(k_layer_tc<1>, dim3(grid), dim3(LayerCfg<1>::kThreads), LayerCfg<1>::kSmem, st, pl->tmap[k], tmap_out, tmap_a, p);
         else if (wide) e = launch_pdl(k_layer_tc<2>, dim3(grid), dim3(LayerCfg<2>::kThreads), LayerCfg<2>::kSmem, st, pl->tmap[k], tmap_out, tmap_a, p);
         else e = launch_pdl(k_layer_tc<0>, dim3(grid), dim3(LayerCfg<0>::kThreads), LayerCfg<0>::kSmem, st, pl->tmap[k], tmap_out, tmap_a, p);
         count_launch();
