@@ -209,9 +209,12 @@ int aif_score(aif_ctx *ctx, const aif_user_state *state, const int32_t *cand_ids
 int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *states, const int32_t *cand_ids,
                     const int64_t *offsets, float *logits, aif_stream stream);
 
-/* aif_score for callers whose buffers live in host memory: copies host_ids (host, pinned for best speed) to
- * the device, scores, copies the logits back into host_logits, all on `stream`; returns after the stream has
- * drained.  This is the end-to-end form the benchmark times. */
+/* aif_score for callers whose buffers live in host memory: brings host_ids (host) to the device, scores, leaves the
+ * logits in host_logits (host), all on `stream`; returns after the stream has drained.  If both buffers are page-locked
+ * and mapped into the device's address space (cudaHostAlloc / cudaHostRegister; pinned torch tensors are), a small
+ * kernel reads the ids across the bus and the last scoring kernel writes the logits straight into host_logits;
+ * otherwise both are staged with cudaMemcpyAsync through buffers of the context.  This is the end-to-end form the
+ * benchmark times. */
 int aif_score_host(aif_ctx *ctx, const aif_user_state *state, const int32_t *host_ids, int32_t n,
                    float *host_logits, aif_stream stream);
 

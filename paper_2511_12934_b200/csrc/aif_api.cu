@@ -506,10 +506,27 @@ int aif_score_host(aif_ctx *ctx, const aif_user_state *state, const int32_t *hos
     if (!host_ids || !host_logits) return AIF_ERR_ARG;
     DeviceGuard g(ctx->device);
     cudaStream_t st = as_stream(stream);
-    AIF_CUDA(cudaMemcpyAsync(ctx->ids_stage, host_ids, (size_t)n * 4, cudaMemcpyHostToDevice, st));
-    rc = aif_score(ctx, state, ctx->ids_stage, n, ctx->logits_stage, stream);
-    if (rc != AIF_OK) return rc;
-    AIF_CUDA(cudaMemcpyAsync(host_logits, ctx->logits_stage, (size_t)n * 4, cudaMemcpyDeviceToHost, st));
+    // Page-locked buffers that are mapped into the device's address space need no copy engine: a small kernel pulls
+    // the ids over, and the last scoring kernel writes the logits straight into the host buffer.
+    auto mapped = [](const void *hp) -> void * {
+        cudaPointerAttributes a{};
+        if (cudaPointerGetAttributes(&a, hp) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
+    };
+    void *d_ids = mapped(host_ids), *d_out = mapped(host_logits);
+    if (d_ids && d_out) {
+        AIF_CUDA(launch_stage_ids(static_cast<const int32_t *>(d_ids), ctx->ids_stage, n, st));
+        rc = aif_score(ctx, state, ctx->ids_stage, n, static_cast<float *>(d_out), stream);
+        if (rc != AIF_OK) return rc;
+    } else {
+        AIF_CUDA(cudaMemcpyAsync(ctx->ids_stage, host_ids, (size_t)n * 4, cudaMemcpyHostToDevice, st));
+        rc = aif_score(ctx, state, ctx->ids_stage, n, ctx->logits_stage, stream);
+        if (rc != AIF_OK) return rc;
+        AIF_CUDA(cudaMemcpyAsync(host_logits, ctx->logits_stage, (size_t)n * 4, cudaMemcpyDeviceToHost, st));
+    }
     AIF_CUDA(cudaStreamSynchronize(st));
     return AIF_OK;
 }

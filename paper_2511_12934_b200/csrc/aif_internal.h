@@ -165,6 +165,7 @@ ModelDev make_model(const aif_ctx *ctx);
 // aif_simt.cu
 cudaError_t launch_scatter_rows(const aif_ctx *ctx, const int32_t *ids, int64_t n, const void *rows, const void *bea_w,
                                 const uint8_t *sig, cudaStream_t st);
+cudaError_t launch_stage_ids(const int32_t *mapped_src, int32_t *dst, int n, cudaStream_t st);
 cudaError_t launch_gather_rows(const aif_ctx *ctx, const int32_t *ids, int64_t n, void *out, cudaStream_t st);
 cudaError_t launch_transpose(const void *in, void *out, int rows, int cols, size_t el, cudaStream_t st);
 cudaError_t launch_score_simt(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st);

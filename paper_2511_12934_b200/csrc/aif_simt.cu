@@ -58,6 +58,20 @@ __global__ void __launch_bounds__(256) k_gather_rows(const uint4 *__restrict__ t
     }
 }
 
+// Copies candidate ids from page-locked host memory that is mapped into the device's address space.
+__global__ void __launch_bounds__(256) k_stage_ids(const int32_t *__restrict__ src, int32_t *__restrict__ dst, int n)
+{
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) dst[i] = src[i];
+}
+
+cudaError_t launch_stage_ids(const int32_t *mapped_src, int32_t *dst, int n, cudaStream_t st)
+{
+    const int grid = (n + 255) / 256 < 148 ? (n + 255) / 256 : 148;
+    k_stage_ids<<<grid, 256, 0, st>>>(mapped_src, dst, n);
+    count_launch();
+    return cudaGetLastError();
+}
+
 static int grid_for(int64_t items, int per_block, int cap)
 {
     int64_t g = (items + per_block - 1) / per_block;

@@ -299,3 +299,23 @@ def test_a_wait_that_runs_out_sets_the_timeout_bit_and_leaves_the_context_usable
         srv.ctx.selftest_bounded_wait(0)
     assert e.value.code == B.ERR_ARG
     srv.close()
+
+
+def test_score_host_with_pinned_and_with_pageable_buffers():
+    """aif_score_host takes the zero-copy route for pinned (mapped) buffers and the staged route for pageable ones;
+    both give the device-buffer result bit for bit."""
+    wl = helpers.MINI["c2"].with_(name="hostbuf", N=777)
+    weights, table, srv, oracle = _setup(wl)
+    rq = synth.make_request(wl, 0)
+    ids = synth.IdSampler(wl).request_ids(0)
+    st = srv.precompute(1, srv.upload_request(rq, B.USER_PROJECTED))
+    ref = srv.score_ids(st, ids)
+    for pinned in (True, False):
+        h_ids = torch.from_numpy(ids.copy())
+        h_out = torch.full((len(ids),), float("nan"), dtype=torch.float32)
+        if pinned:
+            h_ids, h_out = h_ids.pin_memory(), h_out.pin_memory()
+        srv.ctx.score_host(st, h_ids, h_out)
+        assert np.array_equal(h_out.numpy(), ref)
+    assert srv.ctx.poll_status() == 0
+    srv.close()
