@@ -180,6 +180,8 @@ int aif_item_nearline_refresh(aif_ctx *ctx, const int32_t *ids, int64_t n, const
  * the user columns of the first layer again.  Records a "ready" event that aif_score waits on.
  * in: host struct of device pointers; the inputs must stay valid until the work on side_stream is done.
  * request_key: the caller's request identity (Section 3.4 keys the cached state by request), kept in the handle.
+ * Calls with AIF_USER_RAW inputs share scratch of the context (the attention rows of eq. 2): issue them on one side
+ * stream, or order them with events, so that two of them never run on the GPU at the same time.
  * Errors: AIF_ERR_SHAPE (L < 1 or L > L_max), AIF_ERR_OOM (no free slot), AIF_ERR_NOT_READY (no weights). */
 int aif_user_precompute(aif_ctx *ctx, uint64_t request_key, const aif_user_inputs *in, int32_t L,
                         aif_user_state **out, aif_stream side_stream);

@@ -224,7 +224,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     TRY(dev_alloc(ctx, (void **)&ctx->b_b, (size_t)c.d * 4, true));
 
     // user-state arena: fixed-size slots in one allocation
-    struct Off { size_t u, u32, S, T, V, sig, pu, smallB, prof, partial, end; } o{};
+    struct Off { size_t u, u32, S, T, V, sig, pu, smallB, prof, partial, ppart, end; } o{};
     size_t p = 0;
     auto take = [&](size_t bytes) { size_t at = p; p += align_up(bytes ? bytes : 16, 256); return at; };
     o.u = take((size_t)c.d * el);
@@ -237,6 +237,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     o.smallB = take((size_t)c.hidden[0] * 16 * 2);
     o.prof = take((size_t)c.d * 4);
     o.partial = take((size_t)kUserPartials * c.d * 4);
+    o.ppart = take((size_t)kProfParts * (c.d + 2) * 4);
     o.end = p;
     ctx->slot_bytes = o.end;
     TRY(dev_alloc(ctx, (void **)&ctx->arena, ctx->slot_bytes * (size_t)c.max_user_states, true));
@@ -250,7 +251,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
         hs.dev.u = base + o.u, hs.dev.u32 = (const float *)(base + o.u32), hs.dev.S = base + o.S;
         hs.dev.T = base + o.T, hs.dev.V = base + o.V, hs.dev.sigS = (const uint8_t *)(base + o.sig);
         hs.dev.p_u = (const float *)(base + o.pu), hs.dev.smallB = base + o.smallB, hs.dev.L = 0;
-        hs.prof_hat = (float *)(base + o.prof), hs.partial = (float *)(base + o.partial);
+        hs.prof_hat = (float *)(base + o.prof), hs.partial = (float *)(base + o.partial), hs.ppart = (float *)(base + o.ppart);
         cudaError_t e = cudaEventCreateWithFlags(&hs.ev, cudaEventDisableTiming);
         if (e != cudaSuccess) {
             aif_destroy(ctx);

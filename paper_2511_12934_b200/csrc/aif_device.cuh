@@ -90,7 +90,7 @@ __device__ __forceinline__ float dot_row(const __nv_bfloat16 *row, const float *
 template <typename T>
 __device__ void warp_interact(const float *q, const T *S, int L, int d, float scale, bool do_att, bool do_lsh,
                               bool do_tiers, const uint32_t *sig_q, const uint8_t *sigS, int lsh_bits, int n_tiers,
-                              int *tiers, float att[8], float din[8])
+                              int *tiers, float att[8], float din[8], float *ml_out = nullptr)
 {
     const int lane = threadIdx.x & 31, dq = d >> 5, words = lsh_bits >> 5;
     float m = -INFINITY, l = 0.f;
@@ -140,9 +140,13 @@ __device__ void warp_interact(const float *q, const T *S, int L, int d, float sc
         }
     }
     if (do_att) {
-        const float inv = 1.0f / l;
+        if (ml_out) {   // partial result over a slice of the keys: left unnormalised, with its maximum and sum
+            if (lane == 0) ml_out[0] = m, ml_out[1] = l;
+        } else {
+            const float inv = 1.0f / l;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) att[c] *= inv;
+            for (int c = 0; c < 8; ++c) att[c] *= inv;
+        }
     }
 }
 

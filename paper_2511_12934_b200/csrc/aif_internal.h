@@ -78,9 +78,11 @@ struct HostSlot {
     // scratch for the user-side network
     float *prof_hat = nullptr;   // [d]
     float *partial = nullptr;    // [kUserPartials x d]
+    float *ppart = nullptr;      // [kProfParts x (d + 2)]: per key slice, unnormalised attention row, maximum, sum
 };
 
-constexpr int kUserPartials = 1184;   // warps of the self-attention launch (148 SMs x 8)
+constexpr int kUserPartials = 1184;
+constexpr int kProfParts = 256;      // warps (key slices) of the profile-attention launch   // warps of the self-attention launch (148 SMs x 8)
 
 // Optional per-kernel timing of the last scoring call (events on the call's stream).
 struct KernelTiming {
@@ -181,6 +183,9 @@ void tc_destroy_context(aif_ctx *ctx);
 bool tc_att_supported(const aif_config &cfg);
 cudaError_t tc_att_prepare(aif_ctx *ctx);
 void tc_att_destroy(aif_ctx *ctx);
+// eq. 2's attention rows softmax(S S^T / sqrt(d)) S of one user state with the same kernel (queries = the sequence rows);
+// *rows_out: [L x d] bf16 in scratch of the attention plan, valid until the next call
+cudaError_t launch_self_att_tc(const aif_ctx *ctx, int slot_index, int L, cudaStream_t st, const void **rows_out);
 cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, void *X, int x_stride);
 cudaError_t tc_prepare_weights(aif_ctx *ctx, const aif_weights *w, cudaStream_t st);
 cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t total_candidates, cudaStream_t st);

@@ -1,5 +1,7 @@
 // CUDA-core kernels of libaif: table scatter / gather, the general scoring kernel (any storage type, all
 // interaction blocks, fp32 arithmetic) and the user-side network.  The tensor-core kernels live in aif_tc.cu.
+#include <type_traits>
+
 #include "aif_internal.h"
 #include "aif_device.cuh"
 
@@ -367,28 +369,33 @@ __global__ void k_user_project(const T *__restrict__ seq, const T *__restrict__ 
 }
 
 // eq. 2.  Warp g handles rows g, g + n_warps, ...: attention over the whole sequence, FFN, and a running sum
-// for the mean pooling; partial[g] holds the warp's sum (summed later in a fixed order).
+// for the mean pooling; partial[g] holds the warp's sum (summed later in a fixed order).  att_rows != nullptr: the
+// attention rows softmax(S S^T / sqrt(d)) S were already computed by the tensor-core attention kernel.
 template <typename T>
 __global__ void __launch_bounds__(256) k_user_self(const T *__restrict__ S, int L, int d, const T *__restrict__ Wa_t,
                                                    const float *__restrict__ b_a, const T *__restrict__ Wb_t,
                                                    const float *__restrict__ b_b, float *__restrict__ partial,
-                                                   int n_warps)
+                                                   int n_warps, const T *__restrict__ att_rows)
 {
     extern __shared__ float sm[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = blockIdx.x * 8 + warp, dq = d >> 5;
-    float *q = sm + (size_t)warp * 3 * d, *ctx = q + d, *hid = ctx + d;
+    float *q = sm + (size_t)warp * 3 * d, *ctx = q + d;
     float pooled[8];
 #pragma unroll
     for (int c = 0; c < 8; ++c) pooled[c] = 0.f;
     const float scale = rsqrtf((float)d);
     for (int i = g; i < L; i += n_warps) {
-        for (int k = lane; k < d; k += 32) q[k] = to_f(S[(size_t)i * d + k]);
-        __syncwarp();
-        float att[8], din[8];
-        warp_interact<T>(q, S, L, d, scale, true, false, false, nullptr, nullptr, 0, 0, nullptr, att, din);
+        if (att_rows) {
+            for (int k = lane; k < d; k += 32) ctx[k] = to_f(att_rows[(size_t)i * d + k]);
+        } else {
+            for (int k = lane; k < d; k += 32) q[k] = to_f(S[(size_t)i * d + k]);
+            __syncwarp();
+            float att[8], din[8];
+            warp_interact<T>(q, S, L, d, scale, true, false, false, nullptr, nullptr, 0, 0, nullptr, att, din);
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
-            if (c < dq) ctx[lane + 32 * c] = att[c];
+            for (int c = 0; c < 8; ++c)
+                if (c < dq) ctx[lane + 32 * c] = att[c];
+        }
         __syncwarp();
 #pragma unroll
         for (int c = 0; c < 8; ++c)
@@ -396,16 +403,9 @@ __global__ void __launch_bounds__(256) k_user_self(const T *__restrict__ S, int 
                 const int j = lane + 32 * c;
                 float acc = b_a[j];
                 for (int k = 0; k < d; ++k) acc = fmaf(ctx[k], to_f(Wa_t[(size_t)k * d + j]), acc);
-                hid[j] = fmaxf(acc, 0.f);
-            }
-        __syncwarp();
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-            if (c < dq) {
-                const int j = lane + 32 * c;
-                float acc = b_b[j];
-                for (int k = 0; k < d; ++k) acc = fmaf(hid[k], to_f(Wb_t[(size_t)k * d + j]), acc);
-                pooled[c] += acc;
+                // the second FFN layer is linear, so it commutes with the mean pooling: pool the hidden activations
+                // here and apply W_b once, in k_user_finish
+                pooled[c] += fmaxf(acc, 0.f);
             }
         __syncwarp();
     }
@@ -416,6 +416,30 @@ __global__ void __launch_bounds__(256) k_user_self(const T *__restrict__ S, int 
     }
 }
 
+// eq. 3 in slices: warp g attends the profile query to keys [g * slice, (g + 1) * slice) and leaves its unnormalised
+// output row with the slice's maximum and sum; k_user_finish merges the slices.
+template <typename T>
+__global__ void __launch_bounds__(256) k_user_prof(const T *__restrict__ S, int L, int d, const float *__restrict__ prof_hat,
+                                                   int slice, float *__restrict__ ppart)
+{
+    __shared__ float q[256];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = blockIdx.x * 8 + warp, dq = d >> 5;
+    for (int k = threadIdx.x; k < d; k += 256) q[k] = prof_hat[k];
+    __syncthreads();
+    float *out = ppart + (size_t)g * (d + 2);
+    const int start = g * slice, len = min(slice, L - start);
+    if (len <= 0) {
+        if (lane == 0) out[d] = -INFINITY, out[d + 1] = 0.f;
+        return;
+    }
+    float att[8], din[8];
+    warp_interact<T>(q, S + (size_t)start * d, len, d, rsqrtf((float)d), true, false, false, nullptr, nullptr, 0, 0, nullptr, att,
+                     din, out + d);
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+        if (c < dq) out[lane + 32 * c] = att[c];
+}
+
 // eq. 3, the combined vector, and the cached first-layer partial product p_u = W1[:, 0:d] u + b1.
 // raw = 1: u = mean-pooled self-attention + profile attention.  raw = 0: u is given (u_in, storage type).
 template <typename T>
@@ -424,25 +448,43 @@ __global__ void __launch_bounds__(256) k_user_finish(int raw, const T *__restric
                                                      const float *__restrict__ partial, int n_warps,
                                                      const T *__restrict__ u_in, T *__restrict__ u_out,
                                                      float *__restrict__ u32, const T *__restrict__ W1t,
-                                                     const float *__restrict__ b1, int H1, float *__restrict__ p_u)
+                                                     const float *__restrict__ b1, int H1, float *__restrict__ p_u,
+                                                     const T *__restrict__ Wb_t, const float *__restrict__ b_b,
+                                                     const float *__restrict__ ppart)
 {
     __shared__ float q[256], uprof[256], us[256];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, dq = d >> 5;
     if (raw) {
-        for (int k = tid; k < d; k += 256) q[k] = prof_hat[k];
-        __syncthreads();
-        if (warp == 0) {
-            float att[8], din[8];
-            warp_interact<T>(q, S, L, d, rsqrtf((float)d), true, false, false, nullptr, nullptr, 0, 0, nullptr, att, din);
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-                if (c < dq) uprof[lane + 32 * c] = att[c];
+        // merge the key slices of the profile attention: softmax over all keys from per-slice maxima and sums
+        {
+            float m_all = -INFINITY;
+            for (int g = 0; g < kProfParts; ++g) m_all = fmaxf(m_all, ppart[(size_t)g * (d + 2) + d]);
+            float den = 0.f;
+            for (int g = 0; g < kProfParts; ++g) {
+                const float l = ppart[(size_t)g * (d + 2) + d + 1];
+                if (l > 0.f) den += l * expf(ppart[(size_t)g * (d + 2) + d] - m_all);
+            }
+            for (int k = tid; k < d; k += 256) {
+                float num = 0.f;
+                for (int g = 0; g < kProfParts; ++g)
+                    if (ppart[(size_t)g * (d + 2) + d + 1] > 0.f)
+                        num = fmaf(expf(ppart[(size_t)g * (d + 2) + d] - m_all), ppart[(size_t)g * (d + 2) + k], num);
+                uprof[k] = num / den;
+            }
         }
         __syncthreads();
+        // mean over the sequence of the hidden FFN activations (the warps' partial sums, in a fixed order) ...
         for (int k = tid; k < d; k += 256) {
             float acc = 0.f;
             for (int g = 0; g < n_warps; ++g) acc += partial[(size_t)g * d + k];
-            const float u = acc / (float)L + uprof[k];
+            q[k] = acc / (float)L;
+        }
+        __syncthreads();
+        // ... through the second FFN layer, plus the profile attention: the combined user vector
+        for (int k = tid; k < d; k += 256) {
+            float acc = b_b[k];
+            for (int j = 0; j < d; ++j) acc = fmaf(q[j], to_f(Wb_t[(size_t)j * d + k]), acc);
+            const float u = acc + uprof[k];
             us[k] = u;
             u32[k] = u;
             from_f(u_out[k], u);
@@ -479,12 +521,6 @@ static cudaError_t user_network_typed(const aif_ctx *ctx, HostSlot &hs, int slot
                                                                     c.dU, d, S, hs.prof_hat);
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        const int n_warps = kUserPartials;
-        k_user_self<T><<<n_warps / 8, 256, 8 * 3 * d * sizeof(float), st>>>(S, L, d, (const T *)ctx->Wa_t, ctx->b_a,
-                                                                            (const T *)ctx->Wb_t, ctx->b_b, hs.partial,
-                                                                            n_warps);
-        count_launch();
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
     } else {
         if ((e = cudaMemcpyAsync(S, in->seq, (size_t)L * d * sizeof(T), cudaMemcpyDeviceToDevice, st)) != cudaSuccess) return e;
         if ((e = cudaMemcpyAsync((void *)hs.dev.u, in->profile, (size_t)d * sizeof(T), cudaMemcpyDeviceToDevice, st)) !=
@@ -495,12 +531,32 @@ static cudaError_t user_network_typed(const aif_ctx *ctx, HostSlot &hs, int slot
         const int L_pad = (L + 127) / 128 * 128 < c.L_max ? (L + 127) / 128 * 128 : c.L_max;
         if (L_pad > L && (e = cudaMemsetAsync(S + (size_t)L * d, 0, (size_t)(L_pad - L) * d * sizeof(T), st)) != cudaSuccess) return e;
     }
-    k_user_finish<T><<<1, 256, 0, st>>>(raw ? 1 : 0, S, L, d, hs.prof_hat, hs.partial, kUserPartials,
-                                        (const T *)in->profile, (T *)hs.dev.u, (float *)hs.dev.u32, (const T *)ctx->Wt[0],
-                                        ctx->b[0], H1, (float *)hs.dev.p_u);
+    // the slot's length is set here already: the tensor-core self-attention below reads it like any scoring launch
+    k_set_slot_len<<<1, 1, 0, st>>>(ctx->slots_dev, slot_index, L);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    k_set_slot_len<<<1, 1, 0, st>>>(ctx->slots_dev, slot_index, L);
+    if (raw) {
+        // eq. 2: the attention rows on the tensor cores where the shape allows, else inside k_user_self
+        const T *att_rows = nullptr;
+        if (std::is_same<T, __nv_bfloat16>::value && ctx->tc_att_plan) {
+            const void *rows = nullptr;
+            if ((e = launch_self_att_tc(ctx, slot_index, L, st, &rows)) != cudaSuccess) return e;
+            att_rows = static_cast<const T *>(rows);
+        }
+        const int slice = ((L + kProfParts - 1) / kProfParts + 31) / 32 * 32;
+        k_user_prof<T><<<kProfParts / 8, 256, 0, st>>>(S, L, d, hs.prof_hat, slice, hs.ppart);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        const int n_warps = kUserPartials;
+        k_user_self<T><<<n_warps / 8, 256, 8 * 3 * d * sizeof(float), st>>>(S, L, d, (const T *)ctx->Wa_t, ctx->b_a,
+                                                                            (const T *)ctx->Wb_t, ctx->b_b, hs.partial,
+                                                                            n_warps, att_rows);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    k_user_finish<T><<<1, 256, 0, st>>>(raw ? 1 : 0, S, L, d, hs.prof_hat, hs.partial, kUserPartials,
+                                        (const T *)in->profile, (T *)hs.dev.u, (float *)hs.dev.u32, (const T *)ctx->Wt[0],
+                                        ctx->b[0], H1, (float *)hs.dev.p_u, (const T *)ctx->Wb_t, ctx->b_b, hs.ppart);
     count_launch();
     return cudaGetLastError();
 }

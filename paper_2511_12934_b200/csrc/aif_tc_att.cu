@@ -430,7 +430,14 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
 struct AttPlan {
     CUtensorMap tmap;
     int bn = 0;
+    __nv_bfloat16 *self_rows = nullptr;   // [L_max + 128][d]: attention rows of eq. 2 for the user state being computed
+    int32_t *iota = nullptr;              // 0, 1, 2, ...: the "candidate ids" of that launch are the sequence positions
 };
+
+__global__ void k_iota(int32_t *out, int n)
+{
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) out[i] = i;
+}
 
 }  // namespace
 
@@ -457,6 +464,20 @@ cudaError_t tc_att_prepare(aif_ctx *ctx)
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     cudaError_t e;
+    {   // scratch of the user-side self-attention
+        const size_t rows = (size_t)c.L_max + kTcTile;
+        void *ptr = nullptr;
+        if ((e = cudaMalloc(&ptr, rows * c.d * 2)) != cudaSuccess) return e;
+        ctx->allocations.push_back(ptr), ctx->device_bytes += (int64_t)(rows * c.d * 2);
+        pl->self_rows = static_cast<__nv_bfloat16 *>(ptr);
+        if ((e = cudaMemset(ptr, 0, rows * c.d * 2)) != cudaSuccess) return e;
+        if ((e = cudaMalloc(&ptr, rows * 4)) != cudaSuccess) return e;
+        ctx->allocations.push_back(ptr), ctx->device_bytes += (int64_t)(rows * 4);
+        pl->iota = static_cast<int32_t *>(ptr);
+        k_iota<<<64, 256>>>(pl->iota, (int)rows);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
     if (c.d == 128)
         e = cudaFuncSetAttribute(k_att_tc<128, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttCfg<128, 128>::kSmem);
     else
@@ -495,6 +516,30 @@ cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
     else
         e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(kAttThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, p);
     count_launch();
+    return e;
+}
+
+cudaError_t launch_self_att_tc(const aif_ctx *ctx, int slot_index, int L, cudaStream_t st, const void **rows_out)
+{
+    const aif_config &c = ctx->cfg;
+    const AttPlan *pl = reinterpret_cast<const AttPlan *>(ctx->tc_att_plan);
+    ScoreLaunch sl{};
+    sl.slots = ctx->slots_dev, sl.reqs = nullptr, sl.n_req = 1;
+    sl.single = ReqDev{slot_index, L, 0, 0, 0};
+    sl.n_tiles = (L + kTcTile - 1) / kTcTile, sl.total = L;
+    sl.ids = pl->iota, sl.logits = nullptr, sl.status = ctx->status;
+    AttParams p{};
+    p.sl = sl, p.E = reinterpret_cast<const uint8_t *>(ctx->slots[(size_t)slot_index].dev.S), p.M = L, p.mini_batch = 0;
+    p.x_stride = c.d, p.X = pl->self_rows;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.d);
+    const int grid = sl.n_tiles >= 148 * 16 ? 148 : sl.n_tiles;
+    cudaError_t e;
+    if (c.d == 128)
+        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(kAttThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, p);
+    else
+        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(kAttThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, p);
+    count_launch();
+    *rows_out = pl->self_rows;
     return e;
 }
 
