@@ -273,8 +273,9 @@ __global__ void __launch_bounds__(kSimtThreads) k_score_simt(ModelDev md, ScoreL
             const float b0 = bias[j];
 #pragma unroll
             for (int c = 0; c < TM; ++c) acc[c] = b0;
-            for (int k = 0; k < in_w; ++k) {
-                const float w = to_f(W[(size_t)k * H + j]);
+            // weights in batches of 32 independent loads (the accumulation order over k stays sequential): after an L2
+            // flush every weight comes from HBM, and one load per iteration would expose that latency 32 times as often
+            auto step = [&](int k, float w) {
                 const float4 a = *reinterpret_cast<const float4 *>(in_act + k * TM);
                 const float4 b = *reinterpret_cast<const float4 *>(in_act + k * TM + 4);
                 acc[0] = fmaf(w, a.x, acc[0]);
@@ -285,7 +286,16 @@ __global__ void __launch_bounds__(kSimtThreads) k_score_simt(ModelDev md, ScoreL
                 acc[5] = fmaf(w, b.y, acc[5]);
                 acc[6] = fmaf(w, b.z, acc[6]);
                 acc[7] = fmaf(w, b.w, acc[7]);
+            };
+            int k = 0;
+            for (; k + 32 <= in_w; k += 32) {
+                float w[32];
+#pragma unroll
+                for (int u = 0; u < 32; ++u) w[u] = to_f(W[(size_t)(k + u) * H + j]);
+#pragma unroll
+                for (int u = 0; u < 32; ++u) step(k + u, w[u]);
             }
+            for (; k < in_w; ++k) step(k, to_f(W[(size_t)k * H + j]));
 #pragma unroll
             for (int c = 0; c < TM; ++c) out_act[j * TM + c] = fmaxf(acc[c], 0.f);
         }
