@@ -4,14 +4,15 @@
 //
 // Persistent kernel: one CTA per SM walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  224 threads:
 //   warps 0-3  per key block: read the score row from TMEM into registers, online softmax in fp32 (one thread per
-//              candidate row), write the probabilities as a bf16 A operand into shared memory; at the end of a tile
-//              normalise O and store the attention rows
+//              candidate row), write the probabilities back into the same TMEM columns as packed bf16 pairs (the A
+//              operand of P V is read from tensor memory, which keeps it off the shared-memory bandwidth the products
+//              are bound by); at the end of a tile normalise O and store the attention rows
 //   warp  4    allocates TMEM; one lane issues tcgen05.mma over the flat sequence of key blocks of all its tiles:
 //              scores = Q K^T (both K-major) one block ahead of O += P V, with V read from the very same shared-memory
 //              tile as K, as an MN-major B operand
 //   warp  5    one lane streams key/value blocks of S with TMA (3-D tensor map over the user-state arena)
 //   warp  6    gathers the item rows of the next tile (the queries) with cp.async while the current tile is processed
-//              (two query buffers where shared memory allows, d = 128)
+//              (two query buffers)
 // TMEM: two score buffers (so the softmax of block j overlaps Q K^T of block j+1) and the O accumulator.
 // The running maximum is only raised when a row's block maximum exceeds it by more than 8 (in the log2 domain);
 // then the warp rescales its 32 rows of O in TMEM.  Until then probabilities stay below 2^8, which fp32 sums and
@@ -40,14 +41,12 @@ template <int D, int BN>
 struct AttCfg {
     static constexpr int kQChunks = D / 64;             // 64-column (128-byte) chunks of a row
     static constexpr int kQBytes = kQChunks * 128 * 128;
-    static constexpr int kQBufs = D <= 128 ? 2 : 1;     // query buffers
-    static constexpr int kKvStages = 3;
+    static constexpr int kQBufs = 2;                    // query buffers
+    static constexpr int kKvStages = D <= 128 ? 5 : 3;
     static constexpr int kKvChunkBytes = BN * 128;      // one 64-column chunk of a key block
     static constexpr int kKvBytes = kQChunks * kKvChunkBytes;
-    static constexpr int kPChunks = BN / 64;
-    static constexpr int kPBytes = kPChunks * 128 * 128;
     static constexpr int kTmemO = 2 * BN;               // column of the O accumulator
-    static constexpr size_t kSmem = 1024 + kQBufs * kQBytes + kKvStages * kKvBytes + 2 * kPBytes + 512;
+    static constexpr size_t kSmem = 1024 + kQBufs * kQBytes + kKvStages * kKvBytes + 512;
 };
 
 // One tile of the launch as every role needs it.
@@ -77,8 +76,7 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
     unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
     unsigned char *smQ = base;
     unsigned char *smKV = smQ + kQB * C::kQBytes;
-    unsigned char *smP = smKV + kS * C::kKvBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smP + 2 * C::kPBytes);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smKV + kS * C::kKvBytes);
     uint64_t *kv_full = bars, *kv_empty = bars + kS;
     uint64_t *s_full = bars + 2 * kS, *p_full = s_full + 2, *pv_done = p_full + 2;
     uint64_t *q_full = pv_done + 2, *q_empty = q_full + 2, *o_final = q_empty + 2, *o_free = o_final + 1, *q_first = o_free + 1;
@@ -204,19 +202,14 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                         tmem_st_wait();
                     }
                 }
-                // the P buffer was last read by the P V product two blocks ago
-                if (gb >= 2 && !mbar_wait(smem_u32(pv_done + b), ((gb - 2) >> 1) & 1u, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-                // probabilities -> bf16 A operand in shared memory
-                unsigned char *Pb = smP + b * C::kPBytes;
+                // probabilities -> packed bf16 pairs over the first BN / 2 columns of the score buffer just read (P V of
+                // block gb - 2, the buffer's previous reader, precedes the Q K^T that refilled it in the MMA pipe)
                 float ls4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int c0 = 0; c0 < BN; c0 += 32) {
-                    uint32_t packed[16];
+                for (int c0 = 0; c0 < BN; c0 += 64) {
+                    uint32_t packed[32];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
+                    for (int i = 0; i < 32; ++i) {
                         float p0 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i]), k2, -m_used));
                         float p1 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i + 1]), k2, -m_used));
                         if (valid_cols != BN) {
@@ -227,15 +220,10 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                         const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                         packed[i] = *reinterpret_cast<const uint32_t *>(&h);
                     }
-                    unsigned char *chunk = Pb + (c0 >> 6) * 16384 + row * 128;
-                    const int slot0 = (c0 & 63) >> 3;     // first 16-byte slot of these 32 columns inside the 128-byte row
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4 *>(chunk + (((slot0 + q) ^ (row & 7)) << 4)) =
-                            make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                    tmem_st32(ts + (uint32_t)(c0 >> 1), packed);
                 }
+                tmem_st_wait();
                 l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-                fence_proxy_async();
                 tc_fence_before();
                 mbar_arrive(smem_u32(p_full + b));
             }
@@ -297,7 +285,6 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
             };
             // operand descriptors of buffer / stage 0; the others lie a fixed number of 16-byte units further
             const uint64_t qdesc0 = umma_desc_sw128(smem_u32(smQ)), kdesc0 = umma_desc_sw128(smem_u32(smKV));
-            const uint64_t pdesc0 = umma_desc_sw128(smem_u32(smP));
             const uint64_t vdesc0 = umma_desc_mn_sw128(smem_u32(smKV), C::kKvChunkBytes);
             Cursor cq{(int)blockIdx.x, 0, 0, 0, 0u}, cp{(int)blockIdx.x, 0, 0, 0, 0u};
             open_tile(cq);
@@ -344,13 +331,12 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                 tc_fence_after();
                 const int s = (int)(cp.gb % kS);
                 const uint32_t o_tmem = tmem_base + (uint32_t)C::kTmemO;
-                const uint64_t pd = pdesc0 + (uint64_t)((cp.gb & 1u) * (uint32_t)(C::kPBytes >> 4));
+                const uint32_t p_tmem = tmem_base + (uint32_t)((cp.gb & 1u) * BN);   // P: 8 columns per 16 keys
                 const uint64_t vd = vdesc0 + (uint64_t)(uint32_t)(s * (C::kKvBytes >> 4));
-                umma_bf16(o_tmem, pd, vd, idesc_pv, cp.j > 0 ? 1u : 0u);
 #pragma unroll
-                for (int kk = 1; kk < BN / 16; ++kk)   // V: 16 keys further = 16 rows x 128 bytes
-                    umma_bf16_acc(o_tmem, pd + (uint64_t)((kk >> 2) * (16384 >> 4) + 2 * (kk & 3)), vd + (uint64_t)(kk * (2048 >> 4)),
-                                  idesc_pv);
+                for (int kk = 0; kk < BN / 16; ++kk)   // V: 16 keys further = 16 rows x 128 bytes
+                    umma_bf16_ts(o_tmem, p_tmem + (uint32_t)(kk * 8), vd + (uint64_t)(kk * (2048 >> 4)), idesc_pv,
+                                 (cp.j > 0 || kk > 0) ? 1u : 0u);
                 umma_commit(smem_u32(pv_done + (cp.gb & 1u)));
                 umma_commit(smem_u32(kv_empty + s));
                 if (cp.j == cp.nb - 1) umma_commit(smem_u32(o_final));
