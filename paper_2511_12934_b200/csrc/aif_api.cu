@@ -451,7 +451,7 @@ int aif_score(aif_ctx *ctx, const aif_user_state *state, const int32_t *cand_ids
     sl.slots = ctx->slots_dev, sl.reqs = nullptr, sl.n_req = 1;
     sl.single = ReqDev{state->index, n, 0, 0, 0};
     sl.n_tiles = tiles_for(ctx, n);
-    sl.total = n;
+    sl.total = n, sl.max_L = hs.L;
     sl.ids = cand_ids, sl.logits = logits, sl.status = ctx->status;
     return run_score(ctx, sl, n, st);
 }
@@ -479,16 +479,17 @@ int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *st
     const int slot = ring.next;
     ring.next = (ring.next + 1) % PinnedRing::kSlots;
     if (ring.used[slot]) AIF_CUDA(cudaEventSynchronize(ring.ev[slot]));
-    int tiles = 0;
+    int tiles = 0, max_L = 0;
     for (int r = 0; r < n_req; ++r) {
         const int n = (int)(offsets[r + 1] - offsets[r]);
+        if (ctx->slots[(size_t)states[r]->index].L > max_L) max_L = ctx->slots[(size_t)states[r]->index].L;
         ring.host[slot][r] = ReqDev{states[r]->index, n, offsets[r], tiles, 0};
         tiles += tiles_for(ctx, n);
         AIF_CUDA(cudaStreamWaitEvent(st, ctx->slots[(size_t)states[r]->index].ev, 0));
     }
     AIF_CUDA(cudaMemcpyAsync(ring.dev[slot], ring.host[slot], sizeof(ReqDev) * (size_t)n_req, cudaMemcpyHostToDevice, st));
     ScoreLaunch sl{};
-    sl.slots = ctx->slots_dev, sl.reqs = ring.dev[slot], sl.n_req = n_req, sl.n_tiles = tiles, sl.total = total;
+    sl.slots = ctx->slots_dev, sl.reqs = ring.dev[slot], sl.n_req = n_req, sl.n_tiles = tiles, sl.total = total, sl.max_L = max_L;
     sl.ids = cand_ids, sl.logits = logits, sl.status = ctx->status;
     int rc = run_score(ctx, sl, total, st);
     if (rc != AIF_OK) return rc;

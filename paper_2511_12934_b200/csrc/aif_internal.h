@@ -62,6 +62,7 @@ struct ScoreLaunch {
     int32_t n_req;
     int32_t n_tiles;
     int64_t total;          // candidates of the launch
+    int32_t max_L;          // longest behaviour sequence among the launch's requests (host-side hint)
     const int32_t *ids;
     float *logits;
     uint32_t *status;

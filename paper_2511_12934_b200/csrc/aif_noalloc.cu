@@ -88,7 +88,7 @@ extern "C" int aif_score_noalloc(aif_ctx *ctx, const aif_user_state *state, cons
             sl.slots = ctx->slots_dev, sl.reqs = nullptr, sl.n_req = 1;
             sl.single = ReqDev{state->index, n, 0, 0, 0};
             sl.n_tiles = tc_tiles_for(ctx, n);
-            sl.total = n;
+            sl.total = n, sl.max_L = hs.L;
             sl.ids = cand_ids, sl.logits = logits, sl.status = ctx->status;
             e = launch_score_tc_scratch(ctx, sl, st, sc);
         }
