@@ -163,11 +163,11 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                 if (valid_cols == BN) {
 #pragma unroll
-                    for (int i = 0; i < BN; i += 4) {
-                        mx4[0] = fmaxf(mx4[0], __uint_as_float(sc[i]));
-                        mx4[1] = fmaxf(mx4[1], __uint_as_float(sc[i + 1]));
-                        mx4[2] = fmaxf(mx4[2], __uint_as_float(sc[i + 2]));
-                        mx4[3] = fmaxf(mx4[3], __uint_as_float(sc[i + 3]));
+                    for (int i = 0; i < BN; i += 8) {   // three-input maxima: two scores per instruction
+                        mx4[0] = fmax3(mx4[0], __uint_as_float(sc[i]), __uint_as_float(sc[i + 1]));
+                        mx4[1] = fmax3(mx4[1], __uint_as_float(sc[i + 2]), __uint_as_float(sc[i + 3]));
+                        mx4[2] = fmax3(mx4[2], __uint_as_float(sc[i + 4]), __uint_as_float(sc[i + 5]));
+                        mx4[3] = fmax3(mx4[3], __uint_as_float(sc[i + 6]), __uint_as_float(sc[i + 7]));
                     }
                 } else {
 #pragma unroll
@@ -509,11 +509,11 @@ __global__ void __launch_bounds__(kAtt2Threads, 1) k_att_tc_long(const __grid_co
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
             if (valid_cols == BN) {
 #pragma unroll
-                for (int i = 0; i < BN; i += 4) {
-                    mx4[0] = fmaxf(mx4[0], __uint_as_float(sc[i]));
-                    mx4[1] = fmaxf(mx4[1], __uint_as_float(sc[i + 1]));
-                    mx4[2] = fmaxf(mx4[2], __uint_as_float(sc[i + 2]));
-                    mx4[3] = fmaxf(mx4[3], __uint_as_float(sc[i + 3]));
+                for (int i = 0; i < BN; i += 8) {   // three-input maxima: two scores per instruction
+                    mx4[0] = fmax3(mx4[0], __uint_as_float(sc[i]), __uint_as_float(sc[i + 1]));
+                    mx4[1] = fmax3(mx4[1], __uint_as_float(sc[i + 2]), __uint_as_float(sc[i + 3]));
+                    mx4[2] = fmax3(mx4[2], __uint_as_float(sc[i + 4]), __uint_as_float(sc[i + 5]));
+                    mx4[3] = fmax3(mx4[3], __uint_as_float(sc[i + 6]), __uint_as_float(sc[i + 7]));
                 }
             } else {
 #pragma unroll
