@@ -188,6 +188,12 @@ void tc_att_destroy(aif_ctx *ctx);
 // *rows_out: [L x d] bf16 in scratch of the attention plan, valid until the next call
 cudaError_t launch_self_att_tc(const aif_ctx *ctx, int slot_index, int L, cudaStream_t st, const void **rows_out);
 cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, void *X, int x_stride);
+// whole scoring pass of a tile in one CTA (aif_tc_fused.cu); the tensor maps it shares with the other kernels
+bool tc_fused_supported(const aif_config &cfg);
+cudaError_t tc_fused_prepare(aif_ctx *ctx);
+cudaError_t launch_request_fused(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st);
+const void *tc_weight_tmap(const aif_ctx *ctx, int k);   // CUtensorMap over the packed weights of hidden layer k
+const void *tc_att_tmap(const aif_ctx *ctx);             // CUtensorMap over the S regions of the user-state arena
 cudaError_t tc_prepare_weights(aif_ctx *ctx, const aif_weights *w, cudaStream_t st);
 cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t total_candidates, cudaStream_t st);
 // The same kernel chain with its intermediate activations in caller-chosen memory.

@@ -29,6 +29,7 @@ namespace {
 constexpr int kABytes = kTcTile * 128;    // one A chunk of one tile: 128 rows x 64 bf16
 constexpr int kBBytes = 256 * 128;        // one B chunk: up to 256 weight rows x 64 bf16
 constexpr int kMaxChunks = 64;
+constexpr int kFusedMaxTiles = 148;
 
 enum { SRC_ITEM = 0, SRC_DENSE = 1, SRC_CROSS = 2 };
 enum { EPI_STORE = 0, EPI_DOT = 1 };
@@ -752,8 +753,11 @@ cudaError_t tc_prepare_context(aif_ctx *ctx)
     }
     pl->maps_ready = true;
     if (tc_att_supported(c) && (e = tc_att_prepare(ctx)) != cudaSuccess) return e;
+    if (tc_fused_supported(c) && (e = tc_fused_prepare(ctx)) != cudaSuccess) return e;
     return cudaSuccess;
 }
+
+const void *tc_weight_tmap(const aif_ctx *ctx, int k) { return &plan_of(ctx)->tmap[k]; }
 
 void tc_destroy_context(aif_ctx *ctx)
 {
@@ -829,6 +833,12 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
     TcPlan *pl = plan_of(ctx);
     const ModelDev md = make_model(ctx);
     timing_begin(ctx, st);
+    // a launch that fits the machine in one round of tiles: the whole pass in one kernel, one CTA per tile
+    if (sl.n_tiles <= kFusedMaxTiles && sl.max_L <= 256 && tc_fused_supported(c)) {
+        cudaError_t e = launch_request_fused(ctx, sl, st);
+        timing_mark(ctx, "score_fused", st);
+        return e;
+    }
     if (c.blocks & AIF_BLK_CROSS) {
         const int64_t n = sl.total * c.F;
         const int grid = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);

@@ -764,6 +764,8 @@ cudaError_t tc_att_prepare(aif_ctx *ctx)
     return e;
 }
 
+const void *tc_att_tmap(const aif_ctx *ctx) { return &reinterpret_cast<const AttPlan *>(ctx->tc_att_plan)->tmap; }
+
 void tc_att_destroy(aif_ctx *ctx)
 {
     delete reinterpret_cast<AttPlan *>(ctx->tc_att_plan);

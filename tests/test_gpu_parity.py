@@ -248,6 +248,32 @@ def test_sharp_softmax_exercises_the_running_max_rescaling():
     srv.close()
 
 
+@pytest.mark.parametrize("L", [1, 77, 128, 129, 200, 256, 257])
+def test_single_launch_scoring_at_the_sequence_lengths_around_its_key_blocks(L):
+    """Launches of at most one tile per SM with sequences of at most 256 items run the whole pass in one kernel (one or
+    two key blocks of 128); L = 257 takes the kernel-per-layer path on the same inputs.  Ragged last tiles, a launch of
+    several requests, ids outside the table and a zero-length tail of the id array are included."""
+    wl = helpers.MINI["c2"].with_(name=f"fused_L{L}", R=2, N=333, L=L, mini_batch=0)
+    weights, table, srv, oracle = _setup(wl)
+    sampler = synth.IdSampler(wl)
+    states, id_lists, wants = [], [], []
+    for r in range(wl.R):
+        rq = synth.make_request(wl, r)
+        ids = sampler.request_ids(r).copy()
+        if r == 1:
+            ids[5], ids[200] = -3, table["E"].shape[0]
+        st = srv.precompute(7 + r, srv.upload_request(rq, B.USER_PROJECTED))
+        want = oracle.score(table, helpers.projected_request(wl, rq), ids)
+        _check_logits(srv.score_ids(st, ids), want, TOL["bf16"])
+        states.append(st), id_lists.append(ids), wants.append(want)
+    assert srv.ctx.poll_status() == B.STATUS_BAD_ID
+    for o, w in zip(srv.score_many(states, id_lists), wants):
+        _check_logits(o, w, TOL["bf16"])
+    assert srv.ctx.poll_status() == B.STATUS_BAD_ID
+    _check_logits(srv.score_ids(states[0], id_lists[0][:1]), wants[0][:1], TOL["bf16"])
+    srv.close()
+
+
 @pytest.mark.parametrize("name", ["c3", "c4", "c5", "c5b"])
 def test_full_size_batches_on_sampled_candidates(name):
     """The multi-request shapes at their full sizes, scored in one aif_score_batch call exactly as the benchmark
