@@ -224,7 +224,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     TRY(dev_alloc(ctx, (void **)&ctx->b_b, (size_t)c.d * 4, true));
 
     // user-state arena: fixed-size slots in one allocation
-    struct Off { size_t u, u32, S, T, V, sig, pu, smallB, prof, partial, ppart, end; } o{};
+    struct Off { size_t u, u32, S, T, V, sig, pu, pu_hl, prof, partial, ppart, end; } o{};
     size_t p = 0;
     auto take = [&](size_t bytes) { size_t at = p; p += align_up(bytes ? bytes : 16, 256); return at; };
     o.u = take((size_t)c.d * el);
@@ -234,7 +234,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     o.V = take((c.blocks & AIF_BLK_BEA) ? (size_t)c.n_bridge * c.d * el : 0);
     o.sig = take((c.blocks & (AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER)) ? (size_t)c.L_max * c.lsh_bits / 8 : 0);
     o.pu = take((size_t)c.hidden[0] * 4);
-    o.smallB = take((size_t)c.hidden[0] * 16 * 2);
+    o.pu_hl = take((size_t)c.hidden[0] * 2 * 2);
     o.prof = take((size_t)c.d * 4);
     o.partial = take((size_t)kUserPartials * c.d * 4);
     o.ppart = take((size_t)kProfParts * (c.d + 2) * 4);
@@ -250,7 +250,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
         HostSlot &hs = ctx->slots[(size_t)i];
         hs.dev.u = base + o.u, hs.dev.u32 = (const float *)(base + o.u32), hs.dev.S = base + o.S;
         hs.dev.T = base + o.T, hs.dev.V = base + o.V, hs.dev.sigS = (const uint8_t *)(base + o.sig);
-        hs.dev.p_u = (const float *)(base + o.pu), hs.dev.smallB = base + o.smallB, hs.dev.L = 0;
+        hs.dev.p_u = (const float *)(base + o.pu), hs.dev.pu_hl = base + o.pu_hl, hs.dev.L = 0;
         hs.prof_hat = (float *)(base + o.prof), hs.partial = (float *)(base + o.partial), hs.ppart = (float *)(base + o.ppart);
         cudaError_t e = cudaEventCreateWithFlags(&hs.ev, cudaEventDisableTiming);
         if (e != cudaSuccess) {
@@ -344,6 +344,7 @@ int aif_load_weights(aif_ctx *ctx, const aif_weights *w, aif_stream stream)
         AIF_CUDA(cudaMemcpyAsync(ctx->b_b, w->b_b, (size_t)c.d * 4, cudaMemcpyDeviceToDevice, st));
     }
     if (ctx->tensor_path) AIF_CUDA(tc_prepare_weights(ctx, w, st));
+    if (ctx->tensor_path && ctx->tc_fused_plan) AIF_CUDA(tc_fused_prepare_weights(ctx, st));
     ctx->weights_loaded = true;
     ctx->model_version += 1;
     ctx->stats.model_version = ctx->model_version;
@@ -393,6 +394,7 @@ int aif_user_precompute(aif_ctx *ctx, uint64_t request_key, const aif_user_input
     cudaStream_t st = as_stream(side_stream);
     AIF_CUDA(launch_user_network(ctx, hs, idx, in, L, st));
     AIF_CUDA(cudaEventRecord(hs.ev, st));
+    hs.ev_seen_done = false;
     hs.in_use = true, hs.ready = true, hs.L = L, hs.key = request_key, hs.model_version = ctx->model_version;
     hs.dev.L = L;
     ctx->stats.precompute_calls += 1;
@@ -435,6 +437,22 @@ int aif_user_state_export(aif_ctx *ctx, const aif_user_state *state, float *u_ou
     return AIF_OK;
 }
 
+// Orders `st` behind the user-side call that filled the slot.  Once that call is known to have finished, no wait is
+// enqueued any more: a wait between two scoring calls of a stream costs device time and keeps the second call's
+// set-up from overlapping the first call's tail.
+static cudaError_t wait_user_ready(const HostSlot &hs, cudaStream_t st)
+{
+    if (hs.ev_seen_done) return cudaSuccess;
+    const cudaError_t q = cudaEventQuery(hs.ev);
+    if (q == cudaSuccess) {
+        hs.ev_seen_done = true;
+        return cudaSuccess;
+    }
+    if (q != cudaErrorNotReady) return q;
+    (void)cudaGetLastError();   // "not ready" is an answer, not a failure: keep it out of later launch checks
+    return cudaStreamWaitEvent(st, hs.ev, 0);
+}
+
 int aif_score(aif_ctx *ctx, const aif_user_state *state, const int32_t *cand_ids, int32_t n, float *logits, aif_stream stream)
 {
     int rc = state_check(ctx, state);
@@ -446,7 +464,7 @@ int aif_score(aif_ctx *ctx, const aif_user_state *state, const int32_t *cand_ids
     DeviceGuard g(ctx->device);
     cudaStream_t st = as_stream(stream);
     const HostSlot &hs = ctx->slots[(size_t)state->index];
-    AIF_CUDA(cudaStreamWaitEvent(st, hs.ev, 0));
+    AIF_CUDA(wait_user_ready(hs, st));
     ScoreLaunch sl{};
     sl.slots = ctx->slots_dev, sl.reqs = nullptr, sl.n_req = 1;
     sl.single = ReqDev{state->index, n, 0, 0, 0};
@@ -485,7 +503,7 @@ int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *st
         if (ctx->slots[(size_t)states[r]->index].L > max_L) max_L = ctx->slots[(size_t)states[r]->index].L;
         ring.host[slot][r] = ReqDev{states[r]->index, n, offsets[r], tiles, 0};
         tiles += tiles_for(ctx, n);
-        AIF_CUDA(cudaStreamWaitEvent(st, ctx->slots[(size_t)states[r]->index].ev, 0));
+        AIF_CUDA(wait_user_ready(ctx->slots[(size_t)states[r]->index], st));
     }
     AIF_CUDA(cudaMemcpyAsync(ring.dev[slot], ring.host[slot], sizeof(ReqDev) * (size_t)n_req, cudaMemcpyHostToDevice, st));
     ScoreLaunch sl{};

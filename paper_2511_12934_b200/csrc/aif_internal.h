@@ -26,7 +26,7 @@ struct SlotDev {
     const void *V;          // [n_bridge x d] storage type
     const uint8_t *sigS;    // [L x lsh_bits/8]
     const float *p_u;       // [H1] fp32: W1[:, user columns] u + b1
-    const void *smallB;     // [H1 x 16] bf16: per-request B operand of the narrow feature chunk (tensor path)
+    const void *pu_hl;      // [2][H1] bf16: p_u split into high parts and remainders (bias operand of the tensor cores)
     int32_t L;
     int32_t pad_;
 };
@@ -75,6 +75,7 @@ struct HostSlot {
     uint64_t key = 0;
     uint64_t model_version = 0;
     cudaEvent_t ev = nullptr;
+    mutable bool ev_seen_done = false;   // the user-side call that recorded `ev` is known to have completed
     SlotDev dev{};
     // scratch for the user-side network
     float *prof_hat = nullptr;   // [d]
@@ -147,6 +148,7 @@ struct aif_ctx {
     float *logits_stage = nullptr;
     void *tc_plan = nullptr;          // tensor-core path: packed weights, tensor maps, activation scratch
     void *tc_att_plan = nullptr;      // tensor-core attention: tensor map over the arena's S regions
+    void *tc_fused_plan = nullptr;    // single-launch scoring: the second layer's bias split into two bf16 rows
     aif::PinnedRing ring;
 
     aif_stats stats{};
@@ -191,6 +193,7 @@ cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
 // whole scoring pass of a tile in one CTA (aif_tc_fused.cu); the tensor maps it shares with the other kernels
 bool tc_fused_supported(const aif_config &cfg);
 cudaError_t tc_fused_prepare(aif_ctx *ctx);
+cudaError_t tc_fused_prepare_weights(aif_ctx *ctx, cudaStream_t st);
 cudaError_t launch_request_fused(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st);
 const void *tc_weight_tmap(const aif_ctx *ctx, int k);   // CUtensorMap over the packed weights of hidden layer k
 const void *tc_att_tmap(const aif_ctx *ctx);             // CUtensorMap over the S regions of the user-state arena

@@ -459,7 +459,7 @@ __global__ void __launch_bounds__(256) k_user_finish(int raw, const T *__restric
                                                      const T *__restrict__ u_in, T *__restrict__ u_out,
                                                      float *__restrict__ u32, const T *__restrict__ W1t,
                                                      const float *__restrict__ b1, int H1, float *__restrict__ p_u,
-                                                     const T *__restrict__ Wb_t, const float *__restrict__ b_b,
+                                                     __nv_bfloat16 *__restrict__ pu_hl, const T *__restrict__ Wb_t, const float *__restrict__ b_b,
                                                      const float *__restrict__ ppart)
 {
     __shared__ float q[256], uprof[256], us[256];
@@ -511,6 +511,10 @@ __global__ void __launch_bounds__(256) k_user_finish(int raw, const T *__restric
         float acc = b1[j];
         for (int k = 0; k < d; ++k) acc = fmaf(us[k], to_f(W1t[(size_t)k * H1 + j]), acc);
         p_u[j] = acc;
+        // the same partial as two bf16 values (high part, remainder): the form in which the tensor cores add it
+        const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
+        pu_hl[j] = hi;
+        pu_hl[H1 + j] = __float2bfloat16_rn(acc - __bfloat162float(hi));
     }
 }
 
@@ -566,7 +570,7 @@ static cudaError_t user_network_typed(const aif_ctx *ctx, HostSlot &hs, int slot
     }
     k_user_finish<T><<<1, 256, 0, st>>>(raw ? 1 : 0, S, L, d, hs.prof_hat, hs.partial, kUserPartials,
                                         (const T *)in->profile, (T *)hs.dev.u, (float *)hs.dev.u32, (const T *)ctx->Wt[0],
-                                        ctx->b[0], H1, (float *)hs.dev.p_u, (const T *)ctx->Wb_t, ctx->b_b, hs.ppart);
+                                        ctx->b[0], H1, (float *)hs.dev.p_u, (__nv_bfloat16 *)hs.dev.pu_hl, (const T *)ctx->Wb_t, ctx->b_b, hs.ppart);
     count_launch();
     return cudaGetLastError();
 }

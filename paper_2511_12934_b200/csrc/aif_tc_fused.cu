@@ -22,8 +22,8 @@
 //               K-major chunks; buckets are hashed one chunk ahead of their use
 //   warp 13     one lane streams key/value blocks, then first- and second-layer weights with TMA
 //
-// Tensor memory (512 columns): attention uses [0, 256) for the scores of up to two key blocks (probabilities packed
-// over the first half of each block's own columns) and [256, 384) for O.  Layer 1 then fills two 256-column
+// Tensor memory (512 columns): attention uses [0, 256) for the scores of up to two key blocks, [256, 384) for O and
+// [384, 512) for the probabilities (packed bf16, 64 columns per key block).  Layer 1 then fills two 256-column
 // accumulators [0, 256) and [256, 512); its activations are packed in place into [0, 128) and [256, 384); layer 2
 // accumulates its two halves into the freed columns [128, 256) and [384, 512).
 // Shared memory: item tile 32 KB | key/value blocks 64 KB, later the attention chunks and two more stages of the
@@ -50,7 +50,7 @@ constexpr int kH1 = 512;
 
 enum {
     BAR_E_FULL = 0, BAR_KV_FULL, BAR_S_FULL = BAR_KV_FULL + 2, BAR_P_FULL, BAR_O_FINAL, BAR_ATT_FULL, BAR_E_FREE, BAR_ACC1_FULL,
-    BAR_H1_FULL, BAR_ACC2_FULL, BAR_FULL_A, BAR_EMPTY_A = BAR_FULL_A + kAStages, BAR_FULL_B = BAR_EMPTY_A + kAStages,
+    BAR_H1_FULL, BAR_ACC2_FULL, BAR_BIAS_FULL, BAR_FULL_A, BAR_EMPTY_A = BAR_FULL_A + kAStages, BAR_FULL_B = BAR_EMPTY_A + kAStages,
     BAR_EMPTY_B = BAR_FULL_B + kBStages, BAR_COUNT = BAR_EMPTY_B + kBStages
 };
 static_assert(BAR_COUNT * 8 + 16 + 2 * 128 * 4 <= 2048, "misc area");
@@ -63,7 +63,7 @@ struct FusedParams {
     int32_t B, dc, b_mask, bucket_mode, n_cross;
     int32_t H2, emit_sigmoid;
     float scale_log2;       // log2(e) / sqrt(d)
-    const float *b2;
+    const __nv_bfloat16 *b2_hl;   // [2][H2]: second-layer bias, high parts then remainders
     const __nv_bfloat16 *w_out;
     const float *b_out;
 };
@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
         mbar_init(bar(BAR_ACC1_FULL), 1);
         mbar_init(bar(BAR_H1_FULL), 256);
         mbar_init(bar(BAR_ACC2_FULL), 1);
+        mbar_init(bar(BAR_BIAS_FULL), 256);
         for (int s = 0; s < kAStages; ++s) {
             mbar_init(bar(BAR_FULL_A + s), 128);
             mbar_init(bar(BAR_EMPTY_A + s), 1);
@@ -106,6 +107,18 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
         }
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // The gather threads fetch their candidate ids while barriers and tensor memory are being set up: the ids head the
+    // longest chain of dependent memory accesses of the kernel (ids -> item rows -> scores).
+    int id[8];
+    if (warp >= kFProdWarp0 && warp < kFBWarp) {
+        grid_dep_wait();
+        const ReqDev rq0 = find_request(p.sl, blockIdx.x);
+        int start0, cnt0;
+        tile_range(blockIdx.x - rq0.tile_begin, rq0.n, kTcTile, p.mini_batch, start0, cnt0);
+        const int r0 = (tid - kFProdWarp0 * 32) >> 3;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) id[i] = r0 + 16 * i < cnt0 ? p.sl.ids[rq0.off + start0 + r0 + 16 * i] : -1;
     }
     if (warp == kFMmaWarp) tmem_alloc(smem_u32(tmem_slot), 512);
     tc_fence_before();
@@ -136,38 +149,23 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
             const bool got = ok && mbar_wait(bar(b), 0u, abort_flag);
             ok = __all_sync(0xffffffffu, got);
         };
+        const float b_out = p.b_out[0];
         bool good = false;
         if (row < cnt) {
             const int id = p.sl.ids[pos0 + row];
             good = id >= 0 && (int64_t)id < p.M;
         }
         // ---- attention: scores of key block g -> probabilities
+        // Softmax is invariant to the offset subtracted in the exponent, and bf16 keeps its relative precision over the
+        // whole fp32 exponent range.  The first attempt therefore subtracts nothing, p = 2^(s k2), and saves the pass
+        // over the scores that finds the row maxima; a row sum outside [2^-80, 2^80] (scores far from zero: overflow,
+        // or every term flushed to zero) makes the whole CTA repeat the step with the exact row maxima.  The
+        // probabilities go to columns of their own, so the scores are still there for the repeat.
         const bool act = g < nb;
         const int valid_cols = L - g * 128 < 128 ? L - g * 128 : 128;
-        float mx = -INFINITY;
-        if (act) {
-            wait(BAR_S_FULL);
-            tc_fence_after();
-            if (ok) {
-#pragma unroll 1
-                for (int c0 = 0; c0 < 128; c0 += 32) {
-                    uint32_t r[32];
-                    tmem_ld32(lane_base + (uint32_t)(g * 128 + c0), r);
-                    tmem_ld_wait();
-                    float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (c0 + i < valid_cols) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(r[i]));
-                    mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
-                }
-            }
-        }
-        xs[g * 128 + row] = mx;
-        named_bar_sync(1, 256);
-        const float mt = fmaxf(mx, xs[(g ^ 1) * 128 + row]) * k2;   // an inactive group has published -inf
-        named_bar_sync(1, 256);                                    // both maxima are read: xs may now take the sums
-        float lsum = 0.f;
-        if (act && ok) {
+        const uint32_t p_col = 384u + (uint32_t)(g * 64);
+        auto probabilities = [&](float mt) {   // P = 2^(s k2 - mt) as packed bf16; returns the row sum over this block
+            float lsum = 0.f;
 #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
                 uint32_t sc[64];
@@ -176,27 +174,58 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
                 tmem_ld_wait();
                 uint32_t packed[32];
                 float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+                const int left = valid_cols - 64 * h;   // valid columns among these 64
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
                     float p0 = fast_exp2(fmaf(__uint_as_float(sc[2 * i]), k2, -mt));
                     float p1 = fast_exp2(fmaf(__uint_as_float(sc[2 * i + 1]), k2, -mt));
-                    if (64 * h + 2 * i >= valid_cols) p0 = 0.f;
-                    if (64 * h + 2 * i + 1 >= valid_cols) p1 = 0.f;
+                    if (2 * i >= left) p0 = 0.f;
+                    if (2 * i + 1 >= left) p1 = 0.f;
                     ls4[i & 3] += p0 + p1;
                     const __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
                     packed[i] = *reinterpret_cast<const uint32_t *>(&hh);
                 }
-                // over columns this thread has already read: [64 h, 64 h + 64) of the block -> [32 h, 32 h + 32)
-                tmem_st32(lane_base + (uint32_t)(g * 128 + 32 * h), packed);
+                tmem_st32(lane_base + p_col + (uint32_t)(32 * h), packed);
                 lsum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
             }
             tmem_st_wait();
+            return lsum;
+        };
+        float lsum = 0.f;
+        if (act) {
+            wait(BAR_S_FULL);
+            tc_fence_after();
+            if (ok) lsum = probabilities(0.f);
         }
         xs[g * 128 + row] = lsum;
+        const bool off_range = act && ok && !(lsum > 0x1p-80f && lsum < 0x1p80f);
+        float l_other;
+        if (named_bar_or(1, 256, off_range)) {
+            // exact form: row maxima over both key blocks first
+            float mx = -INFINITY;
+            if (act && ok) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < 128; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld32(lane_base + (uint32_t)(g * 128 + c0), r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (c0 + i < valid_cols) mx = fmaxf(mx, __uint_as_float(r[i]));
+                }
+            }
+            xs[g * 128 + row] = mx;
+            named_bar_sync(1, 256);
+            const float mt = fmaxf(mx, xs[(g ^ 1) * 128 + row]) * k2;   // an inactive group has published -inf
+            named_bar_sync(1, 256);                                    // both maxima are read: xs may now take the sums
+            lsum = act && ok ? probabilities(mt) : 0.f;
+            xs[g * 128 + row] = lsum;
+            named_bar_sync(1, 256);
+        }
+        l_other = xs[(g ^ 1) * 128 + row];
         tc_fence_before();
         mbar_arrive(bar(BAR_P_FULL));
-        named_bar_sync(1, 256);
-        const float l_all = lsum + xs[(g ^ 1) * 128 + row];
+        const float l_all = lsum + l_other;
         // ---- O -> attention chunk g of the first layer's input (64 columns, 128B-swizzled K-major)
         wait(BAR_O_FINAL);
         tc_fence_after();
@@ -225,73 +254,109 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
         fence_proxy_async();   // the MMA reads these chunks through the async proxy
         tc_fence_before();
         mbar_arrive(bar(BAR_ATT_FULL));
-        // ---- biases into the item tile's memory once layer 1 has consumed it
+        // ---- bias operands into the item tile's memory once layer 1 has consumed it.  The biases are added by the
+        // tensor cores: one more K step whose A operand is a tile of ones in columns 0 and 1 and whose B operand holds,
+        // per output unit, the bias split into two bf16 values (high part, remainder) in K rows 0 and 1 (fp32
+        // accumulation restores the bias to about 2^-17 of its magnitude).  Reading biases from shared memory in the
+        // epilogue would cost one shared-memory cycle per element and warp, more than everything else there.
+        // Layout: MN-major 128B-swizzled groups of 64 units x 16 K rows (2 KB each): layer 1 at smE, layer 2 behind it.
         wait(BAR_E_FREE);
-        float *bias1 = reinterpret_cast<float *>(smE), *b2_s = bias1 + kH1, *wout_s = b2_s + 256, *dot_s = wout_s + 256;
+        __nv_bfloat16 *wout_s = reinterpret_cast<__nv_bfloat16 *>(smE + 24576);
+        float *dot_s = reinterpret_cast<float *>(smE + 25600);
         {
             const int t = warp * 32 + lane;
-            bias1[t] = slot->p_u[t];
-            bias1[t + 256] = slot->p_u[t + 256];
-            if (t < p.H2) {
-                b2_s[t] = p.b2[t];
-                wout_s[t] = __bfloat162float(p.w_out[t]);
+            const uint4 *hl1 = reinterpret_cast<const uint4 *>(slot->pu_hl);   // [2][512] bf16
+            const uint4 *hl2 = reinterpret_cast<const uint4 *>(p.b2_hl);       // [2][H2] bf16
+            const int n1 = kH1 / 64 * 128, n2 = p.H2 / 64 * 128;              // 16-byte slots of the two operands
+            for (int sidx = t; sidx < n1 + n2; sidx += 256) {
+                const bool second = sidx >= n1;
+                const int q = second ? sidx - n1 : sidx;
+                const int grp = q >> 7, k = (q >> 3) & 15, j = (q & 7) ^ (k & 7);
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (k < 2) v = second ? hl2[(k * p.H2 + grp * 64 + j * 8) >> 3] : hl1[(k * kH1 + grp * 64 + j * 8) >> 3];
+                *reinterpret_cast<uint4 *>(smE + (second ? 16384 : 0) + q * 16) = v;
             }
+            if (t < p.H2 / 8) reinterpret_cast<uint4 *>(wout_s)[t] = reinterpret_cast<const uint4 *>(p.w_out)[t];
         }
+        fence_proxy_async();
+        mbar_arrive(bar(BAR_BIAS_FULL));
         named_bar_sync(1, 256);
-        // ---- layer-1 epilogue: slice g, 64 accumulator columns -> 32 columns of packed bf16, in place
+        // ---- layer-1 epilogue: slice g, ReLU, 32 accumulator columns -> 16 columns of packed bf16, in place (the target
+        // columns [16 c, 16 c + 16) lie in chunks already read); the load of the next chunk is in flight meanwhile
         wait(BAR_ACC1_FULL);
         tc_fence_after();
         if (ok) {
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[64];
-                tmem_ld32(lane_base + (uint32_t)(g * 256 + 64 * c), *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-                tmem_ld32(lane_base + (uint32_t)(g * 256 + 64 * c + 32), *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
-                tmem_ld_wait();
-                const float4 *b4 = reinterpret_cast<const float4 *>(bias1 + g * 256 + 64 * c);
-                uint32_t packed[32];
+            uint32_t ra[32], rb[32];
+            const uint32_t col0 = lane_base + (uint32_t)(g * 256);
+            auto finish = [&](const uint32_t (&r)[32], int c) {
+                uint32_t packed[16];
 #pragma unroll
                 for (int q = 0; q < 16; ++q) {
-                    const float4 bb = b4[q];
-                    const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q]) + bb.x, 0.f),
-                                                                    fmaxf(__uint_as_float(r[4 * q + 1]) + bb.y, 0.f));
-                    const __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q + 2]) + bb.z, 0.f),
-                                                                    fmaxf(__uint_as_float(r[4 * q + 3]) + bb.w, 0.f));
-                    packed[2 * q] = *reinterpret_cast<const uint32_t *>(&h0);
-                    packed[2 * q + 1] = *reinterpret_cast<const uint32_t *>(&h1);
+                    const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[2 * q]), 0.f), fmaxf(__uint_as_float(r[2 * q + 1]), 0.f));
+                    packed[q] = *reinterpret_cast<const uint32_t *>(&h0);
                 }
-                tmem_st32(lane_base + (uint32_t)(g * 256 + 32 * c), packed);
+                tmem_st16(col0 + (uint32_t)(16 * c), packed);
+            };
+            tmem_ld32(col0, ra);
+#pragma unroll 1
+            for (int c = 0; c < 8; c += 2) {
+                tmem_ld_wait();
+                tmem_ld32(col0 + (uint32_t)(32 * (c + 1)), rb);
+                finish(ra, c);
+                tmem_ld_wait();
+                if (c + 2 < 8) tmem_ld32(col0 + (uint32_t)(32 * (c + 2)), ra);
+                finish(rb, c + 1);
             }
             tmem_st_wait();
         }
         tc_fence_before();
         mbar_arrive(bar(BAR_H1_FULL));
-        // ---- layer-2 epilogue: half g of the units, reduced against w_out
+        // ---- layer-2 epilogue: half g of the units, ReLU, reduced against w_out
         wait(BAR_ACC2_FULL);
         tc_fence_after();
         float dot = 0.f;
         if (ok) {
             const int hn = p.H2 >> 1;
-            for (int c0 = 0; c0 < hn; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(lane_base + (uint32_t)((g ? 384 : 128) + c0), r);
-                tmem_ld_wait();
-                const float4 *b4 = reinterpret_cast<const float4 *>(b2_s + g * hn + c0);
-                const float4 *w4 = reinterpret_cast<const float4 *>(wout_s + g * hn + c0);
+            const uint32_t col0 = lane_base + (g ? 384u : 128u);
+            float d4[4] = {0.f, 0.f, 0.f, 0.f};
+            uint32_t ra[32], rb[32];
+            auto reduce = [&](const uint32_t (&r)[32], int c0) {
+                const uint4 *w8 = reinterpret_cast<const uint4 *>(wout_s + g * hn + c0);   // eight bf16 weights per load
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float4 bb = b4[q], ww = w4[q];
-                    dot = fmaf(fmaxf(__uint_as_float(r[4 * q]) + bb.x, 0.f), ww.x, dot);
-                    dot = fmaf(fmaxf(__uint_as_float(r[4 * q + 1]) + bb.y, 0.f), ww.y, dot);
-                    dot = fmaf(fmaxf(__uint_as_float(r[4 * q + 2]) + bb.z, 0.f), ww.z, dot);
-                    dot = fmaf(fmaxf(__uint_as_float(r[4 * q + 3]) + bb.w, 0.f), ww.w, dot);
+                for (int q = 0; q < 4; ++q) {
+                    const uint4 ww = w8[q];
+                    const float2 w0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ww.x));
+                    const float2 w1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ww.y));
+                    const float2 w2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ww.z));
+                    const float2 w3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ww.w));
+                    d4[0] = fmaf(fmaxf(__uint_as_float(r[8 * q]), 0.f), w0.x, d4[0]);
+                    d4[1] = fmaf(fmaxf(__uint_as_float(r[8 * q + 1]), 0.f), w0.y, d4[1]);
+                    d4[2] = fmaf(fmaxf(__uint_as_float(r[8 * q + 2]), 0.f), w1.x, d4[2]);
+                    d4[3] = fmaf(fmaxf(__uint_as_float(r[8 * q + 3]), 0.f), w1.y, d4[3]);
+                    d4[0] = fmaf(fmaxf(__uint_as_float(r[8 * q + 4]), 0.f), w2.x, d4[0]);
+                    d4[1] = fmaf(fmaxf(__uint_as_float(r[8 * q + 5]), 0.f), w2.y, d4[1]);
+                    d4[2] = fmaf(fmaxf(__uint_as_float(r[8 * q + 6]), 0.f), w3.x, d4[2]);
+                    d4[3] = fmaf(fmaxf(__uint_as_float(r[8 * q + 7]), 0.f), w3.y, d4[3]);
+                }
+            };
+            tmem_ld32(col0, ra);
+#pragma unroll 1
+            for (int c0 = 0; c0 < hn; c0 += 64) {   // hn is a multiple of 32
+                tmem_ld_wait();
+                if (c0 + 32 < hn) tmem_ld32(col0 + (uint32_t)(c0 + 32), rb);
+                reduce(ra, c0);
+                if (c0 + 32 < hn) {
+                    tmem_ld_wait();
+                    if (c0 + 64 < hn) tmem_ld32(col0 + (uint32_t)(c0 + 64), ra);
+                    reduce(rb, c0 + 32);
                 }
             }
+            dot = (d4[0] + d4[1]) + (d4[2] + d4[3]);
         }
         if (g == 1) dot_s[row] = dot;
         named_bar_sync(1, 256);
         if (g == 0 && ok && row < cnt) {
-            float logit = dot + dot_s[row] + p.b_out[0];
+            float logit = dot + dot_s[row] + b_out;
             if (p.emit_sigmoid) logit = 1.0f / (1.0f + expf(-logit));
             if (!good) logit = __int_as_float(0x7fc00000);
             p.sl.logits[pos0 + row] = logit;
@@ -329,7 +394,7 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
                     const uint64_t vd = umma_desc_mn_sw128(smem_u32(smKV + j * 32768), kChunk);
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
-                        umma_bf16_ts(tmem_base + 256u, tmem_base + (uint32_t)(j * 128 + kk * 8), vd + (uint64_t)(kk * (2048 >> 4)), idesc_pv,
+                        umma_bf16_ts(tmem_base + 256u, tmem_base + (uint32_t)(384 + j * 64 + kk * 8), vd + (uint64_t)(kk * (2048 >> 4)), idesc_pv,
                                      (j > 0 || kk > 0) ? 1u : 0u);
                 }
                 umma_commit(bar(BAR_O_FINAL));
@@ -368,7 +433,20 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
                 if (sa >= 0) umma_commit(bar(BAR_EMPTY_A + sa));
                 if (kc == 1) umma_commit(bar(BAR_E_FREE));
             }
-            if (ok) umma_commit(bar(BAR_ACC1_FULL));
+            // the cached user partial p_u (first-layer bias of this request): ones x [high; remainder]
+            const int s_ones = p.n_cross % kAStages;
+            uint64_t ones_d = 0;
+            if (ok) ok = mbar_wait(bar(BAR_FULL_A + s_ones), (uint32_t)((p.n_cross / kAStages) & 1), abort_flag) &&
+                         mbar_wait(bar(BAR_BIAS_FULL), 0u, abort_flag);
+            if (ok) {
+                fence_proxy_async();
+                tc_fence_after();
+                ones_d = umma_desc_sw128(smem_u32(a_stage(s_ones)));
+                constexpr uint32_t idesc_b1 = umma_idesc_bf16_bmn(kTcTile, 256);
+                umma_bf16(tmem_base, ones_d, umma_desc_mn_sw128(smem_u32(smE), 2048), idesc_b1, 1u);
+                umma_bf16(tmem_base + 256u, ones_d, umma_desc_mn_sw128(smem_u32(smE + 8192), 2048), idesc_b1, 1u);
+                umma_commit(bar(BAR_ACC1_FULL));
+            }
             // layer 2: A = the packed activations in tensor memory, two halves of the output units
             ok = ok && mbar_wait(bar(BAR_H1_FULL), 0u, abort_flag);
             tc_fence_after();
@@ -392,7 +470,12 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
                 }
                 umma_commit(bar(BAR_EMPTY_B + sb));
             }
-            if (ok) umma_commit(bar(BAR_ACC2_FULL));
+            if (ok) {
+                const uint32_t idesc_b2 = umma_idesc_bf16_bmn(kTcTile, p.H2 >> 1);
+                umma_bf16(tmem_base + 128u, ones_d, umma_desc_mn_sw128(smem_u32(smE + 16384), 2048), idesc_b2, 1u);
+                umma_bf16(tmem_base + 384u, ones_d, umma_desc_mn_sw128(smem_u32(smE + 16384 + (p.H2 >> 7) * 2048), 2048), idesc_b2, 1u);
+                umma_commit(bar(BAR_ACC2_FULL));
+            }
         }
         __syncwarp();
     } else if (warp < kFBWarp) {
@@ -400,20 +483,12 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
         const int pt = tid - kFProdWarp0 * 32;
         const int sub = pt & 7, r0 = pt >> 3;   // 16-byte slot of the 128-byte chunk row; rows r0, r0 + 16, ...
         const uint32_t row_off = (uint32_t)(r0 * 128) + (uint32_t)((sub ^ (r0 & 7)) << 4);
-        int id[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int r = r0 + 16 * i;
-            int v = -1;
-            if (r < cnt) {
-                v = p.sl.ids[pos0 + r];
-                if (v < 0 || (int64_t)v >= p.M) {
-                    v = -1;
-                    if (sub == 0) atomicOr(p.sl.status, AIF_STATUS_BAD_ID);
-                }
+        for (int i = 0; i < 8; ++i)
+            if (r0 + 16 * i < cnt && (id[i] < 0 || (int64_t)id[i] >= p.M)) {
+                id[i] = -1;
+                if (sub == 0) atomicOr(p.sl.status, AIF_STATUS_BAD_ID);
             }
-            id[i] = v;
-        }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const uint8_t *gsrc = p.E + (id[i] >= 0 ? (size_t)id[i] * 256 + sub * 16 : 0);
@@ -457,6 +532,19 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
             cp_async_arrive_noinc(bar(BAR_FULL_A + s));
             if (i + 1 < p.n_cross) resolve(i + 1);
         }
+        // the tile of ones that carries the biases: one more stage of the ring, columns 0 and 1 of row pt
+        if (ok) {
+            const int i = p.n_cross, s = i % kAStages;
+            ok = mbar_wait(bar(BAR_EMPTY_A + s), (uint32_t)(((i / kAStages) & 1) ^ 1), abort_flag);
+            if (ok && s >= 2 && i < kAStages && nb == 2) ok = mbar_wait(bar(BAR_O_FINAL), 0u, abort_flag);
+            if (ok) {
+                unsigned char *rowp = a_stage(s) + pt * 128;
+                *reinterpret_cast<uint4 *>(rowp + ((0 ^ (pt & 7)) << 4)) = make_uint4(0x3F803F80u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4 *>(rowp + ((1 ^ (pt & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                fence_proxy_async();
+                mbar_arrive(bar(BAR_FULL_A + s));
+            }
+        }
         cp_async_wait_all();
     } else {
         // ===================== key/value blocks and weights (TMA) =====================
@@ -499,6 +587,16 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
     if (warp == kFMmaWarp) tmem_dealloc(tmem_base, 512);
 }
 
+// bias [n] fp32 -> [2][n] bf16: high parts, then the remainders bias - high
+__global__ void k_split_bias(const float *__restrict__ b, int n, __nv_bfloat16 *__restrict__ out)
+{
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const __nv_bfloat16 hi = __float2bfloat16_rn(b[i]);
+        out[i] = hi;
+        out[n + i] = __float2bfloat16_rn(b[i] - __bfloat162float(hi));
+    }
+}
+
 }  // namespace
 
 bool tc_fused_supported(const aif_config &c)
@@ -511,9 +609,21 @@ bool tc_fused_supported(const aif_config &c)
     return tc_supported(c) && tc_att_supported(c);
 }
 
-cudaError_t tc_fused_prepare(aif_ctx *)
+cudaError_t tc_fused_prepare(aif_ctx *ctx)
 {
+    void *ptr = nullptr;   // the second layer's bias as the tensor cores take it: [2][hidden[1]] bf16
+    cudaError_t e = cudaMalloc(&ptr, 2 * 256 * 2);
+    if (e != cudaSuccess) return e;
+    ctx->allocations.push_back(ptr), ctx->device_bytes += 2 * 256 * 2;
+    ctx->tc_fused_plan = ptr;
     return cudaFuncSetAttribute(k_request_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
+}
+
+cudaError_t tc_fused_prepare_weights(aif_ctx *ctx, cudaStream_t st)
+{
+    k_split_bias<<<1, 256, 0, st>>>(ctx->b[1], ctx->cfg.hidden[1], reinterpret_cast<__nv_bfloat16 *>(ctx->tc_fused_plan));
+    count_launch();
+    return cudaGetLastError();
 }
 
 // One launch for the whole call; the caller has checked tc_fused_supported and that no sequence is longer than 256.
@@ -526,7 +636,7 @@ cudaError_t launch_request_fused(const aif_ctx *ctx, const ScoreLaunch &sl, cuda
     p.n_cross = c.F * c.dc / 64;
     p.H2 = c.hidden[1], p.emit_sigmoid = c.emit_sigmoid;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.d);
-    p.b2 = ctx->b[1], p.w_out = (const __nv_bfloat16 *)ctx->w_out, p.b_out = ctx->b_out;
+    p.b2_hl = reinterpret_cast<const __nv_bfloat16 *>(ctx->tc_fused_plan), p.w_out = (const __nv_bfloat16 *)ctx->w_out, p.b_out = ctx->b_out;
     const CUtensorMap *ms = reinterpret_cast<const CUtensorMap *>(tc_att_tmap(ctx));
     const CUtensorMap *m1 = reinterpret_cast<const CUtensorMap *>(tc_weight_tmap(ctx, 0));
     const CUtensorMap *m2 = reinterpret_cast<const CUtensorMap *>(tc_weight_tmap(ctx, 1));
