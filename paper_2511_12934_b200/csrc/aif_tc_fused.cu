@@ -24,8 +24,8 @@
 //
 // Tensor memory (512 columns): attention uses [0, 256) for the scores of up to two key blocks, [256, 384) for O and
 // [384, 512) for the probabilities (packed bf16, 64 columns per key block).  Layer 1 then fills two 256-column
-// accumulators [0, 256) and [256, 512); its activations are packed in place into [0, 128) and [256, 384); layer 2
-// accumulates its two halves into the freed columns [128, 256) and [384, 512).
+// accumulators [0, 256) and [256, 512); its activations are packed over them into [0, 128) and [384, 512); layer 2
+// accumulates into the freed columns [128, 384).
 // Shared memory: item tile 32 KB | key/value blocks 64 KB, later the attention chunks and two more stages of the
 // cross-feature ring | two cross-feature stages 32 KB | weight ring 3 x 32 KB | barriers and exchange arrays.
 // Every wait is bounded: on expiry the CTA raises AIF_STATUS_TIMEOUT, every role skips its remaining work, tensor
@@ -281,8 +281,8 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
         fence_proxy_async();
         mbar_arrive(bar(BAR_BIAS_FULL));
         named_bar_sync(1, 256);
-        // ---- layer-1 epilogue: slice g, ReLU, 32 accumulator columns -> 16 columns of packed bf16, in place (the target
-        // columns [16 c, 16 c + 16) lie in chunks already read); the load of the next chunk is in flight meanwhile
+        // ---- layer-1 epilogue: slice g, ReLU, 32 accumulator columns -> 16 columns of packed bf16, over accumulator
+        // columns already read; the load of the next chunk is in flight meanwhile
         wait(BAR_ACC1_FULL);
         tc_fence_after();
         if (ok) {
@@ -295,17 +295,20 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
                     const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[2 * q]), 0.f), fmaxf(__uint_as_float(r[2 * q + 1]), 0.f));
                     packed[q] = *reinterpret_cast<const uint32_t *>(&h0);
                 }
-                tmem_st16(col0 + (uint32_t)(16 * c), packed);
+                tmem_st16(lane_base + (uint32_t)((g ? 384 : 0) + 16 * c), packed);
             };
-            tmem_ld32(col0, ra);
+            // slice 0 is read upwards and packed into [0, 128), slice 1 downwards and packed into [384, 512): either way
+            // a packed piece lands on columns that have been read, and the 256 columns in between become free
+            auto chunk_of = [&](int i) { return g ? 7 - i : i; };
+            tmem_ld32(col0 + (uint32_t)(32 * chunk_of(0)), ra);
 #pragma unroll 1
-            for (int c = 0; c < 8; c += 2) {
+            for (int i = 0; i < 8; i += 2) {
                 tmem_ld_wait();
-                tmem_ld32(col0 + (uint32_t)(32 * (c + 1)), rb);
-                finish(ra, c);
+                tmem_ld32(col0 + (uint32_t)(32 * chunk_of(i + 1)), rb);
+                finish(ra, chunk_of(i));
                 tmem_ld_wait();
-                if (c + 2 < 8) tmem_ld32(col0 + (uint32_t)(32 * (c + 2)), ra);
-                finish(rb, c + 1);
+                if (i + 2 < 8) tmem_ld32(col0 + (uint32_t)(32 * chunk_of(i + 2)), ra);
+                finish(rb, chunk_of(i + 1));
             }
             tmem_st_wait();
         }
@@ -317,7 +320,7 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
         float dot = 0.f;
         if (ok) {
             const int hn = p.H2 >> 1;
-            const uint32_t col0 = lane_base + (g ? 384u : 128u);
+            const uint32_t col0 = lane_base + 128u + (uint32_t)(g * hn);
             float d4[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t ra[32], rb[32];
             auto reduce = [&](const uint32_t (&r)[32], int c0) {
@@ -367,7 +370,7 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
             constexpr uint32_t idesc_qk = umma_idesc_bf16(kTcTile, 128);
             constexpr uint32_t idesc_pv = umma_idesc_bf16_bmn(kTcTile, 128);
             constexpr uint32_t idesc1 = umma_idesc_bf16(kTcTile, 256);
-            const uint32_t idesc2 = umma_idesc_bf16(kTcTile, p.H2 >> 1);
+            const uint32_t idesc2 = umma_idesc_bf16(kTcTile, p.H2);
             bool ok = mbar_wait(bar(BAR_E_FULL), 0u, abort_flag);
             fence_proxy_async();   // the item rows were written by cp.async
             // scores = Q K^T, one key block after the other
@@ -447,33 +450,26 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
                 umma_bf16(tmem_base + 256u, ones_d, umma_desc_mn_sw128(smem_u32(smE + 8192), 2048), idesc_b1, 1u);
                 umma_commit(bar(BAR_ACC1_FULL));
             }
-            // layer 2: A = the packed activations in tensor memory, two halves of the output units
+            // layer 2: A = the packed activations in tensor memory
             ok = ok && mbar_wait(bar(BAR_H1_FULL), 0u, abort_flag);
             tc_fence_after();
-            const uint64_t half_off = (uint64_t)(((p.H2 >> 1) * 128) >> 4);
             for (int kc = 0; ok && kc < kH1 / 64; ++kc, ++qb) {
                 const int sb = qb % kBStages;
                 ok = mbar_wait(bar(BAR_FULL_B + sb), (uint32_t)((qb / kBStages) & 1), abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint64_t bd0 = umma_desc_sw128(smem_u32(smB + sb * kBStage));
+                const uint64_t bd = umma_desc_sw128(smem_u32(smB + sb * kBStage));
 #pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    const uint32_t d_tmem = tmem_base + (hf ? 384u : 128u);
-                    const uint64_t bd = bd0 + (hf ? half_off : 0ull);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const int k16 = kc * 4 + kk;   // 16 activations = 8 packed columns
-                        const uint32_t a_tmem = tmem_base + (uint32_t)(k16 < 16 ? 8 * k16 : 256 + 8 * (k16 - 16));
-                        umma_bf16_ts(d_tmem, a_tmem, bd + (uint64_t)(2 * kk), idesc2, (kc > 0 || kk > 0) ? 1u : 0u);
-                    }
+                for (int kk = 0; kk < 4; ++kk) {
+                    const int k16 = kc * 4 + kk;   // 16 activations = 8 packed columns
+                    const uint32_t a_tmem = tmem_base + (uint32_t)(k16 < 16 ? 8 * k16 : 384 + 8 * (k16 - 16));
+                    umma_bf16_ts(tmem_base + 128u, a_tmem, bd + (uint64_t)(2 * kk), idesc2, (kc > 0 || kk > 0) ? 1u : 0u);
                 }
                 umma_commit(bar(BAR_EMPTY_B + sb));
             }
             if (ok) {
-                const uint32_t idesc_b2 = umma_idesc_bf16_bmn(kTcTile, p.H2 >> 1);
+                const uint32_t idesc_b2 = umma_idesc_bf16_bmn(kTcTile, p.H2);
                 umma_bf16(tmem_base + 128u, ones_d, umma_desc_mn_sw128(smem_u32(smE + 16384), 2048), idesc_b2, 1u);
-                umma_bf16(tmem_base + 384u, ones_d, umma_desc_mn_sw128(smem_u32(smE + 16384 + (p.H2 >> 7) * 2048), 2048), idesc_b2, 1u);
                 umma_commit(bar(BAR_ACC2_FULL));
             }
         }
