@@ -35,7 +35,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # CUDA-core kernels: SMs x lanes x 2 x max clock
 
 # DRAM traffic per launch of the dominant kernel from the committed ncu summary (profiles/), bytes; None = not captured.
-NCU_TRAFFIC_BYTES = {("c2_paper_shaped", "layer1"): 7376128}      # profiles/scoring_step_c2.md
+NCU_TRAFFIC_BYTES = {("c2_paper_shaped", "score_fused"): 4867840}      # profiles/scoring_step_c2.md
 
 
 # ----------------------------------------------------------------------------------------------------------------
