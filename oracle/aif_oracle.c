@@ -250,6 +250,69 @@ static void linear(const void *W, int dtype, const float *b, int rows, int cols,
 }
 
 /* ---------------------------------------------------------------------------------------------
+ * Item side, nearline (Section 3.2 eq. 4; Algorithm 1 step 3; Section 4.2 eq. 5).  One call computes,
+ * for n items, what the nearline pipeline stores in the index table.
+ *   eq. 4   I^ = MLP(I).  Reading (the paper names no widths or activation): one hidden layer,
+ *           I^ = W_1 ReLU(W_0 I + b_0) + b_1, widths dI -> hI -> d, linear output.
+ *   Alg. 1  step 3: w^ = Softmax(I_id B^T / sqrt(d)), one row of n_bridge weights per item; I_id is the
+ *           item's d-wide id embedding (an input of its own; the algorithm's I is d-wide).
+ *   eq. 5   signature bits of the item's multi-modal embedding M (see orc_lsh_hash_bits), packed
+ *           first-bit-most-significant.
+ * Inputs in storage type `dtype`; outputs in double (vectors, weights) and bytes (signatures).  A NULL
+ * output (with its inputs) skips that part.
+ * ------------------------------------------------------------------------------------------- */
+void orc_item_nearline(int dtype, int64_t n, int dI, int hI, int d, const void *I_raw, const void *W0, const float *b0,
+                       const void *W1, const float *b1, double *I_hat, int n_bridge, const void *I_id, const void *bridges,
+                       double *w_hat, int d_mm, int dbits, const void *M_mm, const void *W_hash, uint8_t *sig)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) {
+        if (I_hat) {
+            double *x = (double *)malloc(sizeof(double) * (size_t)(dI + hI));
+            double *h = x + dI;
+            for (int c = 0; c < dI; ++c) x[c] = ld(I_raw, i * dI + c, dtype);
+            linear(W0, dtype, b0, hI, dI, x, h);
+            for (int j = 0; j < hI; ++j) h[j] = h[j] > 0.0 ? h[j] : 0.0;
+            linear(W1, dtype, b1, d, hI, h, I_hat + i * d);
+            free(x);
+        }
+        if (w_hat) {
+            double s[64], mx = -INFINITY, den = 0.0;
+            for (int k = 0; k < n_bridge; ++k) {
+                double acc = 0.0;
+                for (int c = 0; c < d; ++c) acc += ld(I_id, i * d + c, dtype) * ld(bridges, (int64_t)k * d + c, dtype);
+                s[k] = acc / sqrt((double)d);
+                if (s[k] > mx) mx = s[k];
+            }
+            for (int k = 0; k < n_bridge; ++k) den += exp(s[k] - mx);
+            for (int k = 0; k < n_bridge; ++k) w_hat[i * n_bridge + k] = exp(s[k] - mx) / den;
+        }
+        if (sig) {
+            double *m = (double *)malloc(sizeof(double) * (size_t)d_mm * (size_t)(1 + dbits));
+            double *Wd = m + d_mm;
+            uint8_t bits[1024];
+            for (int c = 0; c < d_mm; ++c) m[c] = ld(M_mm, i * d_mm + c, dtype);
+            for (int64_t c = 0; c < (int64_t)d_mm * dbits; ++c) Wd[c] = ld(W_hash, c, dtype);
+            orc_lsh_hash_bits(m, Wd, d_mm, dbits, bits);
+            orc_pack_bits(bits, dbits, sig + i * (dbits / 8));
+            free(m);
+        }
+    }
+}
+
+/* The projections behind eq. 5's bits, for tests that need to know how close to zero a bit was decided. */
+void orc_lsh_projections(int dtype, int64_t n, int d_mm, int dbits, const void *M_mm, const void *W_hash, double *proj)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i)
+        for (int k = 0; k < dbits; ++k) {
+            double p = 0.0;
+            for (int c = 0; c < d_mm; ++c) p += ld(M_mm, i * d_mm + c, dtype) * ld(W_hash, (int64_t)k * d_mm + c, dtype);
+            proj[i * dbits + k] = p;
+        }
+}
+
+/* ---------------------------------------------------------------------------------------------
  * User side, eqs. 1-3 (Section 3.1).  Readings: FFN(x) = ReLU(x W_a^T + b_a) W_b^T + b_b, Pooling =
  * mean over the sequence, combined vector = U_self_attention + U_profile_attention.
  * profile [dU], seq [l x dU] in storage type; u_out [d], S_out [l x d] (= U^_seq) in double.

@@ -196,6 +196,53 @@ def bea(w_hat, V) -> np.ndarray:
     return out
 
 
+def item_nearline(dtype: int, I_raw=None, W0=None, b0=None, W1=None, b1=None, I_id=None, bridges=None, M_mm=None,
+                  W_hash=None) -> dict:
+    """Item side of the nearline pipeline for n items (Section 3.2 eq. 4, Algorithm 1 step 3, Section 4.2 eq. 5).
+    Arrays in storage type (biases float32).  Returns the parts whose inputs were given: "I_hat" [n x d] float64,
+    "w_hat" [n x n_bridge] float64, "sig" [n x dbits/8] uint8."""
+    out = {}
+    n = next(a.shape[0] for a in (I_raw, I_id, M_mm) if a is not None)
+    I_hat = w_hat = sig = None
+    dI = hI = d = nb = d_mm = dbits = 0
+    if I_raw is not None:
+        I_raw, W0, W1 = _store(I_raw, dtype), _store(W0, dtype), _store(W1, dtype)
+        b0, b1 = np.ascontiguousarray(b0, dtype=np.float32), np.ascontiguousarray(b1, dtype=np.float32)
+        (hI, dI), d = W0.shape, W1.shape[0]
+        assert I_raw.shape == (n, dI) and W1.shape == (d, hI) and b0.shape == (hI,) and b1.shape == (d,)
+        I_hat = np.zeros((n, d))
+    if I_id is not None:
+        I_id, bridges = _store(I_id, dtype), _store(bridges, dtype)
+        nb, d = bridges.shape
+        assert I_id.shape == (n, d) and nb <= 64
+        w_hat = np.zeros((n, nb))
+    if M_mm is not None:
+        M_mm, W_hash = _store(M_mm, dtype), _store(W_hash, dtype)
+        dbits, d_mm = W_hash.shape
+        assert M_mm.shape == (n, d_mm) and dbits % 8 == 0 and dbits <= 1024
+        sig = np.zeros((n, dbits // 8), dtype=np.uint8)
+    lib().orc_item_nearline(C.c_int(dtype), C.c_int64(n), C.c_int(dI), C.c_int(hI), C.c_int(d), _p(I_raw), _p(W0), _p(b0),
+                            _p(W1), _p(b1), _p(I_hat), C.c_int(nb), _p(I_id), _p(bridges), _p(w_hat), C.c_int(d_mm),
+                            C.c_int(dbits), _p(M_mm), _p(W_hash), _p(sig))
+    if I_hat is not None:
+        out["I_hat"] = I_hat
+    if w_hat is not None:
+        out["w_hat"] = w_hat
+    if sig is not None:
+        out["sig"] = sig
+    return out
+
+
+def lsh_projections(dtype: int, M_mm: np.ndarray, W_hash: np.ndarray) -> np.ndarray:
+    """The projections M W_hash^T [n x dbits] whose signs eq. 5 keeps."""
+    M_mm, W_hash = _store(M_mm, dtype), _store(W_hash, dtype)
+    n, d_mm = M_mm.shape
+    dbits = W_hash.shape[0]
+    proj = np.zeros((n, dbits))
+    lib().orc_lsh_projections(C.c_int(dtype), C.c_int64(n), C.c_int(d_mm), C.c_int(dbits), _p(M_mm), _p(W_hash), _p(proj))
+    return proj
+
+
 def table_refresh(table: np.ndarray, ids: Optional[np.ndarray], rows: np.ndarray) -> int:
     """In-place write of `rows` into `table` (2-D, same row width); returns the number of bad ids."""
     assert table.flags.c_contiguous and rows.flags.c_contiguous and table.dtype == rows.dtype

@@ -494,3 +494,91 @@ def test_bf16_storage_is_widened_exactly():
     # round to nearest even on the 16 dropped bits
     assert synth.to_bf16_bits(np.array([1.00390625], np.float32))[0] == 0x3F80      # tie -> even (down)
     assert synth.to_bf16_bits(np.array([1.01171875], np.float32))[0] == 0x3F82      # tie -> even (up)
+
+
+# ------------------------------------------------------------------------------------------------
+# item side of the nearline pipeline (Section 3.2 eq. 4, Algorithm 1 step 3, Section 4.2 eq. 5)
+# ------------------------------------------------------------------------------------------------
+def test_item_tower_special_cases_and_brute_force():
+    g = np.random.default_rng(11)
+    n, dI, hI, d = 5, 12, 7, 4
+    I = g.standard_normal((n, dI)).astype(np.float32)
+    W0 = g.standard_normal((hI, dI)).astype(np.float32)
+    b0 = g.standard_normal(hI).astype(np.float32)
+    W1 = g.standard_normal((d, hI)).astype(np.float32)
+    b1 = g.standard_normal(d).astype(np.float32)
+    got = orc.item_nearline(orc.F32, I_raw=I, W0=W0, b0=b0, W1=W1, b1=b1)["I_hat"]
+    # brute force, scalar loops
+    for i in range(n):
+        h = [max(0.0, float(b0[j]) + sum(float(W0[j, c]) * float(I[i, c]) for c in range(dI))) for j in range(hI)]
+        for k in range(d):
+            want = float(b1[k]) + sum(float(W1[k, j]) * h[j] for j in range(hI))
+            assert abs(got[i, k] - want) < 1e-12
+    # zero first layer: the output is W1 ReLU(b0) + b1 for every item
+    z = orc.item_nearline(orc.F32, I_raw=I, W0=np.zeros_like(W0), b0=b0, W1=W1, b1=b1)["I_hat"]
+    assert np.allclose(z, (W1.astype(np.float64) @ np.maximum(b0.astype(np.float64), 0) + b1)[None, :], atol=1e-12)
+    # all pre-activations positive: the network is affine, I^ = W1 (W0 I + b0) + b1
+    big = np.full(hI, 100.0, dtype=np.float32)
+    a = orc.item_nearline(orc.F32, I_raw=I, W0=W0, b0=big, W1=W1, b1=b1)["I_hat"]
+    want = (W1.astype(np.float64) @ (W0.astype(np.float64) @ I.astype(np.float64).T + big[:, None].astype(np.float64))).T + b1
+    assert np.allclose(a, want, atol=1e-10)
+    # all pre-activations negative: only the output bias is left
+    neg = orc.item_nearline(orc.F32, I_raw=I, W0=W0, b0=-big, W1=W1, b1=b1)["I_hat"]
+    assert np.allclose(neg, b1[None, :].astype(np.float64), atol=0)
+    # a hidden unit that is negative for one sign of the input and positive for the other: ReLU sits between the layers
+    one = orc.item_nearline(orc.F32, I_raw=np.array([[1.0], [-1.0]], np.float32), W0=np.array([[2.0]], np.float32),
+                            b0=np.zeros(1, np.float32), W1=np.array([[3.0]], np.float32), b1=np.zeros(1, np.float32))["I_hat"]
+    assert one[0, 0] == 6.0 and one[1, 0] == 0.0
+
+
+def test_item_bridge_weights_are_a_softmax_over_the_bridges():
+    g = np.random.default_rng(12)
+    n, d, nb = 6, 16, 8
+    I = g.standard_normal((n, d)).astype(np.float32)
+    Bm = g.standard_normal((nb, d)).astype(np.float32)
+    w = orc.item_nearline(orc.F32, I_id=I, bridges=Bm)["w_hat"]
+    assert w.shape == (n, nb) and np.allclose(w.sum(axis=1), 1.0, atol=1e-14) and (w > 0).all()
+    # closed form against a hand-written softmax of I B^T / sqrt(d) (item rows times bridge rows: not B I^T transposed wrongly)
+    s = (I.astype(np.float64) @ Bm.astype(np.float64).T) / math.sqrt(d)
+    e = np.exp(s - s.max(axis=1, keepdims=True))
+    assert np.allclose(w, e / e.sum(axis=1, keepdims=True), atol=1e-14)
+    # equal bridges: uniform weights; a bridge equal to a large multiple of the item: weight near one
+    u = orc.item_nearline(orc.F32, I_id=I, bridges=np.tile(Bm[:1], (nb, 1)))["w_hat"]
+    assert np.allclose(u, 1.0 / nb, atol=1e-15)
+    Bs = np.zeros((nb, d), np.float32)
+    Bs[3] = 50.0 * I[2]
+    assert orc.item_nearline(orc.F32, I_id=I, bridges=Bs)["w_hat"][2, 3] > 0.999
+    # the scale is 1 / sqrt(d): with d = 4 and products (2 ln 3, 0) the scores are (ln 3, 0), the weights (3, 1) / 4
+    I2 = np.array([[1.0, 0.0, 0.0, 0.0]], np.float32)
+    B2 = np.array([[2.0 * math.log(3.0), 0, 0, 0], [0, 0, 0, 0]], np.float32)
+    w2 = orc.item_nearline(orc.F32, I_id=I2, bridges=B2)["w_hat"]
+    assert np.allclose(w2, [[0.75, 0.25]], atol=1e-6)
+    # Algorithm 1 step 4 on top: with one-hot weights the weighted sum picks a user-side vector
+    V = g.standard_normal((nb, d))
+    onehot = np.zeros(nb); onehot[5] = 1.0
+    assert np.array_equal(orc.bea(onehot, V), V[5])
+
+
+def test_item_signatures_pack_eq5_bits_first_bit_most_significant():
+    g = np.random.default_rng(13)
+    n, d_mm, dbits = 9, 24, 64
+    M = g.standard_normal((n, d_mm)).astype(np.float32)
+    W = g.standard_normal((dbits, d_mm)).astype(np.float32)
+    sig = orc.item_nearline(orc.F32, M_mm=M, W_hash=W)["sig"]
+    proj = orc.lsh_projections(orc.F32, M, W)
+    assert np.allclose(proj, M.astype(np.float64) @ W.astype(np.float64).T, atol=1e-12)
+    for i in range(n):
+        bits = orc.lsh_hash_bits(M[i], W)
+        assert np.array_equal(bits, (proj[i] > 0).astype(np.uint8))
+        assert np.array_equal(sig[i], np.packbits(bits))        # numpy packs big-endian: first bit = most significant
+        assert np.array_equal(sig[i], orc.pack_bits(bits))
+    # an item whose first eight projections have the signs 0 0 1 1 0 1 0 1 gets the byte 53 (Section 4.2's example)
+    Wd = np.zeros((8, 8), np.float32)
+    for k, b in enumerate([0, 0, 1, 1, 0, 1, 0, 1]):
+        Wd[k, k] = 1.0 if b else -1.0
+    s53 = orc.item_nearline(orc.F32, M_mm=np.ones((1, 8), np.float32), W_hash=Wd)["sig"]
+    assert s53.tolist() == [[53]]
+    # similarity of an item with itself is 1, with its negation 0 (eq. 6 on the produced signatures)
+    both = orc.item_nearline(orc.F32, M_mm=np.vstack([M[:1], -M[:1]]), W_hash=W)["sig"]
+    sim = orc.lsh_similarity(both[:1], both, dbits)
+    assert sim[0, 0] == 1.0 and sim[0, 1] == 0.0
