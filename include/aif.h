@@ -174,6 +174,42 @@ int aif_load_weights(aif_ctx *ctx, const aif_weights *w, aif_stream stream);
 int aif_item_nearline_refresh(aif_ctx *ctx, const int32_t *ids, int64_t n, const void *rows, const void *bea_w,
                               const uint8_t *lsh_sig, aif_stream stream);
 
+/* Weights of the item side of the nearline pipeline.  Device pointers, storage type unless noted; copied in by
+ * aif_load_item_weights.
+ *   eq. 4 (Section 3.2) "dimensionality reduction": I^ = W_i1 ReLU(W_i0 I + b_i0) + b_i1, widths dI -> hI -> d (the
+ *     paper says "a multi-layer perceptron" and no more; one ReLU hidden layer and a linear output is this library's reading)
+ *   Algorithm 1 step 3: w^ = Softmax(I_id B^T / sqrt(d)): `bridges` = B [n_bridge x d] (needed iff the BEA block is on)
+ *   eq. 5 (Section 4.2): signature bits = [M W_hash^T > 0]: `W_hash` [lsh_bits x d_mm] (needed iff an LSH block is on) */
+typedef struct {
+    uint32_t struct_size;
+    int32_t dI, hI, d_mm;
+    const void *W_i0;     /* [hI x dI] */
+    const float *b_i0;    /* [hI] fp32 */
+    const void *W_i1;     /* [d x hI] */
+    const float *b_i1;    /* [d] fp32 */
+    const void *bridges;  /* [n_bridge x d] or NULL */
+    const void *W_hash;   /* [lsh_bits x d_mm] or NULL */
+} aif_item_weights;
+
+/* Copies the item-side weights in (device to device, on `stream`) and sizes the scratch of
+ * aif_item_nearline_compute.  Does not touch model_version: cached user states do not depend on these weights.
+ * Errors: AIF_ERR_ARG (NULL, struct_size), AIF_ERR_SHAPE (widths < 1, not multiples of 4), AIF_ERR_OOM. */
+int aif_load_item_weights(aif_ctx *ctx, const aif_item_weights *w, aif_stream stream);
+
+/* Item side, nearline, as a compute call (Section 3.2: "generating vectors for the full candidate set stored in an
+ * indexing table", triggered by model or feature updates; Section 3.4: full and incremental updates): from raw item
+ * features to the table rows that aif_item_nearline_refresh would have been handed.
+ *   I_raw  device [n x dI] storage type: concatenated item embeddings; gives the item vectors I^ (eq. 4)
+ *   I_id   device [n x d] storage type or NULL: item id embeddings for the BEA weights (Algorithm 1 step 3); NULL: the
+ *          freshly computed I^ takes their place.  Read only when the BEA block is on.
+ *   M_mm   device [n x d_mm] storage type: multi-modal embeddings for the signatures (eq. 5); required iff an LSH block is on
+ * ids == NULL: rows i -> table row i (n <= M); otherwise rows i -> table row ids[i] with the rules of
+ * aif_item_nearline_refresh.  Bumps table_version.  Needs aif_load_item_weights first (AIF_ERR_NOT_READY).
+ * On bf16 contexts whose widths are multiples of 64 the two layers and the hash projections run on the tensor cores;
+ * a signature bit whose projection is within rounding of zero may then differ from an evaluation in another order. */
+int aif_item_nearline_compute(aif_ctx *ctx, const int32_t *ids, int64_t n, const void *I_raw, const void *I_id,
+                              const void *M_mm, aif_stream stream);
+
 /* User side, online-asynchronous (Section 3.1 eqs. 1-3, Section 3.3 "User-Side Pre-Processing").  Takes a free
  * slot of the arena and fills it on `side_stream`: u, S = U^_seq [L x d], the cross pre-cache T, V, the
  * sequence signatures, and p_u = W1[:, user columns] u + b1 (fp32), so that the real-time phase never touches
@@ -250,6 +286,11 @@ int aif_score_noalloc(aif_ctx *ctx, const aif_user_state *state, const int32_t *
  * ids: device int32 [n]; rows_out: device [n x d] storage type.  Bad ids give zero rows and the status bit.
  * Exists so that the gather can be measured against HBM bandwidth by itself. */
 int aif_gather_rows(aif_ctx *ctx, const int32_t *ids, int64_t n, void *rows_out, aif_stream stream);
+
+/* The same for the sidecars that nearline updates write beside the item vectors: bea_w_out[i] = the BEA weight row
+ * (device [n x n_bridge] storage type), sig_out[i] = the signature (device [n x lsh_bits/8]) of item ids[i]; a NULL
+ * output is skipped, an output whose block is off is AIF_ERR_ARG.  Bad ids give zero rows and the status bit. */
+int aif_gather_sidecars(aif_ctx *ctx, const int32_t *ids, int64_t n, void *bea_w_out, uint8_t *sig_out, aif_stream stream);
 
 /* Reads and clears the device status word (synchronises the device).  bits: host. */
 int aif_poll_status(aif_ctx *ctx, uint32_t *bits);

@@ -53,6 +53,13 @@ class aif_weights(C.Structure):
     ]
 
 
+class aif_item_weights(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("dI", C.c_int32), ("hI", C.c_int32), ("d_mm", C.c_int32), ("W_i0", C.c_void_p),
+        ("b_i0", C.c_void_p), ("W_i1", C.c_void_p), ("b_i1", C.c_void_p), ("bridges", C.c_void_p), ("W_hash", C.c_void_p),
+    ]
+
+
 class aif_user_inputs(C.Structure):
     _fields_ = [
         ("struct_size", C.c_uint32), ("mode", C.c_int32), ("profile", C.c_void_p), ("seq", C.c_void_p),
@@ -73,8 +80,9 @@ class aif_stats(C.Structure):
 # every symbol include/aif.h declares
 EXPORTS = [
     "aif_input_width", "aif_mix64", "aif_create", "aif_destroy", "aif_load_weights", "aif_item_nearline_refresh",
+    "aif_load_item_weights", "aif_item_nearline_compute",
     "aif_user_precompute", "aif_user_release", "aif_user_request_key", "aif_user_state_export", "aif_score",
-    "aif_score_batch", "aif_score_host", "aif_score_noalloc", "aif_gather_rows", "aif_poll_status", "aif_get_stats",
+    "aif_score_batch", "aif_score_host", "aif_score_noalloc", "aif_gather_rows", "aif_gather_sidecars", "aif_poll_status", "aif_get_stats",
     "aif_set_kernel_timing", "aif_get_kernel_timing", "aif_kernel_launches", "aif_selftest_bounded_wait", "aif_strerror", "aif_last_error",
 ]
 
@@ -97,6 +105,8 @@ def load_library(path: Optional[str] = None):
     lib.aif_destroy.argtypes = [vp]
     lib.aif_load_weights.argtypes = [vp, C.POINTER(aif_weights), vp]
     lib.aif_item_nearline_refresh.argtypes = [vp, vp, i64, vp, vp, vp, vp]
+    lib.aif_load_item_weights.argtypes = [vp, C.POINTER(aif_item_weights), vp]
+    lib.aif_item_nearline_compute.argtypes = [vp, vp, i64, vp, vp, vp, vp]
     lib.aif_user_precompute.argtypes = [vp, u64, C.POINTER(aif_user_inputs), i32, C.POINTER(vp), vp]
     lib.aif_user_release.argtypes = [vp, vp]
     lib.aif_user_request_key.argtypes, lib.aif_user_request_key.restype = [vp], u64
@@ -106,6 +116,7 @@ def load_library(path: Optional[str] = None):
     lib.aif_score_host.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.aif_score_noalloc.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.aif_gather_rows.argtypes = [vp, vp, i64, vp, vp]
+    lib.aif_gather_sidecars.argtypes = [vp, vp, i64, vp, vp, vp]
     lib.aif_poll_status.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.aif_get_stats.argtypes = [vp, C.POINTER(aif_stats)]
     lib.aif_set_kernel_timing.argtypes = [vp, C.c_int]
@@ -251,8 +262,29 @@ class Aif:
         _check(self.lib.aif_item_nearline_refresh(self.h, _ptr(ids), n, _ptr(rows), _ptr(bea_w), _ptr(lsh_sig),
                                                   _stream(stream)), "aif_item_nearline_refresh")
 
+    def load_item_weights(self, w: dict, stream=None):
+        """w: device tensors "W_i0" [hI x dI], "b_i0", "W_i1" [d x hI], "b_i1" and, for their blocks, "bridges"
+        [n_bridge x d], "W_hash" [lsh_bits x d_mm] (weights in storage type, biases fp32)."""
+        iw = aif_item_weights()
+        iw.struct_size = C.sizeof(aif_item_weights)
+        iw.hI, iw.dI = w["W_i0"].shape
+        iw.d_mm = w["W_hash"].shape[1] if w.get("W_hash") is not None else 0
+        for name in ("W_i0", "b_i0", "W_i1", "b_i1", "bridges", "W_hash"):
+            if w.get(name) is not None:
+                setattr(iw, name, w[name].data_ptr())
+        _check(self.lib.aif_load_item_weights(self.h, C.byref(iw), _stream(stream)), "aif_load_item_weights")
+        self._item_weights_keep = w
+
+    def item_nearline_compute(self, ids: Optional[torch.Tensor], I_raw: torch.Tensor, I_id=None, M_mm=None, stream=None):
+        _check(self.lib.aif_item_nearline_compute(self.h, _ptr(ids), I_raw.shape[0], _ptr(I_raw), _ptr(I_id), _ptr(M_mm),
+                                                  _stream(stream)), "aif_item_nearline_compute")
+
     def gather_rows(self, ids: torch.Tensor, out: torch.Tensor, stream=None):
         _check(self.lib.aif_gather_rows(self.h, _ptr(ids), ids.numel(), _ptr(out), _stream(stream)), "aif_gather_rows")
+
+    def gather_sidecars(self, ids: torch.Tensor, bea_w_out=None, sig_out=None, stream=None):
+        _check(self.lib.aif_gather_sidecars(self.h, _ptr(ids), ids.numel(), _ptr(bea_w_out), _ptr(sig_out), _stream(stream)),
+               "aif_gather_sidecars")
 
     # -- user side -------------------------------------------------------------------------------
     def user_precompute(self, request_key: int, *, mode: int, profile: torch.Tensor, seq: torch.Tensor,

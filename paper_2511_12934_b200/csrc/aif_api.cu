@@ -310,6 +310,7 @@ int aif_destroy(aif_ctx *ctx)
         if (ctx->ring.ev[i]) cudaEventDestroy(ctx->ring.ev[i]);
     }
     if (ctx->tc_plan) tc_destroy_context(ctx);
+    if (ctx->nearline_plan) nearline_destroy(ctx);
     for (void *p : ctx->allocations) cudaFree(p);
     cudaGetLastError();
     delete ctx;
@@ -361,6 +362,31 @@ int aif_item_nearline_refresh(aif_ctx *ctx, const int32_t *ids, int64_t n, const
     if (n == 0) return AIF_OK;
     DeviceGuard g(ctx->device);
     AIF_CUDA(launch_scatter_rows(ctx, ids, n, rows, bea_w, lsh_sig, as_stream(stream)));
+    ctx->table_version += 1;
+    ctx->stats.table_version = ctx->table_version;
+    ctx->stats.refresh_calls += 1;
+    ctx->stats.rows_refreshed += (uint64_t)n;
+    return AIF_OK;
+}
+
+int aif_load_item_weights(aif_ctx *ctx, const aif_item_weights *w, aif_stream stream)
+{
+    if (!ctx || !w || w->struct_size != sizeof(aif_item_weights)) return AIF_ERR_ARG;
+    DeviceGuard g(ctx->device);
+    return nearline_load_weights(ctx, w, as_stream(stream));
+}
+
+int aif_item_nearline_compute(aif_ctx *ctx, const int32_t *ids, int64_t n, const void *I_raw, const void *I_id, const void *M_mm,
+                              aif_stream stream)
+{
+    if (!ctx || !I_raw || n < 0) return AIF_ERR_ARG;
+    if (ctx->sig && !M_mm) return AIF_ERR_ARG;
+    if (!ids && n > ctx->cfg.M) return AIF_ERR_SHAPE;
+    if (!ctx->nearline_plan) return AIF_ERR_NOT_READY;
+    if (n == 0) return AIF_OK;
+    DeviceGuard g(ctx->device);
+    const int rc = nearline_compute(ctx, ids, n, I_raw, I_id, M_mm, as_stream(stream));
+    if (rc != AIF_OK) return rc;
     ctx->table_version += 1;
     ctx->stats.table_version = ctx->table_version;
     ctx->stats.refresh_calls += 1;
@@ -558,6 +584,19 @@ int aif_gather_rows(aif_ctx *ctx, const int32_t *ids, int64_t n, void *rows_out,
     if (!ids || !rows_out) return AIF_ERR_ARG;
     DeviceGuard g(ctx->device);
     AIF_CUDA(launch_gather_rows(ctx, ids, n, rows_out, as_stream(stream)));
+    return AIF_OK;
+}
+
+int aif_gather_sidecars(aif_ctx *ctx, const int32_t *ids, int64_t n, void *bea_w_out, uint8_t *sig_out, aif_stream stream)
+{
+    if (!ctx || n < 0) return AIF_ERR_ARG;
+    if ((bea_w_out && !ctx->bea_w) || (sig_out && !ctx->sig)) return AIF_ERR_ARG;
+    if (bea_w_out && ((size_t)ctx->cfg.n_bridge * ctx->el) % 4 != 0) return AIF_ERR_SHAPE;
+    if (sig_out && ctx->cfg.lsh_bits % 32 != 0) return AIF_ERR_SHAPE;
+    if (n == 0 || (!bea_w_out && !sig_out)) return AIF_OK;
+    if (!ids) return AIF_ERR_ARG;
+    DeviceGuard g(ctx->device);
+    AIF_CUDA(launch_gather_sidecars(ctx, ids, n, bea_w_out, sig_out, as_stream(stream)));
     return AIF_OK;
 }
 

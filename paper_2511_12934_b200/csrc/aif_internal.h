@@ -148,6 +148,7 @@ struct aif_ctx {
     float *logits_stage = nullptr;
     void *tc_plan = nullptr;          // tensor-core path: packed weights, tensor maps, activation scratch
     void *tc_att_plan = nullptr;      // tensor-core attention: tensor map over the arena's S regions
+    void *nearline_plan = nullptr;    // item-side weights and scratch of aif_item_nearline_compute
     void *tc_fused_plan = nullptr;    // single-launch scoring: the second layer's bias split into two bf16 rows
     aif::PinnedRing ring;
 
@@ -172,6 +173,7 @@ cudaError_t launch_scatter_rows(const aif_ctx *ctx, const int32_t *ids, int64_t 
                                 const uint8_t *sig, cudaStream_t st);
 cudaError_t launch_stage_ids(const int32_t *mapped_src, int32_t *dst, int n, cudaStream_t st);
 cudaError_t launch_gather_rows(const aif_ctx *ctx, const int32_t *ids, int64_t n, void *out, cudaStream_t st);
+cudaError_t launch_gather_sidecars(const aif_ctx *ctx, const int32_t *ids, int64_t n, void *bea_w_out, uint8_t *sig_out, cudaStream_t st);
 cudaError_t launch_transpose(const void *in, void *out, int rows, int cols, size_t el, cudaStream_t st);
 cudaError_t launch_score_simt(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st);
 cudaError_t launch_user_network(const aif_ctx *ctx, HostSlot &hs, int slot_index, const aif_user_inputs *in, int L,
@@ -209,6 +211,24 @@ struct TcScratch {
 size_t tc_scratch_row_bytes(const aif_ctx *ctx);
 void tc_scratch_layout(const aif_ctx *ctx, void *base, size_t rows, TcScratch *out);
 cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, const TcScratch &sc);
+// One dense layer on the tensor cores (aif_tc.cu): out [rows x H] bf16 = act(A [rows x in_w] W^T + bias), or, with
+// sign_bits, out [rows x H / 8] bytes = packed signs of A W^T.  in_w a multiple of 64; H <= 256 and a multiple of 32, or a
+// multiple of 256.  W [H x in_w] bf16 row-major.
+struct DenseLayer {
+    const void *A;
+    const void *W;
+    const float *bias;   // [H]
+    void *out;
+    int32_t in_w, H;
+    int32_t relu;        // 0: linear output
+    int32_t sign_bits;
+};
+cudaError_t tc_dense_layer(const aif_ctx *ctx, const DenseLayer &L, int64_t rows, cudaStream_t st);
+// item side of the nearline pipeline (aif_nearline.cu)
+int nearline_load_weights(aif_ctx *ctx, const aif_item_weights *w, cudaStream_t st);
+int nearline_compute(aif_ctx *ctx, const int32_t *ids, int64_t n, const void *I_raw, const void *I_id, const void *M_mm,
+                     cudaStream_t st);
+void nearline_destroy(aif_ctx *ctx);
 // host-side checks shared by the scoring entry points (aif_api.cu)
 int check_user_state(aif_ctx *ctx, const aif_user_state *st);
 void set_last_error(const char *text);

@@ -124,6 +124,40 @@ cudaError_t launch_gather_rows(const aif_ctx *ctx, const int32_t *ids, int64_t n
     return cudaGetLastError();
 }
 
+// out[i] = table[ids[i]] for narrow rows (BEA weights, signatures): one thread per 4 bytes.
+__global__ void __launch_bounds__(256) k_gather_words(const uint32_t *__restrict__ table, const int32_t *__restrict__ ids, int64_t n,
+                                                      int words_per_row, int64_t M, uint32_t *__restrict__ out, uint32_t *status)
+{
+    const int64_t total = n * words_per_row;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / words_per_row;
+        const int c = (int)(i - r * words_per_row);
+        const int64_t src = ids[r];
+        uint32_t v = 0u;
+        if (src >= 0 && src < M) v = __ldg(table + src * words_per_row + c);
+        else if (c == 0) atomicOr(status, AIF_STATUS_BAD_ID);
+        out[i] = v;
+    }
+}
+
+cudaError_t launch_gather_sidecars(const aif_ctx *ctx, const int32_t *ids, int64_t n, void *bea_w_out, uint8_t *sig_out, cudaStream_t st)
+{
+    const aif_config &c = ctx->cfg;
+    if (bea_w_out) {
+        const int words = (int)((size_t)c.n_bridge * ctx->el / 4);
+        k_gather_words<<<grid_for(n * words, 256, 148 * 16), 256, 0, st>>>((const uint32_t *)ctx->bea_w, ids, n, words, c.M,
+                                                                           (uint32_t *)bea_w_out, ctx->status);
+        count_launch();
+    }
+    if (sig_out) {
+        const int words = c.lsh_bits / 32;
+        k_gather_words<<<grid_for(n * words, 256, 148 * 16), 256, 0, st>>>((const uint32_t *)ctx->sig, ids, n, words, c.M,
+                                                                           (uint32_t *)sig_out, ctx->status);
+        count_launch();
+    }
+    return cudaGetLastError();
+}
+
 template <typename T>
 __global__ void k_transpose(const T *__restrict__ in, T *__restrict__ out, int rows, int cols)
 {

@@ -32,7 +32,7 @@ constexpr int kMaxChunks = 64;
 constexpr int kFusedMaxTiles = 148;
 
 enum { SRC_ITEM = 0, SRC_DENSE = 1, SRC_CROSS = 2 };
-enum { EPI_STORE = 0, EPI_DOT = 1 };
+enum { EPI_STORE = 0, EPI_DOT = 1, EPI_SIGN = 2 };
 
 struct ChunkSrc {
     int32_t kind;
@@ -53,6 +53,8 @@ struct LayerParams {
     int32_t check_ids;            // first layer: flag ids outside the table
     // epilogue
     int32_t epi, bias_from_slot, emit_sigmoid, out_stride;
+    int32_t linear_out;           // EPI_STORE without the ReLU (output layer of the item-side tower)
+    uint8_t *sig_out;             // EPI_SIGN: [positions x out_stride / 8] packed sign bits of the outputs
     const float *bias;
     __nv_bfloat16 *out;           // EPI_STORE: [positions x out_stride]
     const __nv_bfloat16 *w_out;
@@ -216,21 +218,30 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
             const bool valid = row < t.cnt;
             const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(buf * 256);
             float dot = 0.f;
+            const float floor_v = p.linear_out ? -INFINITY : 0.f;
             if (t.cnt > 0) {
                 for (int c0 = 0; c0 < p.n_cols; c0 += 32) {
                     uint32_t r[32];
                     tmem_ld32(taddr + (uint32_t)c0, r);
                     tmem_ld_wait();
                     const float4 *b4 = reinterpret_cast<const float4 *>(bs + c0);
-                    if (p.epi == EPI_STORE) {
+                    if (p.epi == EPI_SIGN) {
+                        // eq. 5: one bit per output, set where the projection is positive; eight bits per byte, first bit
+                        // most significant
+                        uint32_t word = 0u;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            word |= (__uint_as_float(r[i]) > 0.f ? 1u : 0u) << (8 * (i >> 3) + 7 - (i & 7));
+                        if (valid) *reinterpret_cast<uint32_t *>(p.sig_out + (size_t)(t.pos0 + row) * (p.out_stride >> 3) + ((n0 + c0) >> 3)) = word;
+                    } else if (p.epi == EPI_STORE) {
                         uint32_t packed[16];
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
                             const float4 bb = b4[q];
-                            const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q]) + bb.x, 0.f),
-                                                                            fmaxf(__uint_as_float(r[4 * q + 1]) + bb.y, 0.f));
-                            const __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q + 2]) + bb.z, 0.f),
-                                                                            fmaxf(__uint_as_float(r[4 * q + 3]) + bb.w, 0.f));
+                            const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q]) + bb.x, floor_v),
+                                                                            fmaxf(__uint_as_float(r[4 * q + 1]) + bb.y, floor_v));
+                            const __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q + 2]) + bb.z, floor_v),
+                                                                            fmaxf(__uint_as_float(r[4 * q + 3]) + bb.w, floor_v));
                             packed[2 * q] = *reinterpret_cast<const uint32_t *>(&h0);
                             packed[2 * q + 1] = *reinterpret_cast<const uint32_t *>(&h1);
                         }
@@ -369,7 +380,7 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
             R.xb = p.xb + (size_t)(t.pos0 + r0) * p.F;
             int id = -1;
             if (lp < t.cnt) {   // this thread fetches the id of row lp; the others read it from shared memory
-                id = p.sl.ids[t.pos0 + lp];
+                id = p.sl.ids ? p.sl.ids[t.pos0 + lp] : 0;   // no id array: a launch over dense rows only
                 if (id < 0 || (int64_t)id >= p.M) {
                     id = -1;
                     if (p.check_ids) atomicOr(p.sl.status, AIF_STATUS_BAD_ID);
@@ -813,6 +824,67 @@ void tc_scratch_layout(const aif_ctx *ctx, void *base, size_t rows, TcScratch *o
     }
     out->xb = (c.blocks & AIF_BLK_CROSS) ? p : nullptr;
     out->rows = rows;
+}
+
+// One dense layer over `rows` consecutive rows of a row-major bf16 matrix, with the layer kernel: out = act(A W^T + b)
+// (bf16), or the packed sign bits of A W^T.  Used by the item side of the nearline pipeline.
+cudaError_t tc_dense_layer(const aif_ctx *ctx, const DenseLayer &L, int64_t rows, cudaStream_t st)
+{
+    if (rows <= 0) return cudaSuccess;
+    EncodeFn enc = encode_fn();
+    if (!enc) return cudaErrorNotSupported;
+    LayerParams p{};
+    p.sl.slots = ctx->slots_dev, p.sl.reqs = nullptr, p.sl.n_req = 1;
+    p.sl.single = ReqDev{0, (int32_t)rows, 0, 0, 0};
+    p.sl.n_tiles = (int32_t)((rows + kTcTile - 1) / kTcTile), p.sl.total = rows, p.sl.max_L = 0;
+    p.sl.ids = nullptr, p.sl.logits = nullptr, p.sl.status = ctx->status;
+    p.n_cols = L.H <= 256 ? L.H : 256, p.n_nchunks = L.H / p.n_cols, p.n_k = L.in_w / 64, p.mini_batch = 0;
+    p.E = (const uint8_t *)ctx->E, p.M = ctx->cfg.M, p.e_row_bytes = ctx->cfg.d * 2;
+    p.X = (const uint8_t *)L.A, p.x_row_bytes = L.in_w * 2;
+    p.B = 1, p.dc = 8, p.F = 0, p.xb = nullptr, p.check_ids = 0;
+    for (int i = 0; i < p.n_k; ++i) p.src[i].kind = SRC_DENSE, p.src[i].off = i * 128;
+    p.epi = L.sign_bits ? EPI_SIGN : EPI_STORE;
+    p.bias_from_slot = 0, p.bias = L.bias, p.emit_sigmoid = 0, p.linear_out = L.relu ? 0 : 1;
+    p.out = (__nv_bfloat16 *)L.out, p.out_stride = L.H, p.sig_out = (uint8_t *)L.out;
+    p.w_out = nullptr, p.b_out = nullptr;
+    const cuuint32_t estr[2] = {1, 1};
+    CUtensorMap tmap_b, tmap_a, tmap_out;
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)L.in_w, (cuuint64_t)L.H};
+        const cuuint64_t strides[1] = {(cuuint64_t)L.in_w * 2};
+        const cuuint32_t box[2] = {64, (cuuint32_t)p.n_cols};
+        if (enc(&tmap_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(L.W), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)L.in_w, (cuuint64_t)rows};
+        const cuuint64_t strides[1] = {(cuuint64_t)L.in_w * 2};
+        const cuuint32_t box[2] = {64, 128};
+        if (enc(&tmap_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(L.A), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    tmap_out = tmap_b;
+    if (!L.sign_bits) {
+        const cuuint64_t dims[2] = {(cuuint64_t)L.H, (cuuint64_t)rows};
+        const cuuint64_t strides[1] = {(cuuint64_t)L.H * 2};
+        const cuuint32_t box[2] = {32, 32};
+        if (enc(&tmap_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L.out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    const int single = p.sl.n_tiles * p.n_nchunks;
+    const bool pair = ((p.sl.n_tiles + 1) / 2) * p.n_nchunks >= 2 * 148;
+    const bool wide = !pair && p.n_nchunks % 2 == 0 && single > 148;
+    const int items = pair ? ((p.sl.n_tiles + 1) / 2) * p.n_nchunks : wide ? single / 2 : single;
+    const int grid = items < 148 ? items : 148;
+    cudaError_t e;
+    if (pair) e = launch_pdl(k_layer_tc<1>, dim3(grid), dim3(LayerCfg<1>::kThreads), LayerCfg<1>::kSmem, st, tmap_b, tmap_out, tmap_a, p);
+    else if (wide) e = launch_pdl(k_layer_tc<2>, dim3(grid), dim3(LayerCfg<2>::kThreads), LayerCfg<2>::kSmem, st, tmap_b, tmap_out, tmap_a, p);
+    else e = launch_pdl(k_layer_tc<0>, dim3(grid), dim3(LayerCfg<0>::kThreads), LayerCfg<0>::kSmem, st, tmap_b, tmap_out, tmap_a, p);
+    count_launch();
+    return e;
 }
 
 cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t, cudaStream_t st)

@@ -209,6 +209,27 @@ def make_item_table(wl: Workload, rows: Optional[int] = None) -> dict:
     return tab
 
 
+def make_item_side(wl: Workload, n: int, dI: Optional[int] = None, hI: Optional[int] = None, d_mm: Optional[int] = None) -> dict:
+    """Inputs and weights of the item side of the nearline pipeline for n items: raw features I_raw [n x dI] (dI = 4 d by
+    default: the paper reports item-side compression of more than 3x), id embeddings I_id [n x d], multi-modal
+    embeddings M_mm [n x d_mm]; tower weights (Glorot uniform, small biases), bridges B [n_bridge x d] ~ N(0, 1) (so that
+    the softmax over bridges is not flat), W_hash [lsh_bits x d_mm] ~ N(0, 1) in storage type."""
+    t = _tag(wl.name)
+    dI, hI, d_mm = dI or 4 * wl.d, hI or 2 * wl.d, d_mm or wl.d
+    out = {
+        "I_raw": normal_rows(n, dI, wl.sigma, wl.dtype, t, 400),
+        "I_id": normal_rows(n, wl.d, 1.0, wl.dtype, t, 401),
+        "M_mm": normal_rows(n, d_mm, 1.0, wl.dtype, t, 402),
+        "W_i0": glorot_uniform(hI, dI, wl.dtype, t, 410),
+        "W_i1": glorot_uniform(wl.d, hI, wl.dtype, t, 411),
+        "b_i0": (_seed(t, 412).standard_normal(hI) * 0.05).astype(np.float32),
+        "b_i1": (_seed(t, 413).standard_normal(wl.d) * 0.05).astype(np.float32),
+        "bridges": normal_rows(max(wl.n_bridge, 1), wl.d, 1.0, wl.dtype, t, 414),
+        "W_hash": normal_rows(max(wl.lsh_bits, 8), d_mm, 1.0, wl.dtype, t, 415),
+    }
+    return out
+
+
 class IdSampler:
     """Candidate ids: distinct within a request; uniform, or Zipf(s) ranks mapped through a fixed random
     permutation of the rows; an optional pool shared by all requests gives cross-request overlap."""
