@@ -360,6 +360,32 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
         states[-1] = stx
         pre_ms = float(np.median(ts[1:]))
 
+    # the item side of the nearline pipeline as a compute call (eq. 4 tower; bridge weights and signatures when their
+    # blocks are on): 2^19 synthetic items with dI = 4 d, hI = 2 d written into the table rows they will be gathered from
+    nearline = None
+    if full and rank == 0 and not wl.blocks & (synth.BLK_BEA | synth.BLK_LSH_DIN | synth.BLK_SIMTIER):
+        nn = int(min(1 << 19, table["E"].shape[0]))
+        it = synth.make_item_side(wl, nn)
+        bdt = B.F32 if wl.dtype == "f32" else B.BF16
+        dev_it = {k: (torch.from_numpy(v).cuda() if v.dtype == np.float32 else B.to_device(v, bdt)) for k, v in it.items()}
+        saved = torch.empty(nn, wl.d, dtype=torch.float32 if wl.dtype == "f32" else torch.bfloat16, device="cuda")
+        srv.ctx.gather_rows(torch.arange(nn, dtype=torch.int32, device="cuda"), saved)   # the table is put back afterwards
+        srv.ctx.load_item_weights(dev_it)
+
+        def nearline_step(i):
+            srv.ctx.item_nearline_compute(None, dev_it["I_raw"], dev_it["I_id"], dev_it["M_mm"])
+
+        nearline_step(0)
+        n_ms = float(np.median(timed(5, nearline_step)))
+        dI, hI = it["W_i0"].shape[1], it["W_i0"].shape[0]
+        n_flops = 2.0 * (dI * hI + hI * wl.d)
+        el = 4 if wl.dtype == "f32" else 2
+        nearline = {"items": nn, "dI": dI, "hI": hI, "ms": n_ms, "items_per_s": nn / (n_ms * 1e-3),
+                    "tflops": nn * n_flops / (n_ms * 1e-3) / 1e12, "gbs": nn * (dI + wl.d) * el / (n_ms * 1e-3) / 1e9,
+                    "note": "tower flops and (raw row in + item vector out) bytes only; the hidden activations pass through HBM"}
+        srv.ctx.item_nearline_refresh(None, saved)
+        del dev_it, saved
+
     peaks, peak_kind = load_peaks()
     gather = {"rows": gn, "row_bytes": row_bytes, "ms": g_ms, "achieved": gn * (2 * row_bytes + 4) / (g_ms * 1e-3) / 1e9,
               "peak": float(peaks["hbm_gbs"]), "unit": "GB/s", "bound": "hbm", "peak_kind": f"copy bandwidth, {peak_kind}",
@@ -400,6 +426,7 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
         "clocks": clocks,
         "roofline": roof,
         "gather_stage": gather,
+        "nearline_item_side": nearline,
         "user_precompute": {"ms": pre_ms, "inputs": "raw embeddings (eqs. 1-3 computed)", "L": wl.L, "stream": "side"},
         "replica_plan": plan,
     }
