@@ -277,6 +277,25 @@ def test_single_launch_scoring_at_the_sequence_lengths_around_its_key_blocks(L):
     srv.close()
 
 
+@pytest.mark.parametrize("H2,F,dc,Bk,mode,sig", [(64, 2, 32, 1024, synth.BUCKET_HASH, 0), (128, 8, 8, 1000, synth.BUCKET_HASH, 1),
+                                                  (192, 12, 16, 1024, synth.BUCKET_MOD, 0), (256, 8, 64, 37, synth.BUCKET_MOD, 1),
+                                                  (256, 24, 16, 512, synth.BUCKET_HASH, 0)])
+def test_single_launch_scoring_over_the_shapes_it_accepts(H2, F, dc, Bk, mode, sig):
+    """Second-layer widths 64..256, one to eight cross-feature chunks of 64 columns, cross embeddings of 8..64 columns
+    (eight fields to one field per chunk), bucket counts that are and are not powers of two, both bucket functions, with and
+    without the final sigmoid; non-zero biases, which this kernel adds on the tensor cores."""
+    wl = helpers.MINI["c2"].with_(name=f"fused_{H2}_{F}_{dc}", R=1, N=300, L=150, mini_batch=0, hidden=(512, H2), F=F, dc=dc,
+                                  B=Bk, bucket_mode=mode, emit_sigmoid=sig)
+    weights, table, srv, oracle = _setup(wl, zero_bias=False)
+    rq = synth.make_request(wl, 0)
+    ids = synth.IdSampler(wl).request_ids(0)
+    st = srv.precompute(3, srv.upload_request(rq, B.USER_PROJECTED))
+    want = oracle.score(table, helpers.projected_request(wl, rq), ids)
+    _check_logits(srv.score_ids(st, ids), want, TOL["bf16"])
+    assert srv.ctx.poll_status() == 0
+    srv.close()
+
+
 @pytest.mark.parametrize("name", ["c3", "c4", "c5", "c5b"])
 def test_full_size_batches_on_sampled_candidates(name):
     """The multi-request shapes at their full sizes, scored in one aif_score_batch call exactly as the benchmark
