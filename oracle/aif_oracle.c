@@ -300,6 +300,35 @@ void orc_item_nearline(int dtype, int64_t n, int dI, int hI, int d, const void *
     }
 }
 
+/* Algorithm 1 steps 1-2, user side: W = Softmax(B U^T / sqrt(d)) [n x m] (one softmax per bridge over the m user-side
+ * feature embeddings), then V = f(U, W | Theta_u) [n x d].  Reading of f (the paper leaves the network open): one linear
+ * layer on the attention-weighted features, V_k = W_f (sum_j W_kj U_j).  bridges [n x d], U [m x d], W_f [d x d] in
+ * storage type; V_out [n x d], W_out [n x m] (may be NULL) in double. */
+void orc_bea_user(int dtype, int n, int m, int d, const void *bridges, const void *U, const void *W_f, double *V_out, double *W_out)
+{
+    double *w = (double *)malloc(sizeof(double) * (size_t)(m + d));
+    double *a = w + m;
+    for (int k = 0; k < n; ++k) {
+        double mx = -INFINITY, den = 0.0;
+        for (int j = 0; j < m; ++j) {
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c) acc += ld(bridges, (int64_t)k * d + c, dtype) * ld(U, (int64_t)j * d + c, dtype);
+            w[j] = acc / sqrt((double)d);
+            if (w[j] > mx) mx = w[j];
+        }
+        for (int j = 0; j < m; ++j) den += exp(w[j] - mx);
+        for (int j = 0; j < m; ++j) w[j] = exp(w[j] - mx) / den;
+        if (W_out)
+            for (int j = 0; j < m; ++j) W_out[(int64_t)k * m + j] = w[j];
+        for (int c = 0; c < d; ++c) {
+            a[c] = 0.0;
+            for (int j = 0; j < m; ++j) a[c] += w[j] * ld(U, (int64_t)j * d + c, dtype);
+        }
+        linear(W_f, dtype, NULL, d, d, a, V_out + (int64_t)k * d);
+    }
+    free(w);
+}
+
 /* The projections behind eq. 5's bits, for tests that need to know how close to zero a bit was decided. */
 void orc_lsh_projections(int dtype, int64_t n, int d_mm, int dbits, const void *M_mm, const void *W_hash, double *proj)
 {

@@ -233,6 +233,17 @@ def item_nearline(dtype: int, I_raw=None, W0=None, b0=None, W1=None, b1=None, I_
     return out
 
 
+def bea_user(dtype: int, bridges: np.ndarray, U: np.ndarray, W_f: np.ndarray):
+    """Algorithm 1 steps 1-2: returns (V [n x d], W [n x m]) in float64; inputs in storage type."""
+    bridges, U, W_f = _store(bridges, dtype), _store(U, dtype), _store(W_f, dtype)
+    n, d = bridges.shape
+    m = U.shape[0]
+    assert U.shape == (m, d) and W_f.shape == (d, d)
+    V, W = np.zeros((n, d)), np.zeros((n, m))
+    lib().orc_bea_user(C.c_int(dtype), C.c_int(n), C.c_int(m), C.c_int(d), _p(bridges), _p(U), _p(W_f), _p(V), _p(W))
+    return V, W
+
+
 def lsh_projections(dtype: int, M_mm: np.ndarray, W_hash: np.ndarray) -> np.ndarray:
     """The projections M W_hash^T [n x dbits] whose signs eq. 5 keeps."""
     M_mm, W_hash = _store(M_mm, dtype), _store(W_hash, dtype)

@@ -582,3 +582,41 @@ def test_item_signatures_pack_eq5_bits_first_bit_most_significant():
     both = orc.item_nearline(orc.F32, M_mm=np.vstack([M[:1], -M[:1]]), W_hash=W)["sig"]
     sim = orc.lsh_similarity(both[:1], both, dbits)
     assert sim[0, 0] == 1.0 and sim[0, 1] == 0.0
+
+
+def test_bea_user_side_and_the_whole_of_algorithm_1():
+    g = np.random.default_rng(14)
+    n, m, d, b = 4, 6, 8, 5
+    Bm = g.standard_normal((n, d)).astype(np.float32)
+    U = g.standard_normal((m, d)).astype(np.float32)
+    Wf = g.standard_normal((d, d)).astype(np.float32)
+    V, W = orc.bea_user(orc.F32, Bm, U, Wf)
+    # step 1: one softmax per bridge over the user-side features (rows of B against rows of U)
+    assert W.shape == (n, m) and np.allclose(W.sum(axis=1), 1.0, atol=1e-14) and (W > 0).all()
+    s = Bm.astype(np.float64) @ U.astype(np.float64).T / math.sqrt(d)
+    e = np.exp(s - s.max(axis=1, keepdims=True))
+    assert np.allclose(W, e / e.sum(axis=1, keepdims=True), atol=1e-14)
+    # step 2 under the reading V_k = W_f (sum_j W_kj U_j): brute force with scalar loops
+    for k in range(n):
+        a = [sum(W[k, j] * float(U[j, c]) for j in range(m)) for c in range(d)]
+        for r in range(d):
+            assert abs(V[k, r] - sum(float(Wf[r, c]) * a[c] for c in range(d))) < 1e-12
+    # one user-side feature: every bridge sees weight 1, V_k = W_f U_0 for every k
+    V1, W1 = orc.bea_user(orc.F32, Bm, U[:1], Wf)
+    assert np.array_equal(W1, np.ones((n, 1)))
+    assert np.allclose(V1, np.tile(Wf.astype(np.float64) @ U[0].astype(np.float64), (n, 1)), atol=1e-13)
+    # identity W_f: V_k is a convex combination of the rows of U; a bridge far along one feature picks that feature
+    Vi, _ = orc.bea_user(orc.F32, Bm, U, np.eye(d, dtype=np.float32))
+    assert (Vi <= U.max(axis=0) + 1e-12).all() and (Vi >= U.min(axis=0) - 1e-12).all()
+    Bs = Bm.copy(); Bs[2] = 60.0 * U[4]
+    Vs, Ws = orc.bea_user(orc.F32, Bs, U, np.eye(d, dtype=np.float32))
+    assert Ws[2, 4] > 0.999 and np.allclose(Vs[2], U[4], atol=1e-2)
+    # the whole algorithm: v^ = Softmax(I B^T / sqrt d) V, composed from the item-side and user-side oracles
+    I = g.standard_normal((b, d)).astype(np.float32)
+    w_hat = orc.item_nearline(orc.F32, I_id=I, bridges=Bm)["w_hat"]
+    for i in range(b):
+        assert np.allclose(orc.bea(w_hat[i], V), w_hat[i] @ V, atol=1e-13)
+    # with a single bridge the approximation collapses to the same vector for every item
+    V0, _ = orc.bea_user(orc.F32, Bm[:1], U, Wf)
+    w0 = orc.item_nearline(orc.F32, I_id=I, bridges=Bm[:1])["w_hat"]
+    assert np.array_equal(w0, np.ones((b, 1))) and np.allclose(orc.bea(w0[3], V0), V0[0], atol=0)
