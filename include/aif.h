@@ -120,6 +120,9 @@ typedef struct {
     const float *b_a;      /* fp32 [d] */
     const void *W_b;       /* [d x d] */
     const float *b_b;      /* fp32 [d] */
+    /* user side of Algorithm 1 (steps 1-2); may be NULL when every caller supplies bea_V itself */
+    const void *bridges;   /* B [n_bridge x d] */
+    const void *W_f;       /* [d x d]: V_k = W_f (sum_j W_kj U_j), this library's reading of f(U, W | Theta_u) */
 } aif_weights;
 
 /* Device pointers to one user's inputs, storage type unless stated. */
@@ -131,9 +134,13 @@ typedef struct {
     const void *profile;
     const void *seq;
     const void *cross_raw;   /* [F x B x dc] user-side part of the cross features; NULL if block off */
-    const void *bea_V;       /* [n_bridge x d] user-side BEA vectors (Algorithm 1, line 2); NULL if block off */
+    const void *bea_V;       /* [n_bridge x d] user-side BEA vectors (Algorithm 1, step 2), computed elsewhere; NULL if
+                                the block is off or bea_U is given instead */
     const uint8_t *seq_sig;  /* [L x lsh_bits/8] packed signatures of the sequence items, first bit = MSB of
                                 byte 0 (Section 4.2); NULL if both LSH blocks are off */
+    const void *bea_U;       /* [bea_m x d] user-side feature embeddings U of Algorithm 1: with bea_V == NULL the call
+                                computes W = Softmax(B U^T / sqrt(d)) and V from them (needs bridges and W_f) */
+    int32_t bea_m;           /* 1 <= bea_m <= 1024 */
 } aif_user_inputs;
 
 typedef struct {
@@ -291,6 +298,10 @@ int aif_gather_rows(aif_ctx *ctx, const int32_t *ids, int64_t n, void *rows_out,
  * (device [n x n_bridge] storage type), sig_out[i] = the signature (device [n x lsh_bits/8]) of item ids[i]; a NULL
  * output is skipped, an output whose block is off is AIF_ERR_ARG.  Bad ids give zero rows and the status bit. */
 int aif_gather_sidecars(aif_ctx *ctx, const int32_t *ids, int64_t n, void *bea_w_out, uint8_t *sig_out, aif_stream stream);
+
+/* Copies the user-side BEA vectors V [n_bridge x d] (storage type) of a state to V_out (device), ordered after the
+ * state's user-side call.  AIF_ERR_ARG when the BEA block is off. */
+int aif_user_state_export_bea(aif_ctx *ctx, const aif_user_state *state, void *V_out, aif_stream stream);
 
 /* Reads and clears the device status word (synchronises the device).  bits: host. */
 int aif_poll_status(aif_ctx *ctx, uint32_t *bits);

@@ -49,7 +49,7 @@ class aif_weights(C.Structure):
     _fields_ = [
         ("struct_size", C.c_uint32), ("W", C.c_void_p * 4), ("b", C.c_void_p * 4), ("w_out", C.c_void_p),
         ("b_out", C.c_void_p), ("W_profile", C.c_void_p), ("W_seq", C.c_void_p), ("W_a", C.c_void_p),
-        ("b_a", C.c_void_p), ("W_b", C.c_void_p), ("b_b", C.c_void_p),
+        ("b_a", C.c_void_p), ("W_b", C.c_void_p), ("b_b", C.c_void_p), ("bridges", C.c_void_p), ("W_f", C.c_void_p),
     ]
 
 
@@ -63,7 +63,7 @@ class aif_item_weights(C.Structure):
 class aif_user_inputs(C.Structure):
     _fields_ = [
         ("struct_size", C.c_uint32), ("mode", C.c_int32), ("profile", C.c_void_p), ("seq", C.c_void_p),
-        ("cross_raw", C.c_void_p), ("bea_V", C.c_void_p), ("seq_sig", C.c_void_p),
+        ("cross_raw", C.c_void_p), ("bea_V", C.c_void_p), ("seq_sig", C.c_void_p), ("bea_U", C.c_void_p), ("bea_m", C.c_int32),
     ]
 
 
@@ -81,7 +81,7 @@ class aif_stats(C.Structure):
 EXPORTS = [
     "aif_input_width", "aif_mix64", "aif_create", "aif_destroy", "aif_load_weights", "aif_item_nearline_refresh",
     "aif_load_item_weights", "aif_item_nearline_compute",
-    "aif_user_precompute", "aif_user_release", "aif_user_request_key", "aif_user_state_export", "aif_score",
+    "aif_user_precompute", "aif_user_release", "aif_user_request_key", "aif_user_state_export", "aif_user_state_export_bea", "aif_score",
     "aif_score_batch", "aif_score_host", "aif_score_noalloc", "aif_gather_rows", "aif_gather_sidecars", "aif_poll_status", "aif_get_stats",
     "aif_set_kernel_timing", "aif_get_kernel_timing", "aif_kernel_launches", "aif_selftest_bounded_wait", "aif_strerror", "aif_last_error",
 ]
@@ -111,6 +111,7 @@ def load_library(path: Optional[str] = None):
     lib.aif_user_release.argtypes = [vp, vp]
     lib.aif_user_request_key.argtypes, lib.aif_user_request_key.restype = [vp], u64
     lib.aif_user_state_export.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.aif_user_state_export_bea.argtypes = [vp, vp, vp, vp]
     lib.aif_score.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.aif_score_batch.argtypes = [vp, i32, C.POINTER(vp), vp, C.POINTER(i64), vp, vp]
     lib.aif_score_host.argtypes = [vp, vp, vp, i32, vp, vp]
@@ -237,8 +238,9 @@ class Aif:
             w.b[k] = mlp["b"][k].data_ptr()
         w.w_out, w.b_out = mlp["w_out"].data_ptr(), mlp["b_out"].data_ptr()
         if user is not None:
-            for name in ("W_profile", "W_seq", "W_a", "b_a", "W_b", "b_b"):
-                setattr(w, name, user[name].data_ptr())
+            for name in ("W_profile", "W_seq", "W_a", "b_a", "W_b", "b_b", "bridges", "W_f"):
+                if user.get(name) is not None:
+                    setattr(w, name, user[name].data_ptr())
         _check(self.lib.aif_load_weights(self.h, C.byref(w), _stream(stream)), "aif_load_weights")
         self._weights_keep = (mlp, user)
 
@@ -251,7 +253,7 @@ class Aif:
         du = None
         if weights.get("user") is not None:
             u = weights["user"]
-            du = {k: (to_device(v, dt) if k.startswith("W") else torch.from_numpy(v).cuda()) for k, v in u.items()}
+            du = {k: (torch.from_numpy(v).cuda() if k.startswith("b_") else to_device(v, dt)) for k, v in u.items()}
         self.load_weights(dm, du)
         torch.cuda.current_stream().synchronize()
 
@@ -282,21 +284,27 @@ class Aif:
     def gather_rows(self, ids: torch.Tensor, out: torch.Tensor, stream=None):
         _check(self.lib.aif_gather_rows(self.h, _ptr(ids), ids.numel(), _ptr(out), _stream(stream)), "aif_gather_rows")
 
+    def user_state_export_bea(self, state: "UserState", stream=None) -> torch.Tensor:
+        V = torch.empty(self.cfg.n_bridge, self.cfg.d, dtype=self.torch_dtype, device="cuda")
+        _check(self.lib.aif_user_state_export_bea(self.h, state.handle, _ptr(V), _stream(stream)), "aif_user_state_export_bea")
+        return V
+
     def gather_sidecars(self, ids: torch.Tensor, bea_w_out=None, sig_out=None, stream=None):
         _check(self.lib.aif_gather_sidecars(self.h, _ptr(ids), ids.numel(), _ptr(bea_w_out), _ptr(sig_out), _stream(stream)),
                "aif_gather_sidecars")
 
     # -- user side -------------------------------------------------------------------------------
     def user_precompute(self, request_key: int, *, mode: int, profile: torch.Tensor, seq: torch.Tensor,
-                        cross_raw=None, bea_V=None, seq_sig=None, stream=None) -> UserState:
+                        cross_raw=None, bea_V=None, seq_sig=None, bea_U=None, stream=None) -> UserState:
         inp = aif_user_inputs(C.sizeof(aif_user_inputs), mode, profile.data_ptr(), seq.data_ptr(),
                               None if cross_raw is None else cross_raw.data_ptr(),
                               None if bea_V is None else bea_V.data_ptr(),
-                              None if seq_sig is None else seq_sig.data_ptr())
+                              None if seq_sig is None else seq_sig.data_ptr(),
+                              None if bea_U is None else bea_U.data_ptr(), 0 if bea_U is None else bea_U.shape[0])
         out = C.c_void_p()
         _check(self.lib.aif_user_precompute(self.h, request_key, C.byref(inp), seq.shape[0], C.byref(out),
                                             _stream(stream)), "aif_user_precompute")
-        return UserState(self, out.value, (profile, seq, cross_raw, bea_V, seq_sig))
+        return UserState(self, out.value, (profile, seq, cross_raw, bea_V, seq_sig, bea_U))
 
     def user_state_export(self, state: UserState, L: int, stream=None):
         u = torch.empty(self.cfg.d, dtype=torch.float32, device="cuda")

@@ -344,6 +344,17 @@ int aif_load_weights(aif_ctx *ctx, const aif_weights *w, aif_stream stream)
         AIF_CUDA(cudaMemcpyAsync(ctx->b_a, w->b_a, (size_t)c.d * 4, cudaMemcpyDeviceToDevice, st));
         AIF_CUDA(cudaMemcpyAsync(ctx->b_b, w->b_b, (size_t)c.d * 4, cudaMemcpyDeviceToDevice, st));
     }
+    ctx->bea_user_weights = false;
+    if ((c.blocks & AIF_BLK_BEA) && w->bridges && w->W_f) {
+        if (!ctx->bridges) {
+            int rc = dev_alloc(ctx, &ctx->bridges, (size_t)c.n_bridge * c.d * el, true);
+            if (rc == AIF_OK) rc = dev_alloc(ctx, &ctx->W_f, (size_t)c.d * c.d * el, true);
+            if (rc != AIF_OK) return rc;
+        }
+        AIF_CUDA(cudaMemcpyAsync(ctx->bridges, w->bridges, (size_t)c.n_bridge * c.d * el, cudaMemcpyDeviceToDevice, st));
+        AIF_CUDA(cudaMemcpyAsync(ctx->W_f, w->W_f, (size_t)c.d * c.d * el, cudaMemcpyDeviceToDevice, st));
+        ctx->bea_user_weights = true;
+    }
     if (ctx->tensor_path) AIF_CUDA(tc_prepare_weights(ctx, w, st));
     if (ctx->tensor_path && ctx->tc_fused_plan) AIF_CUDA(tc_fused_prepare_weights(ctx, st));
     ctx->weights_loaded = true;
@@ -406,7 +417,11 @@ int aif_user_precompute(aif_ctx *ctx, uint64_t request_key, const aif_user_input
     if (L < 1 || L > c.L_max) return AIF_ERR_SHAPE;
     if (!in->profile || !in->seq) return AIF_ERR_ARG;
     if ((c.blocks & AIF_BLK_CROSS) && !in->cross_raw) return AIF_ERR_ARG;
-    if ((c.blocks & AIF_BLK_BEA) && !in->bea_V) return AIF_ERR_ARG;
+    if ((c.blocks & AIF_BLK_BEA) && !in->bea_V) {
+        if (!in->bea_U) return AIF_ERR_ARG;
+        if (in->bea_m < 1 || in->bea_m > 1024) return AIF_ERR_SHAPE;
+        if (!ctx->bea_user_weights) return AIF_ERR_NOT_READY;
+    }
     if ((c.blocks & (AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER)) && !in->seq_sig) return AIF_ERR_ARG;
     int idx = -1;
     for (int i = 0; i < (int)ctx->slots.size(); ++i)
@@ -477,6 +492,19 @@ static cudaError_t wait_user_ready(const HostSlot &hs, cudaStream_t st)
     if (q != cudaErrorNotReady) return q;
     (void)cudaGetLastError();   // "not ready" is an answer, not a failure: keep it out of later launch checks
     return cudaStreamWaitEvent(st, hs.ev, 0);
+}
+
+int aif_user_state_export_bea(aif_ctx *ctx, const aif_user_state *state, void *V_out, aif_stream stream)
+{
+    int rc = state_check(ctx, state);
+    if (rc != AIF_OK) return rc;
+    if (!(ctx->cfg.blocks & AIF_BLK_BEA) || !V_out) return AIF_ERR_ARG;
+    DeviceGuard g(ctx->device);
+    const HostSlot &hs = ctx->slots[(size_t)state->index];
+    cudaStream_t st = as_stream(stream);
+    AIF_CUDA(cudaStreamWaitEvent(st, hs.ev, 0));
+    AIF_CUDA(cudaMemcpyAsync(V_out, hs.dev.V, (size_t)ctx->cfg.n_bridge * ctx->cfg.d * ctx->el, cudaMemcpyDeviceToDevice, st));
+    return AIF_OK;
 }
 
 int aif_score(aif_ctx *ctx, const aif_user_state *state, const int32_t *cand_ids, int32_t n, float *logits, aif_stream stream)

@@ -135,6 +135,8 @@ struct aif_ctx {
     void *Wprofile_t = nullptr, *Wseq_t = nullptr, *Wa_t = nullptr, *Wb_t = nullptr;
     float *b_a = nullptr, *b_b = nullptr;
     bool user_weights = false;
+    void *bridges = nullptr, *W_f = nullptr;   // user side of Algorithm 1: B [n_bridge x d], W_f [d x d]
+    bool bea_user_weights = false;
 
     char *arena = nullptr;
     size_t slot_bytes = 0;

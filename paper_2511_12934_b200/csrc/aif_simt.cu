@@ -609,6 +609,49 @@ static cudaError_t user_network_typed(const aif_ctx *ctx, HostSlot &hs, int slot
     return cudaGetLastError();
 }
 
+// Algorithm 1 steps 1-2 for one user, one block: W = Softmax(B U^T / sqrt(d)) per bridge, A_k = sum_j W_kj U_j,
+// V_k = W_f A_k.  Shared memory: W [n x m] and A [n x d] in fp32.
+template <typename T>
+__global__ void __launch_bounds__(256) k_bea_user(const T *__restrict__ Bm, const T *__restrict__ U, const T *__restrict__ Wf, int n, int m,
+                                                  int d, T *__restrict__ V)
+{
+    extern __shared__ float sm_bea[];
+    float *W = sm_bea, *A = sm_bea + n * m;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float scale = rsqrtf((float)d);
+    for (int p = warp; p < n * m; p += 8) {   // one warp per (bridge, feature) pair
+        const int k = p / m, j = p - k * m;
+        float acc = 0.f;
+        for (int c = lane; c < d; c += 32) acc = fmaf(to_f(Bm[(size_t)k * d + c]), to_f(U[(size_t)j * d + c]), acc);
+        acc = warp_sum(acc);
+        if (lane == 0) W[p] = acc * scale;
+    }
+    __syncthreads();
+    for (int k = warp; k < n; k += 8) {       // one warp per bridge: softmax over the m features
+        float mx = -INFINITY;
+        for (int j = lane; j < m; j += 32) mx = fmaxf(mx, W[k * m + j]);
+        mx = warp_max(mx);
+        float den = 0.f;
+        for (int j = lane; j < m; j += 32) den += expf(W[k * m + j] - mx);
+        den = warp_sum(den);
+        for (int j = lane; j < m; j += 32) W[k * m + j] = expf(W[k * m + j] - mx) / den;
+    }
+    __syncthreads();
+    for (int p = tid; p < n * d; p += 256) {
+        const int k = p / d, c = p - k * d;
+        float acc = 0.f;
+        for (int j = 0; j < m; ++j) acc = fmaf(W[k * m + j], to_f(U[(size_t)j * d + c]), acc);
+        A[p] = acc;
+    }
+    __syncthreads();
+    for (int p = tid; p < n * d; p += 256) {
+        const int k = p / d, r = p - k * d;
+        float acc = 0.f;
+        for (int c = 0; c < d; ++c) acc = fmaf(to_f(Wf[(size_t)r * d + c]), A[k * d + c], acc);
+        from_f(V[p], acc);
+    }
+}
+
 cudaError_t launch_user_network(const aif_ctx *ctx, HostSlot &hs, int slot_index, const aif_user_inputs *in, int L,
                                 cudaStream_t st)
 {
@@ -618,9 +661,20 @@ cudaError_t launch_user_network(const aif_ctx *ctx, HostSlot &hs, int slot_index
         e = cudaMemcpyAsync((void *)hs.dev.T, in->cross_raw, (size_t)c.F * c.B * c.dc * ctx->el, cudaMemcpyDeviceToDevice, st);
         if (e != cudaSuccess) return e;
     }
-    if (c.blocks & AIF_BLK_BEA) {
+    if ((c.blocks & AIF_BLK_BEA) && in->bea_V) {
         e = cudaMemcpyAsync((void *)hs.dev.V, in->bea_V, (size_t)c.n_bridge * c.d * ctx->el, cudaMemcpyDeviceToDevice, st);
         if (e != cudaSuccess) return e;
+    } else if (c.blocks & AIF_BLK_BEA) {
+        const size_t smem = (size_t)(c.n_bridge * in->bea_m + c.n_bridge * c.d) * 4;
+        if (c.dtype == AIF_F32)
+            k_bea_user<float><<<1, 256, smem, st>>>((const float *)ctx->bridges, (const float *)in->bea_U, (const float *)ctx->W_f, c.n_bridge,
+                                                    in->bea_m, c.d, (float *)hs.dev.V);
+        else
+            k_bea_user<__nv_bfloat16><<<1, 256, smem, st>>>((const __nv_bfloat16 *)ctx->bridges, (const __nv_bfloat16 *)in->bea_U,
+                                                            (const __nv_bfloat16 *)ctx->W_f, c.n_bridge, in->bea_m, c.d,
+                                                            (__nv_bfloat16 *)hs.dev.V);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     if (c.blocks & (AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER)) {
         e = cudaMemcpyAsync((void *)hs.dev.sigS, in->seq_sig, (size_t)L * (c.lsh_bits / 8), cudaMemcpyDeviceToDevice, st);

@@ -59,6 +59,7 @@ class Server:
             dev["profile"], dev["seq"] = B.to_device(rq["u"], self.dt), B.to_device(rq["S"], self.dt)
         dev["cross_raw"] = B.to_device(rq["T"], self.dt) if "T" in rq else None
         dev["bea_V"] = B.to_device(rq["V"], self.dt) if "V" in rq else None
+        dev["bea_U"] = B.to_device(rq["bea_U"], self.dt) if "bea_U" in rq else None   # Algorithm 1's U: V is computed
         dev["seq_sig"] = torch.from_numpy(np.ascontiguousarray(rq["sig_seq"])).cuda() if "sig_seq" in rq else None
         return dev
 
@@ -66,7 +67,7 @@ class Server:
         """aif_user_precompute on the side stream (or `stream`)."""
         return self.ctx.user_precompute(key, mode=dev["mode"], profile=dev["profile"], seq=dev["seq"],
                                         cross_raw=dev["cross_raw"], bea_V=dev["bea_V"], seq_sig=dev["seq_sig"],
-                                        stream=stream or self.side)
+                                        bea_U=dev.get("bea_U"), stream=stream or self.side)
 
     def score_ids(self, state: B.UserState, ids: np.ndarray) -> np.ndarray:
         ids_t = torch.from_numpy(np.ascontiguousarray(ids, dtype=np.int32)).cuda()

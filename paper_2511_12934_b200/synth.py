@@ -176,6 +176,9 @@ def make_weights(wl: Workload, zero_bias: bool = True) -> dict:
         "b_a": np.zeros(d, dtype=np.float32) if zero_bias else (_seed(t, 204).standard_normal(d) * 0.05).astype(np.float32),
         "b_b": np.zeros(d, dtype=np.float32) if zero_bias else (_seed(t, 205).standard_normal(d) * 0.05).astype(np.float32),
     }
+    if wl.blocks & BLK_BEA:   # user side of Algorithm 1: bridges B ~ N(0, 1) (a softmax that is not flat), W_f Glorot
+        user["bridges"] = normal_rows(wl.n_bridge, d, 1.0, wl.dtype, t, 414)
+        user["W_f"] = glorot_uniform(d, d, wl.dtype, t, 206)
     return {"mlp": {"W": W, "b": b, "w_out": w_out, "b_out": b_out}, "user": user}
 
 

@@ -37,8 +37,9 @@ def test_every_declared_symbol_is_exported(lib):
 def test_struct_layouts_match_the_header(lib):
     # sizes follow from the header's field lists under the C ABI (natural alignment)
     assert C.sizeof(B.aif_config) == 112
-    assert C.sizeof(B.aif_weights) == 8 + 4 * 8 + 4 * 8 + 8 * 8
-    assert C.sizeof(B.aif_user_inputs) == 8 + 5 * 8
+    assert C.sizeof(B.aif_weights) == 8 + 4 * 8 + 4 * 8 + 10 * 8
+    assert C.sizeof(B.aif_user_inputs) == 8 + 6 * 8 + 8
+    assert C.sizeof(B.aif_item_weights) == 16 + 6 * 8
     cfg = B.make_config(dtype=B.BF16, M=1000, d=128, L_max=10, hidden=(512, 256), F=16, B=1024, dc=32)
     assert lib.aif_input_width(C.byref(cfg)) == 128 * 3 + 16 * 32
     assert synth.C2.input_width() == 896 and synth.C1.input_width() == 320 and synth.C5.input_width() == 2816

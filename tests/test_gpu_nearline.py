@@ -132,3 +132,40 @@ def test_nearline_call_errors():
         srv.ctx.load_item_weights(bad)
     assert e.value.code == B.ERR_SHAPE
     srv.close()
+
+
+@pytest.mark.parametrize("name,m", [("c1", 5), ("c2", 37)])
+def test_user_side_of_algorithm_1_is_computed_when_only_U_is_given(name, m):
+    """aif_user_precompute with bea_U instead of bea_V: W = Softmax(B U^T / sqrt(d)), V_k = W_f (sum_j W_kj U_j) on the GPU,
+    against the oracle; then scoring with the BEA block on, where the item-side weights meet these vectors (step 4)."""
+    wl = helpers.MINI[name].with_(name=f"bea_user_{name}", blocks=helpers.ALL_BLOCKS, N=200, L=40,
+                                  lsh_din_norm=synth.NORM_MEAN, simtier_norm=synth.NORM_MEAN, emit_sigmoid=0)
+    weights = synth.make_weights(wl)
+    table = synth.make_item_table(wl)
+    srv = serving.Server(wl, weights, table)
+    dt = orc.F32 if wl.dtype == "f32" else orc.BF16
+    rq = synth.make_request(wl, 0)
+    U = synth.normal_rows(m, wl.d, 1.0, wl.dtype, 77, m)
+    V_want, _ = orc.bea_user(dt, weights["user"]["bridges"], U, weights["user"]["W_f"])
+    rq_gpu = dict(rq, bea_U=U)
+    del rq_gpu["V"]
+    st = srv.precompute(9, srv.upload_request(rq_gpu, B.USER_PROJECTED))
+    V_got = srv.ctx.user_state_export_bea(st)
+    torch.cuda.synchronize()
+    V_got = V_got.float().cpu().numpy().astype(np.float64)
+    rtol, atol = (1e-5, 1e-6) if wl.dtype == "f32" else (2.0 ** -8, 1e-4)
+    assert np.allclose(V_got, V_want, rtol=rtol, atol=atol), np.abs(V_got - V_want).max()
+    # scoring: the oracle gets the vectors the GPU stored (exact inputs), so the usual logit tolerance applies
+    stored = V_got.astype(np.float32) if wl.dtype == "f32" else synth.to_bf16_bits(V_got.astype(np.float32))
+    oracle = helpers.make_oracle(wl, weights, M=table["E"].shape[0])
+    ids = synth.IdSampler(wl).request_ids(0)
+    want = oracle.score(table, helpers.projected_request(wl, dict(rq, V=stored)), ids)
+    got = srv.score_ids(st, ids)
+    assert np.abs(got - want).max() <= (1e-5 if wl.dtype == "f32" else 2e-3)
+    # neither V nor U: refused
+    rq_none = dict(rq)
+    del rq_none["V"]
+    with pytest.raises(B.AifError) as e:
+        srv.precompute(10, srv.upload_request(rq_none, B.USER_PROJECTED))
+    assert e.value.code == B.ERR_ARG
+    srv.close()
