@@ -55,6 +55,16 @@ struct ModelDev {
     const float *b_out;
 };
 
+// One 128-candidate tile of a launch over several requests, looked up once per launch (k_tile_table) so that no kernel
+// role has to search the request table per tile.
+struct TileDev {
+    int32_t slot;
+    int32_t cnt;     // candidates in the tile
+    int64_t pos0;    // position of its first candidate in ids / logits
+    int32_t L;       // sequence length of the tile's request
+    int32_t pad_[3];
+};
+
 struct ScoreLaunch {
     const SlotDev *slots;   // device array of all slots
     const ReqDev *reqs;     // device array [n_req], or nullptr: use `single`
@@ -66,6 +76,7 @@ struct ScoreLaunch {
     const int32_t *ids;
     float *logits;
     uint32_t *status;
+    const TileDev *tiles;   // [n_tiles] (tensor-core tiles), or nullptr: search `reqs` per tile
 };
 
 struct HostSlot {
@@ -208,6 +219,7 @@ struct TcScratch {
     void *X;               // dense interaction columns, [rows x x_cols] bf16
     void *H[kMaxHidden];   // activations after hidden layer k (k < last), [rows x hidden[k]] bf16
     void *xb;              // cross-feature buckets, [rows x F] uint16
+    void *tiles;           // tile table, [rows / 128 + requests] TileDev, or nullptr
     size_t rows;           // rows every array has room for
 };
 size_t tc_scratch_row_bytes(const aif_ctx *ctx);

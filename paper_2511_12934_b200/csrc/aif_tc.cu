@@ -106,6 +106,13 @@ __device__ __forceinline__ TileInfo decode_tile(const LayerParams &p, int tile)
         t.start = 0, t.cnt = 0, t.pos0 = 0;
         return t;
     }
+    if (p.sl.tiles) {   // looked up once per launch
+        const int4 v = *reinterpret_cast<const int4 *>(p.sl.tiles + tile);   // slot, cnt, pos0
+        t.rq = ReqDev{v.x, 0, 0, 0, 0};
+        t.start = 0, t.cnt = v.y;
+        t.pos0 = ((int64_t)(uint32_t)v.w << 32) | (int64_t)(uint32_t)v.z;
+        return t;
+    }
     t.rq = find_request(p.sl, tile);
     tile_range(tile - t.rq.tile_begin, t.rq.n, kTcTile, p.mini_batch, t.start, t.cnt);
     t.pos0 = t.rq.off + t.start;
@@ -136,6 +143,24 @@ __global__ void __launch_bounds__(256) k_cross_buckets(const int32_t *__restrict
         }
         xb[i] = (uint16_t)bk;
     }
+}
+
+// Tile table of a launch over several requests: one thread per tile does the search of the request table that every
+// role of every kernel would otherwise repeat per tile (a chain of dependent loads on the critical path of the MMA
+// issuers).
+__global__ void __launch_bounds__(256) k_tile_table(ScoreLaunch sl, int mini_batch, TileDev *__restrict__ out)
+{
+    grid_dep_launch();
+    grid_dep_wait();
+    const int tile = blockIdx.x * blockDim.x + threadIdx.x;
+    if (tile >= sl.n_tiles) return;
+    const ReqDev rq = find_request(sl, tile);
+    int start, cnt;
+    tile_range(tile - rq.tile_begin, rq.n, kTcTile, mini_batch, start, cnt);
+    TileDev t;
+    t.slot = rq.slot, t.cnt = cnt, t.pos0 = rq.off + start, t.L = sl.slots[rq.slot].L;
+    t.pad_[0] = t.pad_[1] = t.pad_[2] = 0;
+    out[tile] = t;
 }
 
 // ---- the layer kernel -----------------------------------------------------------------------------------------
@@ -647,6 +672,7 @@ struct TcPlan {
     __nv_bfloat16 *H[kMaxHidden] = {};   // activations after layer k (k < last)
     __nv_bfloat16 *X = nullptr;
     uint16_t *xb = nullptr;              // cross-feature buckets [positions x F]
+    TileDev *tiles = nullptr;            // tile table of a launch over several requests
     bool maps_ready = false;
 };
 
@@ -739,6 +765,7 @@ cudaError_t tc_prepare_context(aif_ctx *ctx)
     }
     if (pl->x_cols && (e = alloc((void **)&pl->X, cap * pl->x_cols * 2)) != cudaSuccess) return e;
     if ((c.blocks & AIF_BLK_CROSS) && (e = alloc((void **)&pl->xb, cap * c.F * 2)) != cudaSuccess) return e;
+    if ((e = alloc((void **)&pl->tiles, (cap / kTcTile + (size_t)c.max_user_states * 8 + 64) * sizeof(TileDev))) != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_layer_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LayerCfg<0>::kSmem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_layer_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LayerCfg<1>::kSmem);
@@ -823,6 +850,7 @@ void tc_scratch_layout(const aif_ctx *ctx, void *base, size_t rows, TcScratch *o
         }
     }
     out->xb = (c.blocks & AIF_BLK_CROSS) ? p : nullptr;
+    out->tiles = nullptr;
     out->rows = rows;
 }
 
@@ -893,14 +921,17 @@ cudaError_t launch_score_tc(const aif_ctx *ctx, const ScoreLaunch &sl, int64_t, 
     TcScratch sc;
     sc.X = pl->X;
     sc.xb = pl->xb;
+    sc.tiles = pl->tiles;
     sc.rows = pl->cap_rows;
     for (int k = 0; k < kMaxHidden; ++k) sc.H[k] = pl->H[k];
     return launch_score_tc_scratch(ctx, sl, st, sc);
 }
 
-cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, const TcScratch &sc)
+cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl_in, cudaStream_t st, const TcScratch &sc)
 {
-    if (sl.n_tiles <= 0) return cudaSuccess;
+    if (sl_in.n_tiles <= 0) return cudaSuccess;
+    ScoreLaunch sl = sl_in;
+    sl.tiles = nullptr;
     const aif_config &c = ctx->cfg;
     TcPlan *pl = plan_of(ctx);
     const ModelDev md = make_model(ctx);
@@ -910,6 +941,12 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl, c
         cudaError_t e = launch_request_fused(ctx, sl, st);
         timing_mark(ctx, "score_fused", st);
         return e;
+    }
+    if (sl.reqs && sc.tiles) {   // several requests: look every tile up once
+        cudaError_t e = launch_pdl(k_tile_table, dim3((sl.n_tiles + 255) / 256), dim3(256), 0, st, sl, c.mini_batch, (TileDev *)sc.tiles);
+        count_launch();
+        if (e != cudaSuccess) return e;
+        sl.tiles = (const TileDev *)sc.tiles;
     }
     if (c.blocks & AIF_BLK_CROSS) {
         const int64_t n = sl.total * c.F;

@@ -51,19 +51,28 @@ struct AttCfg {
 
 // One tile of the launch as every role needs it.
 struct AttTile {
-    int slot, cnt, nb;
+    int slot, cnt, nb, L;
     int64_t pos0;
 };
 
 template <int BN>
 __device__ __forceinline__ AttTile att_tile(const AttParams &p, int tile)
 {
+    AttTile t;
+    if (p.sl.tiles) {   // looked up once per launch (k_tile_table)
+        const int4 v = *reinterpret_cast<const int4 *>(p.sl.tiles + tile);   // slot, cnt, pos0
+        t.slot = v.x, t.cnt = v.y;
+        t.pos0 = ((int64_t)(uint32_t)v.w << 32) | (int64_t)(uint32_t)v.z;
+        t.L = p.sl.tiles[tile].L;
+        t.nb = (t.L + BN - 1) / BN;
+        return t;
+    }
     const ReqDev rq = find_request(p.sl, tile);
     int start, cnt;
     tile_range(tile - rq.tile_begin, rq.n, kTcTile, p.mini_batch, start, cnt);
-    AttTile t;
     t.slot = rq.slot, t.cnt = cnt, t.pos0 = rq.off + start;
-    t.nb = (p.sl.slots[rq.slot].L + BN - 1) / BN;
+    t.L = p.sl.slots[rq.slot].L;
+    t.nb = (t.L + BN - 1) / BN;
     return t;
 }
 
@@ -143,7 +152,7 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
         }
         for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++k) {
             const AttTile t = att_tile<BN>(p, tile);
-            const int L = p.sl.slots[t.slot].L;
+            const int L = t.L;
             float m_used = -INFINITY, l_sum = 0.f;
             for (int j = 0; j < t.nb; ++j, ++gb) {
                 const int b = (int)(gb & 1u);
@@ -272,9 +281,12 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
             struct Cursor {
                 int tile, k, j, nb;
                 uint32_t gb;
+                int nb_next;   // key blocks of the tile after this one, fetched a whole tile ahead of its use
             };
+            auto blocks_of = [&](int tile) { return tile < n_tiles ? att_tile<BN>(p, tile).nb : 0; };
             auto open_tile = [&](Cursor &c) {
-                if (c.tile < n_tiles) c.nb = att_tile<BN>(p, c.tile).nb;
+                c.nb = c.nb_next;
+                c.nb_next = blocks_of(c.tile + (int)gridDim.x);
             };
             auto advance = [&](Cursor &c) {
                 ++c.gb;
@@ -286,9 +298,10 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
             // operand descriptors of buffer / stage 0; the others lie a fixed number of 16-byte units further
             const uint64_t qdesc0 = umma_desc_sw128(smem_u32(smQ)), kdesc0 = umma_desc_sw128(smem_u32(smKV));
             const uint64_t vdesc0 = umma_desc_mn_sw128(smem_u32(smKV), C::kKvChunkBytes);
-            Cursor cq{(int)blockIdx.x, 0, 0, 0, 0u}, cp{(int)blockIdx.x, 0, 0, 0, 0u};
+            Cursor cq{(int)blockIdx.x, 0, 0, 0, 0u, 0}, cp{(int)blockIdx.x, 0, 0, 0, 0u, 0};
+            cq.nb_next = blocks_of(cq.tile);
             open_tile(cq);
-            cp.nb = cq.nb;
+            cp.nb = cq.nb, cp.nb_next = cq.nb_next;
             auto issue_qk = [&]() -> bool {
                 const int qb = cq.k % kQB;
                 if (cq.j == 0) {   // first block of a tile: its queries must have landed (cp.async, generic proxy)
@@ -465,7 +478,7 @@ __global__ void __launch_bounds__(kAtt2Threads, 1) k_att_tc_long(const __grid_co
     grid_dep_launch();
     grid_dep_wait();
     const AttTile t = att_tile<BN>(p, blockIdx.x);
-    const int L = p.sl.slots[t.slot].L, nb = t.nb;
+    const int L = t.L, nb = t.nb;
 
     if (warp < kAtt2MmaWarp) {
         // ===================== queries, softmax, output =====================
