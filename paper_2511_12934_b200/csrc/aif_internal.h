@@ -204,7 +204,7 @@ void tc_att_destroy(aif_ctx *ctx);
 // eq. 2's attention rows softmax(S S^T / sqrt(d)) S of one user state with the same kernel (queries = the sequence rows);
 // *rows_out: [L x d] bf16 in scratch of the attention plan, valid until the next call
 cudaError_t launch_self_att_tc(const aif_ctx *ctx, int slot_index, int L, cudaStream_t st, const void **rows_out);
-cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, void *X, int x_stride);
+cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, void *X, int x_stride, size_t x_rows);
 // whole scoring pass of a tile in one CTA (aif_tc_fused.cu); the tensor maps it shares with the other kernels
 bool tc_fused_supported(const aif_config &cfg);
 cudaError_t tc_fused_prepare(aif_ctx *ctx);

@@ -959,7 +959,7 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl_in
     }
     const bool att_tc = ctx->tc_att_plan != nullptr;
     if (att_tc) {
-        cudaError_t e = launch_att_tc(ctx, sl, st, sc.X, pl->x_cols);
+        cudaError_t e = launch_att_tc(ctx, sl, st, sc.X, pl->x_cols, sc.rows);
         timing_mark(ctx, "attention", st);
         if (e != cudaSuccess) return e;
     }

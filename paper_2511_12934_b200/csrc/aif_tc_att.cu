@@ -77,7 +77,8 @@ __device__ __forceinline__ AttTile att_tile(const AttParams &p, int tile)
 }
 
 template <int D, int BN>
-__global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant__ CUtensorMap tmapS, const AttParams p)
+__global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant__ CUtensorMap tmapS,
+                                                           const __grid_constant__ CUtensorMap tmapX, const AttParams p)
 {
     using C = AttCfg<D, BN>;
     constexpr int kS = C::kKvStages, kQB = C::kQBufs;
@@ -104,7 +105,7 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
             mbar_init(smem_u32(p_full + b), 128);
             mbar_init(smem_u32(pv_done + b), 1);
             mbar_init(smem_u32(q_full + b), 32);
-            mbar_init(smem_u32(q_empty + b), 1);
+            mbar_init(smem_u32(q_empty + b), 5);   // the last Q K^T of the tenant, and the four softmax warps' output staging
         }
         mbar_init(smem_u32(o_final), 1);
         mbar_init(smem_u32(o_free), 128);
@@ -247,30 +248,67 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                 const int id = p.sl.ids[t.pos0 + row];
                 good = id >= 0 && (int64_t)id < p.M;
             }
-#pragma unroll 1
-            for (int c0 = 0; c0 < D; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(lane_base + (uint32_t)(C::kTmemO + c0), r);
-                tmem_ld_wait();
-                if (c0 + 32 == D) {   // O is in registers: the next tile's first P V may overwrite the accumulator
-                    tc_fence_before();
-                    mbar_arrive(smem_u32(o_free));
-                }
-                if (row < t.cnt) {
-                    uint32_t packed[16];
+            // Output rows leave through shared memory and asynchronous tile stores: a thread owns a row, so direct stores
+            // are 32 scattered half-used sectors per instruction, which cost several thousand cycles per tile.  The
+            // staging slabs (2 x 2 KB per warp, 64-byte swizzle) live in the tile's own query buffer: every Q K^T of the
+            // tile is complete, and the gather of the buffer's next tenant waits for these warps as well.
+            const int qb_out = k % kQB;
+            unsigned char *stg = smQ + qb_out * C::kQBytes + warp * 4096;
+            const bool whole = warp * 32 + 32 <= t.cnt;   // ragged last tiles keep the guarded direct stores
+            uint32_t slab = 0;
+            auto emit = [&](const uint32_t (&r)[32], int c0) {
+                uint32_t packed[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(good ? __uint_as_float(r[2 * i]) * inv : 0.f,
-                                                                       good ? __uint_as_float(r[2 * i + 1]) * inv : 0.f);
-                        packed[i] = *reinterpret_cast<const uint32_t *>(&h);
+                for (int i = 0; i < 16; ++i) {
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(good ? __uint_as_float(r[2 * i]) * inv : 0.f,
+                                                                   good ? __uint_as_float(r[2 * i + 1]) * inv : 0.f);
+                    packed[i] = *reinterpret_cast<const uint32_t *>(&h);
+                }
+                if (whole) {
+                    unsigned char *sb = stg + slab * 2048;
+                    if (lane == 0) bulk_wait_read<1>();   // the store that last read this slab is done with it
+                    __syncwarp();
+                    const int swz = (lane >> 1) & 3;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        *reinterpret_cast<uint4 *>(sb + lane * 64 + ((q ^ swz) << 4)) =
+                            make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tmapX, smem_u32(sb), c0, (int)(t.pos0 + warp * 32));
+                        bulk_commit();
                     }
+                    slab ^= 1u;
+                } else if (row < t.cnt) {
                     uint4 *dst = reinterpret_cast<uint4 *>(p.X + (size_t)(t.pos0 + row) * p.x_stride + c0);
 #pragma unroll
                     for (int q = 0; q < 4; ++q)
                         dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
                 }
+            };
+            // two chunks of 32 columns per round; the load of the next chunk is in flight while one is converted and staged
+            uint32_t ra[32], rb[32];
+            tmem_ld32(lane_base + (uint32_t)C::kTmemO, ra);
+#pragma unroll 1
+            for (int c0 = 0; c0 < D; c0 += 64) {
+                tmem_ld_wait();
+                tmem_ld32(lane_base + (uint32_t)(C::kTmemO + c0 + 32), rb);
+                emit(ra, c0);
+                tmem_ld_wait();
+                if (c0 + 64 < D) tmem_ld32(lane_base + (uint32_t)(C::kTmemO + c0 + 64), ra);
+                else {   // O is in registers: the next tile's first P V may overwrite the accumulator
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(o_free));
+                }
+                emit(rb, c0 + 32);
+            }
+            if (lane == 0) {
+                bulk_wait_read<0>();   // the staging is no longer read: the query buffer may take its next tenant
+                mbar_arrive(smem_u32(q_empty + qb_out));
             }
         }
+        if (lane == 0) bulk_wait<0>();   // all tile stores of this warp have reached global memory
     } else if (warp == kAttMmaWarp) {
         // ===================== MMA issuer =====================
         if (lane == 0) {
@@ -792,10 +830,25 @@ int tc_att_key_block(const aif_ctx *ctx)
     return pl ? pl->bn : 0;
 }
 
-cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, void *X, int x_stride)
+// Store target of the attention rows: X as a [rows x x_stride] bf16 tensor, 32 x 32 boxes, 64-byte swizzle.
+static cudaError_t encode_x_map(CUtensorMap *m, void *X, int x_stride, size_t rows)
+{
+    const cuuint64_t dims[2] = {(cuuint64_t)x_stride, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)x_stride * 2};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                             CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, void *X, int x_stride, size_t x_rows)
 {
     const aif_config &c = ctx->cfg;
     const AttPlan *pl = reinterpret_cast<const AttPlan *>(ctx->tc_att_plan);
+    CUtensorMap tmap_x;
+    cudaError_t ex = encode_x_map(&tmap_x, X, x_stride, x_rows);
+    if (ex != cudaSuccess) return ex;
     AttParams p{};
     p.sl = sl, p.E = (const uint8_t *)ctx->E, p.M = c.M, p.mini_batch = c.mini_batch;
     p.x_stride = x_stride, p.X = (__nv_bfloat16 *)X;
@@ -808,9 +861,9 @@ cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
     if (c.d == 128 && grid == sl.n_tiles && sl.max_L >= 16 * 128)   // one CTA per tile and many key blocks per tile
         e = launch_pdl(k_att_tc_long, dim3(grid), dim3(kAtt2Threads), kAtt2Smem, st, pl->tmap, p);
     else if (c.d == 128)
-        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(kAttThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, p);
+        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(kAttThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, tmap_x, p);
     else
-        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(kAttThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, p);
+        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(kAttThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, tmap_x, p);
     count_launch();
     return e;
 }
@@ -828,14 +881,17 @@ cudaError_t launch_self_att_tc(const aif_ctx *ctx, int slot_index, int L, cudaSt
     p.sl = sl, p.E = reinterpret_cast<const uint8_t *>(ctx->slots[(size_t)slot_index].dev.S), p.M = L, p.mini_batch = 0;
     p.x_stride = c.d, p.X = pl->self_rows;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.d);
+    CUtensorMap tmap_x;
+    cudaError_t ex = encode_x_map(&tmap_x, pl->self_rows, c.d, (size_t)c.L_max + kTcTile);
+    if (ex != cudaSuccess) return ex;
     const int grid = sl.n_tiles >= 148 * 16 ? 148 : sl.n_tiles;
     cudaError_t e;
     if (c.d == 128 && grid == sl.n_tiles && sl.max_L >= 16 * 128)   // one CTA per tile and many key blocks per tile
         e = launch_pdl(k_att_tc_long, dim3(grid), dim3(kAtt2Threads), kAtt2Smem, st, pl->tmap, p);
     else if (c.d == 128)
-        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(kAttThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, p);
+        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(kAttThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, tmap_x, p);
     else
-        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(kAttThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, p);
+        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(kAttThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, tmap_x, p);
     count_launch();
     *rows_out = pl->self_rows;
     return e;
