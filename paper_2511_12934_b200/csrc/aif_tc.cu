@@ -128,20 +128,24 @@ __global__ void __launch_bounds__(256) k_cross_buckets(const int32_t *__restrict
 {
     grid_dep_launch();
     grid_dep_wait();
-    const int64_t n = total * F;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t pos = i / F;
-        const int f = (int)(i - pos * F);
+    // eight threads per candidate, each taking every eighth field: the id is read once per thread, nothing is divided,
+    // and a warp's stores cover four candidates' rows of F entries
+    const int sub = threadIdx.x & 7;
+    for (int64_t pos = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 3; pos < total; pos += ((int64_t)gridDim.x * blockDim.x) >> 3) {
         const int id = ids[pos];
-        uint32_t bk = kNoBucket;
-        if (id >= 0 && (int64_t)id < M) {
-            if (mode == AIF_BUCKET_MOD) bk = (uint32_t)(id % B);
-            else {
-                const uint64_t h = mix64((uint64_t)id, (uint64_t)f);
-                bk = b_mask >= 0 ? (uint32_t)(h & (uint64_t)b_mask) : (uint32_t)(h % (uint64_t)B);
+        const bool good = id >= 0 && (int64_t)id < M;
+        uint16_t *row = xb + pos * F;
+        for (int f = sub; f < F; f += 8) {
+            uint32_t bk = kNoBucket;
+            if (good) {
+                if (mode == AIF_BUCKET_MOD) bk = (uint32_t)(id % B);
+                else {
+                    const uint64_t h = mix64((uint64_t)id, (uint64_t)f);
+                    bk = b_mask >= 0 ? (uint32_t)(h & (uint64_t)b_mask) : (uint32_t)(h % (uint64_t)B);
+                }
             }
+            row[f] = (uint16_t)bk;
         }
-        xb[i] = (uint16_t)bk;
     }
 }
 
@@ -949,7 +953,7 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl_in
         sl.tiles = (const TileDev *)sc.tiles;
     }
     if (c.blocks & AIF_BLK_CROSS) {
-        const int64_t n = sl.total * c.F;
+        const int64_t n = sl.total * 8;   // eight threads per candidate
         const int grid = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
         cudaError_t e = launch_pdl(k_cross_buckets, dim3(grid), dim3(256), 0, st, sl.ids, sl.total, c.M, c.F, c.B,
                                    (c.B & (c.B - 1)) == 0 ? c.B - 1 : -1, c.bucket_mode, (uint16_t *)sc.xb);
