@@ -1,21 +1,23 @@
 // Tensor-core scoring path for sm_100a (bf16 storage): the scoring MLP as tcgen05 GEMMs with a fused gather
 // prologue and fused epilogues.
 //
-// One layer = one persistent kernel (k_layer_tc<G>).  A work item is (group of G 128-candidate tiles, 256-wide slice
-// of the layer's outputs).  Roles inside a CTA (G = 1: 320 threads, G = 2: 576 threads):
-//   epilogue   4 warps per tile: read the fp32 accumulator from TMEM (tcgen05.ld), add the bias (for the first layer
-//              the request's cached user partial p_u), ReLU, then either store bf16 activations for the next layer or
-//              reduce against w_out and write the logit
+// One layer = one persistent kernel (k_layer_tc<MODE>).  A work item is one or two 128-candidate tiles times one or two
+// 256-wide slices of the layer's outputs (LayerCfg below).  Roles inside a CTA (one accumulator: 320 threads, two: 576):
+//   epilogue   4 warps per accumulator: read the fp32 accumulator from TMEM (tcgen05.ld), add the bias (for the first
+//              layer the request's cached user partial p_u), ReLU, then either store bf16 activations for the next
+//              layer (through a staging slab and a TMA tile store), reduce against w_out and write the logit, or (item
+//              side of the nearline pipeline) store without ReLU / pack the sign bits of the outputs
 //   MMA        one warp allocates TMEM; one lane issues tcgen05.mma (M=128, N<=256, K=16, bf16 in, fp32 accumulate)
 //   A producer 4 warps per tile: gather the tile's input rows chunk by chunk (64 columns = 128 bytes per row) with
 //              16-byte cp.async into the 128B-swizzled K-major layout the MMA reads: item-table rows by candidate
 //              id, cross-feature rows by (field, bucket) from the request's pre-cache with the bucket looked up in
-//              the table k_cross_buckets wrote, dense rows (attention output, previous activations) by position.
+//              the table k_cross_buckets wrote; dense rows (attention output, previous activations, raw item
+//              features) come by position as one TMA tile per chunk.
 //              Ids of the next item and the sources of the next chunk are fetched ahead of their use.
 //   B producer one lane streams the weight slice with TMA (cp.async.bulk.tensor, 128B swizzle)
-// A shared-memory ring (mbarriers) decouples producers from the MMA.  Two TMEM accumulators of 256 columns: with
-// G = 1 they alternate so that the epilogue of one item overlaps the main loop of the next; with G = 2 each tile of
-// the group owns one and both are fed from the same weight chunk.  Every wait is bounded: on expiry the CTA raises
+// Shared-memory rings (mbarriers) decouple producers from the MMA.  Two TMEM accumulators of 256 columns: with one
+// accumulator per item they alternate so that the epilogue of one item overlaps the main loop of the next; with two,
+// each tile (or output slice) of the item owns one.  Every wait is bounded: on expiry the CTA raises
 // AIF_STATUS_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel returns.
 #include <cuda.h>
 

@@ -10,24 +10,27 @@
 //
 // 448 threads:
 //   warps 0-7   two groups of four warps, one thread per candidate row (TMEM lane) in each.  Softmax: group g takes
-//               the scores of key block g; the groups exchange row maxima and sums through shared memory, write the
-//               probabilities back into tensor memory as packed bf16 (A operand of P V), then normalise O into the
-//               attention chunks of the first layer's input (group g: columns [64 g, 64 g + 64)).  Layer-1 epilogue:
-//               group g adds the request's cached user partial p_u to output slice g, applies ReLU and writes the bf16
-//               activations back into tensor memory over the accumulator it has just read (A operand of layer 2).
-//               Layer-2 epilogue: bias, ReLU and the dot with w_out, half of the units per group.
+//               the scores of key block g, writes the probabilities into tensor memory as packed bf16 (A operand of
+//               P V) and exchanges its row sums with the other group through shared memory; then it normalises O into
+//               the attention chunks of the first layer's input (group g: columns [64 g, 64 g + 64)).  While layer 1
+//               runs, the groups build the bias operands in shared memory: both layers' biases (for layer 1 the
+//               request's cached user partial p_u) are added by the tensor cores.  Layer-1 epilogue: ReLU on output
+//               slice g, bf16 activations written back into tensor memory over accumulator columns already read (A
+//               operand of layer 2).  Layer-2 epilogue: ReLU and the dot with w_out, half of the units per group.
 //   warp 8      allocates tensor memory; one lane issues every tcgen05.mma
 //   warps 9-12  gather the tile's item rows (queries of the attention and first K chunks of layer 1) and, chunk by
 //               chunk, its cross-feature rows from the request's pre-cache, with 16-byte cp.async into 128B-swizzled
-//               K-major chunks; buckets are hashed one chunk ahead of their use
+//               K-major chunks; buckets are hashed one chunk ahead of their use; last, the tile of ones that multiplies
+//               the bias operands
 //   warp 13     one lane streams key/value blocks, then first- and second-layer weights with TMA
 //
 // Tensor memory (512 columns): attention uses [0, 256) for the scores of up to two key blocks, [256, 384) for O and
 // [384, 512) for the probabilities (packed bf16, 64 columns per key block).  Layer 1 then fills two 256-column
 // accumulators [0, 256) and [256, 512); its activations are packed over them into [0, 128) and [384, 512); layer 2
 // accumulates into the freed columns [128, 384).
-// Shared memory: item tile 32 KB | key/value blocks 64 KB, later the attention chunks and two more stages of the
-// cross-feature ring | two cross-feature stages 32 KB | weight ring 3 x 32 KB | barriers and exchange arrays.
+// Shared memory: item tile 32 KB, later the bias operands and the output weights | key/value blocks 64 KB, later the
+// attention chunks and two more stages of the cross-feature ring | two cross-feature stages 32 KB | weight ring
+// 3 x 32 KB | barriers and the exchange array.
 // Every wait is bounded: on expiry the CTA raises AIF_STATUS_TIMEOUT, every role skips its remaining work, tensor
 // memory is freed and the kernel returns.
 #include <cuda.h>
