@@ -382,7 +382,7 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
         el = 4 if wl.dtype == "f32" else 2
         nearline = {"items": nn, "dI": dI, "hI": hI, "ms": n_ms, "items_per_s": nn / (n_ms * 1e-3),
                     "tflops": nn * n_flops / (n_ms * 1e-3) / 1e12, "gbs": nn * (dI + wl.d) * el / (n_ms * 1e-3) / 1e9,
-                    "note": "tower flops and (raw row in + item vector out) bytes only; the hidden activations pass through HBM"}
+                    "note": "tower flops and (raw row in + item vector out) bytes; one kernel, hidden activations in tensor memory"}
         srv.ctx.item_nearline_refresh(None, saved)
         del dev_it, saved
 

@@ -1,8 +1,9 @@
 // Item side of the nearline pipeline as a compute call (Section 3.2 eq. 4, Algorithm 1 step 3, Section 4.2 eq. 5):
 // raw item features -> item vectors, BEA weight rows and LSH signatures, written into the item table.
 //
-// bf16 contexts whose widths fit the layer kernel run the tower's two layers and the hash projections on the tensor
-// cores (tc_dense_layer: the scoring MLP's kernel over dense rows, with a linear-output and a sign-bit epilogue); every
+// bf16 contexts whose widths fit run on the tensor cores: the tower as one kernel with its hidden activations in tensor
+// memory (aif_tc_tower.cu; hidden width <= 256, d <= 128) or as two launches of the scoring MLP's layer kernel over dense
+// rows (tc_dense_layer, linear-output epilogue), the hash projections as one such launch with a sign-bit epilogue; every
 // other case runs the CUDA-core kernels below.  The BEA weights are 2 n d flop per item against d element reads: a
 // warp per item on CUDA cores.  Items are processed in passes of at most kPassRows rows so that the scratch
 // (hidden activations; for incremental updates also the rows before their scatter) stays bounded.
@@ -19,6 +20,7 @@ constexpr int64_t kPassRows = 1 << 20;
 struct NearlinePlan {
     int dI = 0, hI = 0, d_mm = 0;
     bool ready = false, tensor = false;
+    bool fused_tower = false;             // both tower layers in one kernel (hidden activations in tensor memory)
     void *W0 = nullptr, *W1 = nullptr, *bridges = nullptr, *W_hash = nullptr;
     float *b0 = nullptr, *b1 = nullptr, *zeros = nullptr;
     int64_t cap = 0;                      // rows per pass the scratch has room for
@@ -122,7 +124,9 @@ cudaError_t run_pass(aif_ctx *ctx, NearlinePlan *pl, int64_t m, const void *I_ra
 {
     const aif_config &c = ctx->cfg;
     cudaError_t e;
-    if (pl->tensor) {
+    if (pl->tensor && pl->fused_tower) {
+        if ((e = launch_item_tower_tc(ctx, I_raw, pl->W0, pl->b0, pl->W1, pl->b1, rows_out, m, pl->dI, pl->hI, st)) != cudaSuccess) return e;
+    } else if (pl->tensor) {
         DenseLayer l0{I_raw, pl->W0, pl->b0, pl->hidden, pl->dI, pl->hI, 1, 0};
         if ((e = tc_dense_layer(ctx, l0, m, st)) != cudaSuccess) return e;
         DenseLayer l1{pl->hidden, pl->W1, pl->b1, rows_out, pl->hI, c.d, 0, 0};
@@ -174,6 +178,7 @@ int nearline_load_weights(aif_ctx *ctx, const aif_item_weights *w, cudaStream_t 
         const int H = w->hI;
         pl->tensor = ctx->tensor_path && w->dI % 64 == 0 && H % 64 == 0 && (H <= 256 || H % 256 == 0) && w->dI <= 4096 && H <= 4096 &&
                      c.d % 32 == 0 && c.d <= 256 && (!lsh || (w->d_mm % 64 == 0 && w->d_mm <= 4096 && c.lsh_bits <= 256));
+        pl->fused_tower = pl->tensor && tc_tower_supported(w->dI, H, c.d) && tc_tower_prepare() == cudaSuccess;
         pl->cap = c.M < kPassRows ? c.M : kPassRows;
         cudaError_t e = cudaSuccess;
         auto need = [&](void **p, size_t bytes) {
@@ -186,7 +191,7 @@ int nearline_load_weights(aif_ctx *ctx, const aif_item_weights *w, cudaStream_t 
         need((void **)&pl->zeros, 4096 * 4);
         if (bea) need(&pl->bridges, (size_t)c.n_bridge * c.d * el);
         if (lsh) need(&pl->W_hash, (size_t)c.lsh_bits * w->d_mm * el);
-        if (pl->tensor) need(&pl->hidden, (size_t)(pl->cap + kTcTile) * w->hI * 2);
+        if (pl->tensor && !pl->fused_tower) need(&pl->hidden, (size_t)(pl->cap + kTcTile) * w->hI * 2);
         need(&pl->rows, (size_t)(pl->cap + kTcTile) * c.d * el);
         if (bea) need(&pl->bea, (size_t)pl->cap * c.n_bridge * el);
         if (lsh) need((void **)&pl->sig, (size_t)(pl->cap + kTcTile) * c.lsh_bits / 8);

@@ -32,10 +32,13 @@ def _read_back(srv, wl, ids):
     return rows.float().cpu().numpy().astype(np.float64), bea.float().cpu().numpy().astype(np.float64), sig.cpu().numpy()
 
 
-# widths: (dI, hI, d_mm).  bf16 with multiples of 64 runs on the tensor cores (ragged last tile, several tiles, a hidden
-# layer wider than one 256-column slice); the other shapes run the CUDA-core kernels.
+# widths: (dI, hI, d_mm).  bf16 with multiples of 64 runs on the tensor cores: hidden widths up to 256 at d = 128 in the
+# one-kernel tower (ragged last tile, an odd number of tiles, more tile pairs than one CTA round at M = 4000 is not needed:
+# pairs are walked persistently), wider ones and d = 256 as two launches of the layer kernel; the other shapes run the
+# CUDA-core kernels.
 @pytest.mark.parametrize("name,dims,n", [("c1", (40, 24, 20), 777), ("c2", (512, 256, 128), 1111), ("c2", (192, 512, 64), 300),
-                                         ("c2", (100, 60, 36), 333), ("c5", (256, 128, 256), 515)])
+                                         ("c2", (100, 60, 36), 333), ("c5", (256, 128, 256), 515), ("c2", (128, 192, 128), 3000),
+                                         ("c2", (64, 64, 64), 130)])
 @pytest.mark.parametrize("incremental", [False, True])
 def test_nearline_compute_matches_the_oracle(name, dims, n, incremental):
     dI, hI, d_mm = dims
