@@ -277,6 +277,28 @@ def test_single_launch_scoring_at_the_sequence_lengths_around_its_key_blocks(L):
     srv.close()
 
 
+@pytest.mark.parametrize("L", [200, 300])
+def test_several_requests_with_mini_batches_in_one_launch(L):
+    """Requests of different sizes, each cut into mini-batches of 500 (tiles never straddle a mini-batch), scored in one
+    launch: the tile table of the kernel-per-layer path (L = 300) and the request search of the single-launch kernel
+    (L = 200) must both place every tile in its request."""
+    wl = helpers.MINI["c2"].with_(name=f"batch_mb_{L}", R=4, N=1100, L=L, mini_batch=500, mixed_sizes=(300, 1300))
+    weights, table, srv, oracle = _setup(wl)
+    sampler = synth.IdSampler(wl)
+    states, id_lists, wants = [], [], []
+    for r in range(wl.R):
+        rq = synth.make_request(wl, r)
+        ids = sampler.request_ids(r)
+        states.append(srv.precompute(20 + r, srv.upload_request(rq, B.USER_PROJECTED)))
+        id_lists.append(ids)
+        wants.append(oracle.score(table, helpers.projected_request(wl, rq), ids))
+    assert len({len(x) for x in id_lists}) > 1
+    for o, w in zip(srv.score_many(states, id_lists), wants):
+        _check_logits(o, w, TOL["bf16"])
+    assert srv.ctx.poll_status() == 0
+    srv.close()
+
+
 @pytest.mark.parametrize("H2,F,dc,Bk,mode,sig", [(64, 2, 32, 1024, synth.BUCKET_HASH, 0), (128, 8, 8, 1000, synth.BUCKET_HASH, 1),
                                                   (192, 12, 16, 1024, synth.BUCKET_MOD, 0), (256, 8, 64, 37, synth.BUCKET_MOD, 1),
                                                   (256, 24, 16, 512, synth.BUCKET_HASH, 0)])
