@@ -496,32 +496,62 @@ __global__ void __launch_bounds__(256) k_user_finish(int raw, const T *__restric
                                                      __nv_bfloat16 *__restrict__ pu_hl, const T *__restrict__ Wb_t, const float *__restrict__ b_b,
                                                      const float *__restrict__ ppart)
 {
-    __shared__ float q[256], uprof[256], us[256];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, dq = d >> 5;
+    __shared__ float q[256], uprof[256], us[256], wgt[kProfParts], red[256];
+    static_assert(kProfParts == 256, "one thread per key slice");
+    const int tid = threadIdx.x;
     if (raw) {
-        // merge the key slices of the profile attention: softmax over all keys from per-slice maxima and sums
+        // merge the key slices of the profile attention: softmax over all keys from per-slice maxima and sums.  One
+        // thread per slice for the weights 2^(m_g - m) (kProfParts = blockDim), then one thread per output column.
         {
-            float m_all = -INFINITY;
-            for (int g = 0; g < kProfParts; ++g) m_all = fmaxf(m_all, ppart[(size_t)g * (d + 2) + d]);
-            float den = 0.f;
-            for (int g = 0; g < kProfParts; ++g) {
-                const float l = ppart[(size_t)g * (d + 2) + d + 1];
-                if (l > 0.f) den += l * expf(ppart[(size_t)g * (d + 2) + d] - m_all);
+            const float m_g = ppart[(size_t)tid * (d + 2) + d], l_g = ppart[(size_t)tid * (d + 2) + d + 1];
+            red[tid] = l_g > 0.f ? m_g : -INFINITY;
+            __syncthreads();
+            for (int o = 128; o > 0; o >>= 1) {
+                if (tid < o) red[tid] = fmaxf(red[tid], red[tid + o]);
+                __syncthreads();
             }
+            const float m_all = red[0];
+            __syncthreads();
+            const float w = l_g > 0.f ? expf(m_g - m_all) : 0.f;
+            wgt[tid] = w;
+            red[tid] = w * l_g;
+            __syncthreads();
+            for (int o = 128; o > 0; o >>= 1) {   // fixed tree: the same sum in every run
+                if (tid < o) red[tid] += red[tid + o];
+                __syncthreads();
+            }
+            const float den = red[0];
             for (int k = tid; k < d; k += 256) {
-                float num = 0.f;
-                for (int g = 0; g < kProfParts; ++g)
-                    if (ppart[(size_t)g * (d + 2) + d + 1] > 0.f)
-                        num = fmaf(expf(ppart[(size_t)g * (d + 2) + d] - m_all), ppart[(size_t)g * (d + 2) + k], num);
-                uprof[k] = num / den;
+                float n4[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int g = 0; g < kProfParts; g += 4) {   // four independent loads in flight
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) n4[u] = fmaf(wgt[g + u], ppart[(size_t)(g + u) * (d + 2) + k], n4[u]);
+                }
+                uprof[k] = ((n4[0] + n4[1]) + (n4[2] + n4[3])) / den;
             }
         }
         __syncthreads();
-        // mean over the sequence of the hidden FFN activations (the warps' partial sums, in a fixed order) ...
-        for (int k = tid; k < d; k += 256) {
-            float acc = 0.f;
-            for (int g = 0; g < n_warps; ++g) acc += partial[(size_t)g * d + k];
-            q[k] = acc / (float)L;
+        // mean over the sequence of the hidden FFN activations: the warps' partial sums in a fixed order, 256 / d threads
+        // per column over interleaved slices of the partials, eight loads in flight per thread
+        {
+            const int parts = 256 / d > 0 ? 256 / d : 1;
+            const int k = tid % d, part = tid / d;
+            float a8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            if (part < parts && k < d) {
+                int g = part;
+                for (; g + 7 * parts < n_warps; g += 8 * parts) {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) a8[u] += partial[(size_t)(g + u * parts) * d + k];
+                }
+                for (; g < n_warps; g += parts) a8[0] += partial[(size_t)g * d + k];
+            }
+            red[tid] = ((a8[0] + a8[1]) + (a8[2] + a8[3])) + ((a8[4] + a8[5]) + (a8[6] + a8[7]));
+            __syncthreads();
+            for (int kk = tid; kk < d; kk += 256) {
+                float acc = 0.f;
+                for (int pp = 0; pp < parts; ++pp) acc += red[pp * d + kk];
+                q[kk] = acc / (float)L;
+            }
         }
         __syncthreads();
         // ... through the second FFN layer, plus the profile attention: the combined user vector

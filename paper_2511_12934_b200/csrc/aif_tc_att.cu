@@ -25,7 +25,7 @@ namespace aif {
 namespace {
 
 constexpr int kAttThreads = 224;
-constexpr int kAttMmaWarp = 4, kAttTmaWarp = 5, kAttQWarp = 6;
+constexpr int kAttMmaWarp = 4, kAttTmaWarp = 5;   // warp 6 gathers queries
 
 struct AttParams {
     ScoreLaunch sl;

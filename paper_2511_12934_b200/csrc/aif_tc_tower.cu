@@ -22,7 +22,7 @@
 namespace aif {
 namespace {
 
-constexpr int kTThreads = 320, kTMmaWarp = 8, kTTmaWarp = 9;
+constexpr int kTThreads = 320, kTMmaWarp = 8;   // warp 9 streams rows and weights
 constexpr int kTStagesA = 3, kTStagesB = 3, kTAStage = 32768, kTBStage = 32768;
 constexpr int kTOffB = kTStagesA * kTAStage, kTOffSlab = kTOffB + kTStagesB * kTBStage, kTOffMisc = kTOffSlab + 8 * 2048;
 constexpr size_t kTSmem = 1024 + kTOffMisc + 2048;
