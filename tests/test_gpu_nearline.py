@@ -89,6 +89,27 @@ def test_nearline_compute_matches_the_oracle(name, dims, n, incremental):
     srv.close()
 
 
+def test_one_kernel_tower_with_several_tile_pairs_per_cta():
+    """More rows than 148 CTAs take in one round of tile pairs (each CTA walks over three pairs, the last one ragged):
+    the reuse of tensor memory, of the barriers' phases and of the operand rings from pair to pair."""
+    n = 148 * 256 * 2 + 9 * 256 + 77
+    wl = helpers.MINI["c2"].with_(name="nearline_pairs", M=n, L=20, N=50)
+    srv = serving.Server(wl, synth.make_weights(wl), {"E": np.zeros((n, wl.d), dtype=np.uint16)})
+    it = synth.make_item_side(wl, n, 128, 128, 64)
+    dev = {k: (torch.from_numpy(v).cuda() if v.dtype == np.float32 else B.to_device(v, B.BF16)) for k, v in it.items()}
+    srv.ctx.load_item_weights(dev)
+    srv.ctx.item_nearline_compute(None, dev["I_raw"])
+    assert srv.ctx.poll_status() == 0
+    want = orc.item_nearline(orc.BF16, I_raw=it["I_raw"], W0=it["W_i0"], b0=it["b_i0"], W1=it["W_i1"], b1=it["b_i1"])["I_hat"]
+    ids_t = torch.arange(n, dtype=torch.int32, device="cuda")
+    rows = torch.empty(n, wl.d, dtype=torch.bfloat16, device="cuda")
+    srv.ctx.gather_rows(ids_t, rows)
+    torch.cuda.synchronize()
+    got = rows.float().cpu().numpy().astype(np.float64)
+    assert np.allclose(got, want, rtol=2.0 ** -7, atol=5e-4), np.abs(got - want).max()
+    srv.close()
+
+
 def test_scoring_on_a_table_built_by_the_nearline_call():
     """End to end: the table rows come from aif_item_nearline_compute, the scores from aif_score; the oracle does both
     from the same raw inputs.  The item vectors differ from the oracle's by bf16 rounding, so the budget is the bf16
