@@ -301,6 +301,29 @@ def test_several_requests_with_mini_batches_in_one_launch(L):
     srv.close()
 
 
+@pytest.mark.parametrize("L", [200, 300])
+def test_a_launch_with_empty_requests_among_the_others(L):
+    """Requests without candidates at the start, in the middle and at the end of a batch: their tiles do not exist, and
+    every existing tile must still find its own request (single-launch kernel at L = 200, tile table at L = 300)."""
+    wl = helpers.MINI["c2"].with_(name=f"empty_req_{L}", R=5, N=260, L=L, mini_batch=0)
+    weights, table, srv, oracle = _setup(wl)
+    sampler = synth.IdSampler(wl)
+    states, id_lists, wants = [], [], []
+    for r in range(wl.R):
+        rq = synth.make_request(wl, r)
+        ids = sampler.request_ids(r) if r in (1, 3) else np.zeros(0, dtype=np.int32)
+        states.append(srv.precompute(30 + r, srv.upload_request(rq, B.USER_PROJECTED)))
+        id_lists.append(ids)
+        wants.append(oracle.score(table, helpers.projected_request(wl, rq), ids) if len(ids) else np.zeros(0))
+    outs = srv.score_many(states, id_lists)
+    for o, w in zip(outs, wants):
+        assert len(o) == len(w)
+        if len(w):
+            _check_logits(o, w, TOL["bf16"])
+    assert srv.ctx.poll_status() == 0
+    srv.close()
+
+
 @pytest.mark.parametrize("H2,F,dc,Bk,mode,sig", [(64, 2, 32, 1024, synth.BUCKET_HASH, 0), (128, 8, 8, 1000, synth.BUCKET_HASH, 1),
                                                   (192, 12, 16, 1024, synth.BUCKET_MOD, 0), (256, 8, 64, 37, synth.BUCKET_MOD, 1),
                                                   (256, 24, 16, 512, synth.BUCKET_HASH, 0)])
