@@ -2,17 +2,21 @@
 // candidates against the request's projected behaviour sequence S [L x d] (Section 4.2, first paragraph: similarity
 // of the target item with every historical item, then pooling; here in its dense softmax form).
 //
-// Persistent kernel: one CTA per SM walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  224 threads:
+// Persistent kernel: one CTA per SM walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  224 threads (d = 256)
+// or 352 (d = 128):
 //   warps 0-3  per key block: read the score row from TMEM into registers, online softmax in fp32 (one thread per
 //              candidate row), write the probabilities back into the same TMEM columns as packed bf16 pairs (the A
 //              operand of P V is read from tensor memory, which keeps it off the shared-memory bandwidth the products
-//              are bound by); at the end of a tile normalise O and store the attention rows
+//              are bound by); at the end of a tile normalise O and store the attention rows (d = 256) or hand the
+//              row sums to warps 7-10 (d = 128)
 //   warp  4    allocates TMEM; one lane issues tcgen05.mma over the flat sequence of key blocks of all its tiles:
 //              scores = Q K^T (both K-major) one block ahead of O += P V, with V read from the very same shared-memory
 //              tile as K, as an MN-major B operand
 //   warp  5    one lane streams key/value blocks of S with TMA (3-D tensor map over the user-state arena)
 //   warp  6    gathers the item rows of the next tile (the queries) with cp.async while the current tile is processed
 //              (two query buffers)
+//   warps 7-10 d = 128 only: normalise the finished tile's O accumulator and store its rows while the other warps are
+//              on the next tile (two O accumulators fill the 512 tensor-memory columns)
 // TMEM: two score buffers (so the softmax of block j overlaps Q K^T of block j+1) and the O accumulator.
 // The running maximum is only raised when a row's block maximum exceeds it by more than 8 (in the log2 domain);
 // then the warp rescales its 32 rows of O in TMEM.  Until then probabilities stay below 2^8, which fp32 sums and
@@ -24,7 +28,6 @@
 namespace aif {
 namespace {
 
-constexpr int kAttThreads = 224;
 constexpr int kAttMmaWarp = 4, kAttTmaWarp = 5;   // warp 6 gathers queries
 
 struct AttParams {
@@ -45,8 +48,12 @@ struct AttCfg {
     static constexpr int kKvStages = D <= 128 ? 5 : 3;
     static constexpr int kKvChunkBytes = BN * 128;      // one 64-column chunk of a key block
     static constexpr int kKvBytes = kQChunks * kKvChunkBytes;
-    static constexpr int kTmemO = 2 * BN;               // column of the O accumulator
-    static constexpr size_t kSmem = 1024 + kQBufs * kQBytes + kKvStages * kKvBytes + 512;
+    static constexpr int kTmemO = 2 * BN;               // column of the (first) O accumulator
+    // d = 128 leaves 128 tensor-memory columns free: a second O accumulator, and four more warps that normalise and store
+    // a finished tile while the softmax warps and the MMAs are already on the next one
+    static constexpr bool kSplitEpi = D <= 128;
+    static constexpr int kThreads = kSplitEpi ? 352 : 224;
+    static constexpr size_t kSmem = 1024 + kQBufs * kQBytes + kKvStages * kKvBytes + 1536;
 };
 
 // One tile of the launch as every role needs it.
@@ -77,11 +84,12 @@ __device__ __forceinline__ AttTile att_tile(const AttParams &p, int tile)
 }
 
 template <int D, int BN>
-__global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant__ CUtensorMap tmapS,
+__global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const __grid_constant__ CUtensorMap tmapS,
                                                            const __grid_constant__ CUtensorMap tmapX, const AttParams p)
 {
     using C = AttCfg<D, BN>;
     constexpr int kS = C::kKvStages, kQB = C::kQBufs;
+    constexpr bool kSplit = C::kSplitEpi;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
     unsigned char *smQ = base;
@@ -89,9 +97,11 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
     uint64_t *bars = reinterpret_cast<uint64_t *>(smKV + kS * C::kKvBytes);
     uint64_t *kv_full = bars, *kv_empty = bars + kS;
     uint64_t *s_full = bars + 2 * kS, *p_full = s_full + 2, *pv_done = p_full + 2;
-    uint64_t *q_full = pv_done + 2, *q_empty = q_full + 2, *o_final = q_empty + 2, *o_free = o_final + 1, *q_first = o_free + 1;
+    uint64_t *q_full = pv_done + 2, *q_empty = q_full + 2, *o_final = q_empty + 2, *o_free = o_final + 2, *l_ready = o_free + 2;
+    uint64_t *q_first = l_ready + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_first + 1);
     volatile uint32_t *abort_flag = tmem_slot + 1;
+    float *l_s = reinterpret_cast<float *>(tmem_slot + 4);   // [2][128] row sums handed to the epilogue warps
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -107,8 +117,11 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
             mbar_init(smem_u32(q_full + b), 32);
             mbar_init(smem_u32(q_empty + b), 5);   // the last Q K^T of the tenant, and the four softmax warps' output staging
         }
-        mbar_init(smem_u32(o_final), 1);
-        mbar_init(smem_u32(o_free), 128);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(o_final + b), 1);
+            mbar_init(smem_u32(o_free + b), 128);
+            mbar_init(smem_u32(l_ready + b), 128);
+        }
         mbar_init(smem_u32(q_first), 128);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -122,6 +135,80 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
     grid_dep_wait();   // the set-up above overlapped the previous kernel; the request table and slots are read from here on
 
     const int n_tiles = p.sl.n_tiles;
+
+    // Normalises a finished tile's O accumulator and stores the attention rows.  Run by the softmax warps themselves
+    // (d = 256) or by the epilogue warps (d = 128); wq = the warp's quarter of the TMEM lanes.
+    auto tile_epilogue = [&](int k, const AttTile &t, float l_sum, int wq, int lane) {
+        const int row = wq * 32 + lane;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(wq * 32) << 16);
+        const uint32_t o_col = (uint32_t)(C::kTmemO + (kSplit ? (k & 1) * D : 0));
+        uint64_t *o_free_k = o_free + (kSplit ? (k & 1) : 0);
+        const float inv = 1.0f / l_sum;
+        bool good = false;
+        if (row < t.cnt) {
+            const int id = p.sl.ids[t.pos0 + row];
+            good = id >= 0 && (int64_t)id < p.M;
+        }
+        // Output rows leave through shared memory and asynchronous tile stores: a thread owns a row, so direct stores
+        // are 32 scattered half-used sectors per instruction, which cost several thousand cycles per tile.  The
+        // staging slabs (2 x 2 KB per warp, 64-byte swizzle) live in the tile's own query buffer: every Q K^T of the
+        // tile is complete, and the gather of the buffer's next tenant waits for these warps as well.
+        const int qb_out = k % kQB;
+        unsigned char *stg = smQ + qb_out * C::kQBytes + wq * 4096;
+        const bool whole = wq * 32 + 32 <= t.cnt;   // ragged last tiles keep the guarded direct stores
+        uint32_t slab = 0;
+        auto emit = [&](const uint32_t (&r)[32], int c0) {
+            uint32_t packed[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const __nv_bfloat162 h = __floats2bfloat162_rn(good ? __uint_as_float(r[2 * i]) * inv : 0.f,
+                                                               good ? __uint_as_float(r[2 * i + 1]) * inv : 0.f);
+                packed[i] = *reinterpret_cast<const uint32_t *>(&h);
+            }
+            if (whole) {
+                unsigned char *sb = stg + slab * 2048;
+                if (lane == 0) bulk_wait_read<1>();   // the store that last read this slab is done with it
+                __syncwarp();
+                const int swz = (lane >> 1) & 3;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    *reinterpret_cast<uint4 *>(sb + lane * 64 + ((q ^ swz) << 4)) =
+                        make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(&tmapX, smem_u32(sb), c0, (int)(t.pos0 + wq * 32));
+                    bulk_commit();
+                }
+                slab ^= 1u;
+            } else if (row < t.cnt) {
+                uint4 *dst = reinterpret_cast<uint4 *>(p.X + (size_t)(t.pos0 + row) * p.x_stride + c0);
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+            }
+        };
+        // two chunks of 32 columns per round; the load of the next chunk is in flight while one is converted and staged
+        uint32_t ra[32], rb[32];
+        tmem_ld32(lane_base + o_col, ra);
+#pragma unroll 1
+        for (int c0 = 0; c0 < D; c0 += 64) {
+            tmem_ld_wait();
+            tmem_ld32(lane_base + o_col + (uint32_t)(c0 + 32), rb);
+            emit(ra, c0);
+            tmem_ld_wait();
+            if (c0 + 64 < D) tmem_ld32(lane_base + o_col + (uint32_t)(c0 + 64), ra);
+            else {   // O is in registers: the next tile's first P V may overwrite the accumulator
+                tc_fence_before();
+                mbar_arrive(smem_u32(o_free_k));
+            }
+            emit(rb, c0 + 32);
+        }
+        if (lane == 0) {
+            bulk_wait_read<0>();   // the staging is no longer read: the query buffer may take its next tenant
+            mbar_arrive(smem_u32(q_empty + qb_out));
+        }
+    };
 
     if (warp < 4) {
         // ===================== softmax, output =====================
@@ -203,11 +290,12 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
 #pragma unroll 1
                         for (int c0 = 0; c0 < D; c0 += 32) {
                             uint32_t r[32];
-                            tmem_ld32(lane_base + (uint32_t)(C::kTmemO + c0), r);
+                            const uint32_t oc = (uint32_t)(C::kTmemO + (kSplit ? (k & 1) * D : 0) + c0);
+                            tmem_ld32(lane_base + oc, r);
                             tmem_ld_wait();
 #pragma unroll
                             for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
-                            tmem_st32(lane_base + (uint32_t)(C::kTmemO + c0), r);
+                            tmem_st32(lane_base + oc, r);
                         }
                         tmem_st_wait();
                     }
@@ -237,75 +325,23 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                 tc_fence_before();
                 mbar_arrive(smem_u32(p_full + b));
             }
-            if (!ok || !mbar_wait(smem_u32(o_final), (uint32_t)(k & 1), abort_flag)) {
-                ok = false;
-                break;
-            }
-            tc_fence_after();
-            const float inv = 1.0f / l_sum;
-            bool good = false;
-            if (row < t.cnt) {
-                const int id = p.sl.ids[t.pos0 + row];
-                good = id >= 0 && (int64_t)id < p.M;
-            }
-            // Output rows leave through shared memory and asynchronous tile stores: a thread owns a row, so direct stores
-            // are 32 scattered half-used sectors per instruction, which cost several thousand cycles per tile.  The
-            // staging slabs (2 x 2 KB per warp, 64-byte swizzle) live in the tile's own query buffer: every Q K^T of the
-            // tile is complete, and the gather of the buffer's next tenant waits for these warps as well.
-            const int qb_out = k % kQB;
-            unsigned char *stg = smQ + qb_out * C::kQBytes + warp * 4096;
-            const bool whole = warp * 32 + 32 <= t.cnt;   // ragged last tiles keep the guarded direct stores
-            uint32_t slab = 0;
-            auto emit = [&](const uint32_t (&r)[32], int c0) {
-                uint32_t packed[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const __nv_bfloat162 h = __floats2bfloat162_rn(good ? __uint_as_float(r[2 * i]) * inv : 0.f,
-                                                                   good ? __uint_as_float(r[2 * i + 1]) * inv : 0.f);
-                    packed[i] = *reinterpret_cast<const uint32_t *>(&h);
+            if (!ok) break;
+            if (kSplit) {
+                // hand the row sums to the epilogue warps and go on with the next tile.  l_s[k & 1] was last read by the
+                // epilogue of tile k - 2, before that epilogue released its O accumulator.
+                if (k >= 2 && !mbar_wait(smem_u32(o_free + (k & 1)), (uint32_t)(((k - 2) >> 1) & 1), abort_flag)) {
+                    ok = false;
+                    break;
                 }
-                if (whole) {
-                    unsigned char *sb = stg + slab * 2048;
-                    if (lane == 0) bulk_wait_read<1>();   // the store that last read this slab is done with it
-                    __syncwarp();
-                    const int swz = (lane >> 1) & 3;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4 *>(sb + lane * 64 + ((q ^ swz) << 4)) =
-                            make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&tmapX, smem_u32(sb), c0, (int)(t.pos0 + warp * 32));
-                        bulk_commit();
-                    }
-                    slab ^= 1u;
-                } else if (row < t.cnt) {
-                    uint4 *dst = reinterpret_cast<uint4 *>(p.X + (size_t)(t.pos0 + row) * p.x_stride + c0);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                l_s[(k & 1) * 128 + row] = l_sum;
+                mbar_arrive(smem_u32(l_ready + (k & 1)));
+            } else {
+                if (!mbar_wait(smem_u32(o_final), (uint32_t)(k & 1), abort_flag)) {
+                    ok = false;
+                    break;
                 }
-            };
-            // two chunks of 32 columns per round; the load of the next chunk is in flight while one is converted and staged
-            uint32_t ra[32], rb[32];
-            tmem_ld32(lane_base + (uint32_t)C::kTmemO, ra);
-#pragma unroll 1
-            for (int c0 = 0; c0 < D; c0 += 64) {
-                tmem_ld_wait();
-                tmem_ld32(lane_base + (uint32_t)(C::kTmemO + c0 + 32), rb);
-                emit(ra, c0);
-                tmem_ld_wait();
-                if (c0 + 64 < D) tmem_ld32(lane_base + (uint32_t)(C::kTmemO + c0 + 64), ra);
-                else {   // O is in registers: the next tile's first P V may overwrite the accumulator
-                    tc_fence_before();
-                    mbar_arrive(smem_u32(o_free));
-                }
-                emit(rb, c0 + 32);
-            }
-            if (lane == 0) {
-                bulk_wait_read<0>();   // the staging is no longer read: the query buffer may take its next tenant
-                mbar_arrive(smem_u32(q_empty + qb_out));
+                tc_fence_after();
+                tile_epilogue(k, t, l_sum, warp, lane);
             }
         }
         if (lane == 0) bulk_wait<0>();   // all tile stores of this warp have reached global memory
@@ -375,13 +411,14 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                     break;
                 }
                 // the first P V of a tile overwrites O: the previous tile's output must have been read
-                if (cp.j == 0 && cp.k > 0 && !mbar_wait(smem_u32(o_free), (uint32_t)((cp.k - 1) & 1), abort_flag)) {
+                if (cp.j == 0 && (kSplit ? cp.k >= 2 && !mbar_wait(smem_u32(o_free + (cp.k & 1)), (uint32_t)(((cp.k - 2) >> 1) & 1), abort_flag)
+                                         : cp.k > 0 && !mbar_wait(smem_u32(o_free), (uint32_t)((cp.k - 1) & 1), abort_flag))) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
                 const int s = (int)(cp.gb % kS);
-                const uint32_t o_tmem = tmem_base + (uint32_t)C::kTmemO;
+                const uint32_t o_tmem = tmem_base + (uint32_t)(C::kTmemO + (kSplit ? (cp.k & 1) * D : 0));
                 const uint32_t p_tmem = tmem_base + (uint32_t)((cp.gb & 1u) * BN);   // P: 8 columns per 16 keys
                 const uint64_t vd = vdesc0 + (uint64_t)(uint32_t)(s * (C::kKvBytes >> 4));
 #pragma unroll
@@ -390,7 +427,7 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
                                  (cp.j > 0 || kk > 0) ? 1u : 0u);
                 umma_commit(smem_u32(pv_done + (cp.gb & 1u)));
                 umma_commit(smem_u32(kv_empty + s));
-                if (cp.j == cp.nb - 1) umma_commit(smem_u32(o_final));
+                if (cp.j == cp.nb - 1) umma_commit(smem_u32(o_final + (kSplit ? (cp.k & 1) : 0)));
                 advance(cp);
             }
         }
@@ -417,7 +454,22 @@ __global__ void __launch_bounds__(kAttThreads, 1) k_att_tc(const __grid_constant
             }
         }
         __syncwarp();
-    } else {
+    } else if (kSplit && warp >= 7) {
+        // ===================== output of finished tiles (d = 128: 128 threads) =====================
+        const int wq = warp & 3;   // the quarter of the tensor-memory lanes this warp may read
+        int k = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++k) {
+            const AttTile t = att_tile<BN>(p, tile);
+            const int b = k & 1;
+            const uint32_t parity = (uint32_t)((k >> 1) & 1);
+            if (!mbar_wait(smem_u32(l_ready + b), parity, abort_flag)) break;
+            const float l_sum = l_s[b * 128 + wq * 32 + lane];
+            if (!mbar_wait(smem_u32(o_final + b), parity, abort_flag)) break;
+            tc_fence_after();
+            tile_epilogue(k, t, l_sum, wq, lane);
+        }
+        if (lane == 0) bulk_wait<0>();   // all tile stores of this warp have reached global memory
+    } else if (warp == 6) {
         // ===================== query gather (32 threads) =====================
         // 8 threads per row (16 bytes each per 128-byte chunk), rows lane / 8 + 4 i, 128B-swizzled K-major chunks
         const int sub = lane & 7, r0 = lane >> 3;
@@ -861,9 +913,9 @@ cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
     if (c.d == 128 && grid == sl.n_tiles && sl.max_L >= 16 * 128)   // one CTA per tile and many key blocks per tile
         e = launch_pdl(k_att_tc_long, dim3(grid), dim3(kAtt2Threads), kAtt2Smem, st, pl->tmap, p);
     else if (c.d == 128)
-        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(kAttThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, tmap_x, p);
+        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(AttCfg<128, 128>::kThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, tmap_x, p);
     else
-        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(kAttThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, tmap_x, p);
+        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(AttCfg<256, 64>::kThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, tmap_x, p);
     count_launch();
     return e;
 }
@@ -889,9 +941,9 @@ cudaError_t launch_self_att_tc(const aif_ctx *ctx, int slot_index, int L, cudaSt
     if (c.d == 128 && grid == sl.n_tiles && sl.max_L >= 16 * 128)   // one CTA per tile and many key blocks per tile
         e = launch_pdl(k_att_tc_long, dim3(grid), dim3(kAtt2Threads), kAtt2Smem, st, pl->tmap, p);
     else if (c.d == 128)
-        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(kAttThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, tmap_x, p);
+        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(AttCfg<128, 128>::kThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, tmap_x, p);
     else
-        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(kAttThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, tmap_x, p);
+        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(AttCfg<256, 64>::kThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, tmap_x, p);
     count_launch();
     *rows_out = pl->self_rows;
     return e;
