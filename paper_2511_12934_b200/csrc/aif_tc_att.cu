@@ -28,7 +28,6 @@
 namespace aif {
 namespace {
 
-constexpr int kAttMmaWarp = 4, kAttTmaWarp = 5;   // warp 6 gathers queries
 
 struct AttParams {
     ScoreLaunch sl;
@@ -45,15 +44,23 @@ struct AttCfg {
     static constexpr int kQChunks = D / 64;             // 64-column (128-byte) chunks of a row
     static constexpr int kQBytes = kQChunks * 128 * 128;
     static constexpr int kQBufs = 2;                    // query buffers
-    static constexpr int kKvStages = D <= 128 ? 5 : 3;
+    static constexpr int kKvStages = D <= 128 ? 4 : 3;
     static constexpr int kKvChunkBytes = BN * 128;      // one 64-column chunk of a key block
     static constexpr int kKvBytes = kQChunks * kKvChunkBytes;
     static constexpr int kTmemO = 2 * BN;               // column of the (first) O accumulator
     // d = 128 leaves 128 tensor-memory columns free: a second O accumulator, and four more warps that normalise and store
     // a finished tile while the softmax warps and the MMAs are already on the next one
     static constexpr bool kSplitEpi = D <= 128;
-    static constexpr int kThreads = kSplitEpi ? 352 : 224;
-    static constexpr size_t kSmem = 1024 + kQBufs * kQBytes + kKvStages * kKvBytes + 1536;
+    // softmax warps per quarter of the rows, each with its share of a block's keys: one warp alone leaves its scheduler
+    // idle through every tensor-memory round trip and hand-over
+    static constexpr int kHalves = D <= 128 ? 2 : 1;
+    static constexpr int kSoftWarps = 4 * kHalves;
+    static constexpr int kMmaWarp = kSoftWarps, kTmaWarp = kSoftWarps + 1, kGatherWarp = kSoftWarps + 2;
+    static constexpr int kEpiWarp0 = kSoftWarps + 3;   // first of the four output warps (kSplitEpi)
+    static constexpr int kThreads = (kSoftWarps + 3 + (kSplitEpi ? 4 : 0)) * 32;
+    // barriers and the tensor-memory slot; row sums [2 tiles][kHalves][128]; block maxima [2 blocks][2][128]
+    static constexpr int kMisc = 512 + (kSplitEpi ? 2 * kHalves * 512 : 0) + (kHalves == 2 ? 2048 : 0);
+    static constexpr size_t kSmem = 1024 + kQBufs * kQBytes + kKvStages * kKvBytes + kMisc;
 };
 
 // One tile of the launch as every role needs it.
@@ -101,7 +108,8 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
     uint64_t *q_first = l_ready + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_first + 1);
     volatile uint32_t *abort_flag = tmem_slot + 1;
-    float *l_s = reinterpret_cast<float *>(tmem_slot + 4);   // [2][128] row sums handed to the epilogue warps
+    float *l_s = reinterpret_cast<float *>(tmem_slot + 4);   // [2][kHalves][128] row sums handed to the output warps
+    float *mx_s = l_s + (kSplit ? 2 * C::kHalves * 128 : 0);    // [2][2][128] block maxima exchanged between partner warps
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -112,7 +120,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(s_full + b), 1);
-            mbar_init(smem_u32(p_full + b), 128);
+            mbar_init(smem_u32(p_full + b), C::kSoftWarps * 32);
             mbar_init(smem_u32(pv_done + b), 1);
             mbar_init(smem_u32(q_full + b), 32);
             mbar_init(smem_u32(q_empty + b), 5);   // the last Q K^T of the tenant, and the four softmax warps' output staging
@@ -120,13 +128,13 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(o_final + b), 1);
             mbar_init(smem_u32(o_free + b), 128);
-            mbar_init(smem_u32(l_ready + b), 128);
+            mbar_init(smem_u32(l_ready + b), C::kSoftWarps * 32);
         }
-        mbar_init(smem_u32(q_first), 128);
+        mbar_init(smem_u32(q_first), C::kSoftWarps * 32);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == kAttMmaWarp) tmem_alloc(smem_u32(tmem_slot), 512);
+    if (warp == C::kMmaWarp) tmem_alloc(smem_u32(tmem_slot), 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -210,22 +218,26 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
         }
     };
 
-    if (warp < 4) {
+    if (warp < C::kSoftWarps) {
         // ===================== softmax, output =====================
-        const int row = warp * 32 + lane;
-        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        // kH warps share a quarter of the rows (the tensor-memory lanes 32 wq ...): each takes CW of a block's BN keys.
+        constexpr int kH = C::kHalves, CW = BN / kH;
+        const int wq = warp & 3, half = warp >> 2;
+        const int row = wq * 32 + lane;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(wq * 32) << 16);
         const float k2 = p.scale_log2;
         bool ok = true;
+        bool late = false;   // kH = 2: a wait failed where the partner warp cannot see it; both leave at the next pair barrier
         uint32_t gb = 0;     // key blocks processed so far by this CTA (all tiles): selects score / P buffers and phases
         int k = 0;           // tiles processed so far
         if ((int)blockIdx.x < n_tiles) {
-            // The CTA's first tile has nobody to prefetch it: these four warps, idle until the first scores arrive, gather
+            // The CTA's first tile has nobody to prefetch it: these warps, idle until the first scores arrive, gather
             // its queries (8 threads per row, 16 bytes each per 128-byte chunk); later tiles come from the gather warp.
             const AttTile t = att_tile<BN>(p, blockIdx.x);
             const int sub = tid & 7, r0 = tid >> 3;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int r = r0 + 16 * i;
+            for (int i = 0; i < 8 / kH; ++i) {
+                const int r = r0 + 16 * kH * i;
                 int id = -1;
                 if (r < t.cnt) {
                     id = p.sl.ids[t.pos0 + r];
@@ -245,80 +257,107 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
             for (int j = 0; j < t.nb; ++j, ++gb) {
                 const int b = (int)(gb & 1u);
                 const int valid_cols = min(BN, L - j * BN);
-                if (!mbar_wait(smem_u32(s_full + b), (gb >> 1) & 1u, abort_flag)) {
+                const int vc = min(CW, valid_cols - half * CW);   // this warp's keys of the block that exist (may be <= 0)
+                const bool got = __all_sync(0xffffffffu, mbar_wait(smem_u32(s_full + b), (gb >> 1) & 1u, abort_flag));
+                const uint32_t ts = lane_base + (uint32_t)(b * BN);
+                // the row's CW scores: all loads first, one wait
+                uint32_t sc[CW];
+                float mt = -INFINITY;
+                if (got) {
+                    tc_fence_after();
+#pragma unroll
+                    for (int c0 = 0; c0 < CW; c0 += 32)
+                        tmem_ld32(ts + (uint32_t)(half * CW + c0), *reinterpret_cast<uint32_t(*)[32]>(&sc[c0]));
+                    tmem_ld_wait();
+                    // block maximum of the row (four independent chains)
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                    if (vc == CW) {
+#pragma unroll
+                        for (int i = 0; i < CW; i += 8) {   // three-input maxima: two scores per instruction
+                            mx4[0] = fmax3(mx4[0], __uint_as_float(sc[i]), __uint_as_float(sc[i + 1]));
+                            mx4[1] = fmax3(mx4[1], __uint_as_float(sc[i + 2]), __uint_as_float(sc[i + 3]));
+                            mx4[2] = fmax3(mx4[2], __uint_as_float(sc[i + 4]), __uint_as_float(sc[i + 5]));
+                            mx4[3] = fmax3(mx4[3], __uint_as_float(sc[i + 6]), __uint_as_float(sc[i + 7]));
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < CW; ++i)
+                            if (i < vc) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sc[i]));
+                    }
+                    mt = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * k2;
+                }
+                if (kH == 2) {
+                    // The two warps of a row quarter agree on the block maximum through shared memory (two buffers: the
+                    // partner may still read block gb - 1's value).  The barrier also orders this warp's score loads
+                    // before the partner's probability stores, which for the second half land in the first half's columns.
+                    float *mx = mx_s + (gb & 1u) * 256;
+                    mx[half * 128 + row] = mt;
+                    tc_fence_before();
+                    const bool bad = named_bar_or(1 + wq, 64, !got || late);
+                    tc_fence_after();
+                    if (bad) {
+                        ok = false;
+                        break;
+                    }
+                    mt = fmaxf(mt, mx[(half ^ 1) * 128 + row]);
+                } else if (!got) {
                     ok = false;
                     break;
                 }
-                tc_fence_after();
-                const uint32_t ts = lane_base + (uint32_t)(b * BN);
-                // the row's BN scores: all loads first, one wait
-                uint32_t sc[BN];
-#pragma unroll
-                for (int c0 = 0; c0 < BN; c0 += 32) tmem_ld32(ts + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[32]>(&sc[c0]));
-                tmem_ld_wait();
-                // block maximum of the row (four independent chains)
-                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                if (valid_cols == BN) {
-#pragma unroll
-                    for (int i = 0; i < BN; i += 8) {   // three-input maxima: two scores per instruction
-                        mx4[0] = fmax3(mx4[0], __uint_as_float(sc[i]), __uint_as_float(sc[i + 1]));
-                        mx4[1] = fmax3(mx4[1], __uint_as_float(sc[i + 2]), __uint_as_float(sc[i + 3]));
-                        mx4[2] = fmax3(mx4[2], __uint_as_float(sc[i + 4]), __uint_as_float(sc[i + 5]));
-                        mx4[3] = fmax3(mx4[3], __uint_as_float(sc[i + 6]), __uint_as_float(sc[i + 7]));
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < BN; ++i)
-                        if (i < valid_cols) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sc[i]));
-                }
-                const float mt = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * k2;
                 if (j == 0) {
                     m_used = mt;
                 } else {
                     const bool need = mt > m_used + 8.0f;
                     if (__any_sync(0xffffffffu, need)) {
-                        // raise the running maximum and rescale this warp's rows of O (rare)
+                        // raise the running maximum and rescale this warp's share of its rows of O (rare)
                         const float m_new = need ? mt : m_used;
                         const float f = fast_exp2(m_used - m_new);
                         l_sum *= f;
                         m_used = m_new;
-                        if (!mbar_wait(smem_u32(pv_done + ((gb - 1) & 1u)), ((gb - 1) >> 1) & 1u, abort_flag)) {
-                            ok = false;
-                            break;
-                        }
-                        tc_fence_after();
+                        const bool pv = __all_sync(0xffffffffu, mbar_wait(smem_u32(pv_done + ((gb - 1) & 1u)),
+                                                                           ((gb - 1) >> 1) & 1u, abort_flag));
+                        if (!pv) {
+                            if (kH == 2) {
+                                late = true;
+                            } else {
+                                ok = false;
+                                break;
+                            }
+                        } else {
+                            tc_fence_after();
 #pragma unroll 1
-                        for (int c0 = 0; c0 < D; c0 += 32) {
-                            uint32_t r[32];
-                            const uint32_t oc = (uint32_t)(C::kTmemO + (kSplit ? (k & 1) * D : 0) + c0);
-                            tmem_ld32(lane_base + oc, r);
-                            tmem_ld_wait();
+                            for (int c0 = half * (D / kH); c0 < (half + 1) * (D / kH); c0 += 32) {
+                                uint32_t r[32];
+                                const uint32_t oc = (uint32_t)(C::kTmemO + (kSplit ? (k & 1) * D : 0) + c0);
+                                tmem_ld32(lane_base + oc, r);
+                                tmem_ld_wait();
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
-                            tmem_st32(lane_base + oc, r);
+                                for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+                                tmem_st32(lane_base + oc, r);
+                            }
+                            tmem_st_wait();
                         }
-                        tmem_st_wait();
                     }
                 }
                 // probabilities -> packed bf16 pairs over the first BN / 2 columns of the score buffer just read (P V of
                 // block gb - 2, the buffer's previous reader, precedes the Q K^T that refilled it in the MMA pipe)
                 float ls4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int c0 = 0; c0 < BN; c0 += 64) {
+                for (int c0 = 0; c0 < CW; c0 += 64) {
                     uint32_t packed[32];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         float p0 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i]), k2, -m_used));
                         float p1 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i + 1]), k2, -m_used));
-                        if (valid_cols != BN) {
-                            if (c0 + 2 * i >= valid_cols) p0 = 0.f;
-                            if (c0 + 2 * i + 1 >= valid_cols) p1 = 0.f;
+                        if (vc != CW) {
+                            if (c0 + 2 * i >= vc) p0 = 0.f;
+                            if (c0 + 2 * i + 1 >= vc) p1 = 0.f;
                         }
                         ls4[i & 3] += p0 + p1;
                         const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                         packed[i] = *reinterpret_cast<const uint32_t *>(&h);
                     }
-                    tmem_st32(ts + (uint32_t)(c0 >> 1), packed);
+                    tmem_st32(ts + (uint32_t)((half * CW + c0) >> 1), packed);
                 }
                 tmem_st_wait();
                 l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
@@ -327,13 +366,17 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
             }
             if (!ok) break;
             if (kSplit) {
-                // hand the row sums to the epilogue warps and go on with the next tile.  l_s[k & 1] was last read by the
-                // epilogue of tile k - 2, before that epilogue released its O accumulator.
-                if (k >= 2 && !mbar_wait(smem_u32(o_free + (k & 1)), (uint32_t)(((k - 2) >> 1) & 1), abort_flag)) {
+                // hand the row sums to the output warps and go on with the next tile.  l_s[k & 1] was last read by the
+                // output of tile k - 2, before it released that O accumulator.
+                if (k >= 2 && !__all_sync(0xffffffffu, mbar_wait(smem_u32(o_free + (k & 1)), (uint32_t)(((k - 2) >> 1) & 1), abort_flag))) {
+                    if (kH == 2) {
+                        late = true;
+                        continue;
+                    }
                     ok = false;
                     break;
                 }
-                l_s[(k & 1) * 128 + row] = l_sum;
+                l_s[((k & 1) * kH + half) * 128 + row] = l_sum;
                 mbar_arrive(smem_u32(l_ready + (k & 1)));
             } else {
                 if (!mbar_wait(smem_u32(o_final), (uint32_t)(k & 1), abort_flag)) {
@@ -345,7 +388,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
             }
         }
         if (lane == 0) bulk_wait<0>();   // all tile stores of this warp have reached global memory
-    } else if (warp == kAttMmaWarp) {
+    } else if (warp == C::kMmaWarp) {
         // ===================== MMA issuer =====================
         if (lane == 0) {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(kTcTile, BN);
@@ -432,7 +475,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
             }
         }
         __syncwarp();
-    } else if (warp == kAttTmaWarp) {
+    } else if (warp == C::kTmaWarp) {
         // ===================== key/value producer (TMA) =====================
         if (lane == 0) {
             uint32_t gb = 0;
@@ -454,7 +497,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
             }
         }
         __syncwarp();
-    } else if (kSplit && warp >= 7) {
+    } else if (kSplit && warp >= C::kEpiWarp0) {
         // ===================== output of finished tiles (d = 128: 128 threads) =====================
         const int wq = warp & 3;   // the quarter of the tensor-memory lanes this warp may read
         int k = 0;
@@ -463,13 +506,15 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
             const int b = k & 1;
             const uint32_t parity = (uint32_t)((k >> 1) & 1);
             if (!mbar_wait(smem_u32(l_ready + b), parity, abort_flag)) break;
-            const float l_sum = l_s[b * 128 + wq * 32 + lane];
+            float l_sum = 0.f;
+#pragma unroll
+            for (int h = 0; h < C::kHalves; ++h) l_sum += l_s[(b * C::kHalves + h) * 128 + wq * 32 + lane];
             if (!mbar_wait(smem_u32(o_final + b), parity, abort_flag)) break;
             tc_fence_after();
             tile_epilogue(k, t, l_sum, wq, lane);
         }
         if (lane == 0) bulk_wait<0>();   // all tile stores of this warp have reached global memory
-    } else if (warp == 6) {
+    } else if (warp == C::kGatherWarp) {
         // ===================== query gather (32 threads) =====================
         // 8 threads per row (16 bytes each per 128-byte chunk), rows lane / 8 + 4 i, 128B-swizzled K-major chunks
         const int sub = lane & 7, r0 = lane >> 3;
@@ -513,7 +558,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == kAttMmaWarp) tmem_dealloc(tmem_base, 512);
+    if (warp == C::kMmaWarp) tmem_dealloc(tmem_base, 512);
 }
 
 // ---- long sequences ------------------------------------------------------------------------------------------
