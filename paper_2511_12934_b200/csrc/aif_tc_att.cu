@@ -950,12 +950,14 @@ cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
     p.sl = sl, p.E = (const uint8_t *)ctx->E, p.M = c.M, p.mini_batch = c.mini_batch;
     p.x_stride = x_stride, p.X = (__nv_bfloat16 *)X;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.d);
-    // One CTA per SM walking over many tiles saves the per-tile set-up and prefetches the next tile's queries, but its
-    // static tile assignment loses to the hardware's dynamic CTA scheduling when an SM gets only a few tiles (8.4 tiles
-    // per SM cost 9 tile times everywhere): below 16 tiles per SM every tile gets a CTA of its own.
-    const int grid = sl.n_tiles >= 148 * 16 ? 148 : sl.n_tiles;
+    // One CTA per SM walking over its tiles hides a tile's query gather and output behind its neighbours' key blocks:
+    // 22 k against 31 k cycles per 8-block tile, which outweighs the static assignment's rounding (8.5 tiles per SM cost
+    // 9 tile times) as soon as some SM has two tiles.  Tiles of many key blocks have little to hide and lose only the
+    // rounding: up to 16 tiles per SM they get a CTA each, in the two-group kernel.
+    const bool long_tiles = c.d == 128 && sl.max_L >= 16 * 128 && sl.n_tiles < 148 * 16;
+    const int grid = sl.n_tiles > 148 && !long_tiles ? 148 : sl.n_tiles;
     cudaError_t e;
-    if (c.d == 128 && grid == sl.n_tiles && sl.max_L >= 16 * 128)   // one CTA per tile and many key blocks per tile
+    if (long_tiles)
         e = launch_pdl(k_att_tc_long, dim3(grid), dim3(kAtt2Threads), kAtt2Smem, st, pl->tmap, p);
     else if (c.d == 128)
         e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(AttCfg<128, 128>::kThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, tmap_x, p);
@@ -981,9 +983,10 @@ cudaError_t launch_self_att_tc(const aif_ctx *ctx, int slot_index, int L, cudaSt
     CUtensorMap tmap_x;
     cudaError_t ex = encode_x_map(&tmap_x, pl->self_rows, c.d, (size_t)c.L_max + kTcTile);
     if (ex != cudaSuccess) return ex;
-    const int grid = sl.n_tiles >= 148 * 16 ? 148 : sl.n_tiles;
+    const bool long_tiles = c.d == 128 && sl.max_L >= 16 * 128 && sl.n_tiles < 148 * 16;   // as in launch_att_tc
+    const int grid = sl.n_tiles > 148 && !long_tiles ? 148 : sl.n_tiles;
     cudaError_t e;
-    if (c.d == 128 && grid == sl.n_tiles && sl.max_L >= 16 * 128)   // one CTA per tile and many key blocks per tile
+    if (long_tiles)
         e = launch_pdl(k_att_tc_long, dim3(grid), dim3(kAtt2Threads), kAtt2Smem, st, pl->tmap, p);
     else if (c.d == 128)
         e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(AttCfg<128, 128>::kThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, tmap_x, p);
