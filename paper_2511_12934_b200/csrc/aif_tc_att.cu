@@ -2,20 +2,20 @@
 // candidates against the request's projected behaviour sequence S [L x d] (Section 4.2, first paragraph: similarity
 // of the target item with every historical item, then pooling; here in its dense softmax form).
 //
-// Persistent kernel: one CTA per SM walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  224 threads (d = 256)
-// or 352 (d = 128):
-//   warps 0-3  per key block: read the score row from TMEM into registers, online softmax in fp32 (one thread per
-//              candidate row), write the probabilities back into the same TMEM columns as packed bf16 pairs (the A
-//              operand of P V is read from tensor memory, which keeps it off the shared-memory bandwidth the products
-//              are bound by); at the end of a tile normalise O and store the attention rows (d = 256) or hand the
-//              row sums to warps 7-10 (d = 128)
-//   warp  4    allocates TMEM; one lane issues tcgen05.mma over the flat sequence of key blocks of all its tiles:
-//              scores = Q K^T (both K-major) one block ahead of O += P V, with V read from the very same shared-memory
-//              tile as K, as an MN-major B operand
-//   warp  5    one lane streams key/value blocks of S with TMA (3-D tensor map over the user-state arena)
-//   warp  6    gathers the item rows of the next tile (the queries) with cp.async while the current tile is processed
+// One CTA per SM walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ... (or one CTA per tile when no SM has two).
+// Warps at d = 128 (512 threads; d = 256 in brackets, 256 threads):
+//   0-7 [0-3]  softmax: per key block read the score row from TMEM into registers, exponentials in fp32, and write the
+//              probabilities back into the same TMEM columns as packed bf16 pairs (the A operand of P V is read from
+//              tensor memory and never crosses shared memory).  A thread owns a candidate row; at d = 128 two warps
+//              share each quarter of the rows, each with half of a block's keys, and agree on the block maximum through
+//              shared memory.  At the end of a tile: hand the row sums to the output warps (d = 128) or normalise O and
+//              store the attention rows themselves (d = 256)
+//   8  [4]     allocates TMEM; one lane issues scores = Q K^T (both K-major) up to two blocks ahead of the softmax
+//   9  [5]     one lane streams key/value blocks of S with TMA (3-D tensor map over the user-state arena)
+//   10 [6]     gathers the item rows of the next tile (the queries) with cp.async while the current tile is processed
 //              (two query buffers)
-//   warps 7-10 d = 128 only: normalise the finished tile's O accumulator and store its rows while the other warps are
+//   11 [7]     one lane issues O += P V, with V read from the very same shared-memory tile as K, as an MN-major B operand
+//   12-15      d = 128 only: normalise the finished tile's O accumulator and store its rows while the other warps are
 //              on the next tile (two O accumulators fill the 512 tensor-memory columns)
 // TMEM: two score buffers (so the softmax of block j overlaps Q K^T of block j+1) and the O accumulator.
 // The running maximum is only raised when a row's block maximum exceeds it by more than 8 (in the log2 domain);
@@ -56,8 +56,9 @@ struct AttCfg {
     static constexpr int kHalves = D <= 128 ? 2 : 1;
     static constexpr int kSoftWarps = 4 * kHalves;
     static constexpr int kMmaWarp = kSoftWarps, kTmaWarp = kSoftWarps + 1, kGatherWarp = kSoftWarps + 2;
-    static constexpr int kEpiWarp0 = kSoftWarps + 3;   // first of the four output warps (kSplitEpi)
-    static constexpr int kThreads = (kSoftWarps + 3 + (kSplitEpi ? 4 : 0)) * 32;
+    static constexpr int kPvWarp = kSoftWarps + 3;     // issues the P V products (kMmaWarp: Q K^T, and owns tensor memory)
+    static constexpr int kEpiWarp0 = kSoftWarps + 4;   // first of the four output warps (kSplitEpi)
+    static constexpr int kThreads = (kSoftWarps + 4 + (kSplitEpi ? 4 : 0)) * 32;
     // barriers and the tensor-memory slot; row sums [2 tiles][kHalves][128]; block maxima [2 blocks][2][128]
     static constexpr int kMisc = 512 + (kSplitEpi ? 2 * kHalves * 512 : 0) + (kHalves == 2 ? 2048 : 0);
     static constexpr size_t kSmem = 1024 + kQBufs * kQBytes + kKvStages * kKvBytes + kMisc;
@@ -388,13 +389,14 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
             }
         }
         if (lane == 0) bulk_wait<0>();   // all tile stores of this warp have reached global memory
-    } else if (warp == C::kMmaWarp) {
-        // ===================== MMA issuer =====================
+    } else if (warp == C::kMmaWarp || warp == C::kPvWarp) {
+        // ===================== MMA issuers =====================
+        // One lane of one warp issues the Q K^T products, one lane of another the P V products: a single issuer spends
+        // more time in its waits, fences and commits than the sixteen products of a key block take, and the tensor pipe
+        // idles meanwhile.  Each walks the flat sequence of key blocks of this CTA's tiles with a cursor of its own.
         if (lane == 0) {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(kTcTile, BN);
             constexpr uint32_t idesc_pv = umma_idesc_bf16_bmn(kTcTile, D);
-            bool ok = true;
-            // two cursors over the flat sequence of key blocks of this CTA's tiles: Q K^T runs one block ahead of P V
             struct Cursor {
                 int tile, k, j, nb;
                 uint32_t gb;
@@ -412,66 +414,62 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
                     open_tile(c);
                 }
             };
-            // operand descriptors of buffer / stage 0; the others lie a fixed number of 16-byte units further
-            const uint64_t qdesc0 = umma_desc_sw128(smem_u32(smQ)), kdesc0 = umma_desc_sw128(smem_u32(smKV));
-            const uint64_t vdesc0 = umma_desc_mn_sw128(smem_u32(smKV), C::kKvChunkBytes);
-            Cursor cq{(int)blockIdx.x, 0, 0, 0, 0u, 0}, cp{(int)blockIdx.x, 0, 0, 0, 0u, 0};
-            cq.nb_next = blocks_of(cq.tile);
-            open_tile(cq);
-            cp.nb = cq.nb, cp.nb_next = cq.nb_next;
-            auto issue_qk = [&]() -> bool {
-                const int qb = cq.k % kQB;
-                if (cq.j == 0) {   // first block of a tile: its queries must have landed (cp.async, generic proxy)
-                    const bool got = cq.k == 0 ? mbar_wait(smem_u32(q_first), 0u, abort_flag)
-                                               : mbar_wait(smem_u32(q_full + qb), (uint32_t)(((cq.k - 1) / kQB) & 1), abort_flag);
-                    if (!got) return false;
-                    fence_proxy_async();
-                }
-                const int s = (int)(cq.gb % kS);
-                if (!mbar_wait(smem_u32(kv_full + s), (cq.gb / kS) & 1u, abort_flag)) return false;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)((cq.gb & 1u) * BN);
-                const uint64_t qd = qdesc0 + (uint64_t)(uint32_t)(qb * (C::kQBytes >> 4));
-                const uint64_t kd = kdesc0 + (uint64_t)(uint32_t)(s * (C::kKvBytes >> 4));
-                umma_bf16(d_tmem, qd, kd, idesc_qk, 0u);
+            Cursor c{(int)blockIdx.x, 0, 0, 0, 0u, 0};
+            c.nb_next = blocks_of(c.tile);
+            open_tile(c);
+            bool ok = true;
+            if (warp == C::kMmaWarp) {
+                // scores of block gb into buffer gb & 1, up to two blocks ahead of the softmax
+                // operand descriptors of buffer / stage 0; the others lie a fixed number of 16-byte units further
+                const uint64_t qdesc0 = umma_desc_sw128(smem_u32(smQ)), kdesc0 = umma_desc_sw128(smem_u32(smKV));
+                while (ok && c.tile < n_tiles) {
+                    const int qb = c.k % kQB;
+                    if (c.j == 0) {   // first block of a tile: its queries must have landed (cp.async, generic proxy)
+                        ok = c.k == 0 ? mbar_wait(smem_u32(q_first), 0u, abort_flag)
+                                      : mbar_wait(smem_u32(q_full + qb), (uint32_t)(((c.k - 1) / kQB) & 1), abort_flag);
+                        if (!ok) break;
+                        fence_proxy_async();
+                    }
+                    const int s = (int)(c.gb % kS);
+                    if (!mbar_wait(smem_u32(kv_full + s), (c.gb / kS) & 1u, abort_flag)) break;
+                    // the buffer's previous content, the probabilities of block gb - 2, must have been consumed by its P V
+                    if (c.gb >= 2 && !mbar_wait(smem_u32(pv_done + (c.gb & 1u)), ((c.gb - 2) >> 1) & 1u, abort_flag)) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)((c.gb & 1u) * BN);
+                    const uint64_t qd = qdesc0 + (uint64_t)(uint32_t)(qb * (C::kQBytes >> 4));
+                    const uint64_t kd = kdesc0 + (uint64_t)(uint32_t)(s * (C::kKvBytes >> 4));
+                    umma_bf16(d_tmem, qd, kd, idesc_qk, 0u);
 #pragma unroll
-                for (int kk = 1; kk < D / 16; ++kk)
-                    umma_bf16_acc(d_tmem, qd + (uint64_t)((kk >> 2) * (16384 >> 4) + 2 * (kk & 3)),
-                                  kd + (uint64_t)((kk >> 2) * (C::kKvChunkBytes >> 4) + 2 * (kk & 3)), idesc_qk);
-                umma_commit(smem_u32(s_full + (cq.gb & 1u)));
-                if (cq.j == cq.nb - 1) umma_commit(smem_u32(q_empty + qb));   // the tile's queries are no longer needed
-                advance(cq);
-                return true;
-            };
-            if (cq.tile < n_tiles) ok = issue_qk();
-            while (ok && cp.tile < n_tiles) {
-                if (cq.tile < n_tiles && !issue_qk()) {
-                    ok = false;
-                    break;
+                    for (int kk = 1; kk < D / 16; ++kk)
+                        umma_bf16_acc(d_tmem, qd + (uint64_t)((kk >> 2) * (16384 >> 4) + 2 * (kk & 3)),
+                                      kd + (uint64_t)((kk >> 2) * (C::kKvChunkBytes >> 4) + 2 * (kk & 3)), idesc_qk);
+                    umma_commit(smem_u32(s_full + (c.gb & 1u)));
+                    if (c.j == c.nb - 1) umma_commit(smem_u32(q_empty + qb));   // the tile's queries are no longer needed
+                    advance(c);
                 }
-                if (!mbar_wait(smem_u32(p_full + (cp.gb & 1u)), (cp.gb >> 1) & 1u, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-                // the first P V of a tile overwrites O: the previous tile's output must have been read
-                if (cp.j == 0 && (kSplit ? cp.k >= 2 && !mbar_wait(smem_u32(o_free + (cp.k & 1)), (uint32_t)(((cp.k - 2) >> 1) & 1), abort_flag)
-                                         : cp.k > 0 && !mbar_wait(smem_u32(o_free), (uint32_t)((cp.k - 1) & 1), abort_flag))) {
-                    ok = false;
-                    break;
-                }
-                tc_fence_after();
-                const int s = (int)(cp.gb % kS);
-                const uint32_t o_tmem = tmem_base + (uint32_t)(C::kTmemO + (kSplit ? (cp.k & 1) * D : 0));
-                const uint32_t p_tmem = tmem_base + (uint32_t)((cp.gb & 1u) * BN);   // P: 8 columns per 16 keys
-                const uint64_t vd = vdesc0 + (uint64_t)(uint32_t)(s * (C::kKvBytes >> 4));
+            } else {
+                // O += P V of block gb as soon as its probabilities are in tensor memory
+                const uint64_t vdesc0 = umma_desc_mn_sw128(smem_u32(smKV), C::kKvChunkBytes);
+                while (ok && c.tile < n_tiles) {
+                    if (!mbar_wait(smem_u32(p_full + (c.gb & 1u)), (c.gb >> 1) & 1u, abort_flag)) break;
+                    // the first P V of a tile overwrites O: the output of the accumulator's previous tile must have been read
+                    if (c.j == 0 && (kSplit ? c.k >= 2 && !mbar_wait(smem_u32(o_free + (c.k & 1)), (uint32_t)(((c.k - 2) >> 1) & 1), abort_flag)
+                                            : c.k > 0 && !mbar_wait(smem_u32(o_free), (uint32_t)((c.k - 1) & 1), abort_flag)))
+                        break;
+                    tc_fence_after();
+                    const int s = (int)(c.gb % kS);
+                    const uint32_t o_tmem = tmem_base + (uint32_t)(C::kTmemO + (kSplit ? (c.k & 1) * D : 0));
+                    const uint32_t p_tmem = tmem_base + (uint32_t)((c.gb & 1u) * BN);   // P: 8 columns per 16 keys
+                    const uint64_t vd = vdesc0 + (uint64_t)(uint32_t)(s * (C::kKvBytes >> 4));
 #pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk)   // V: 16 keys further = 16 rows x 128 bytes
-                    umma_bf16_ts(o_tmem, p_tmem + (uint32_t)(kk * 8), vd + (uint64_t)(kk * (2048 >> 4)), idesc_pv,
-                                 (cp.j > 0 || kk > 0) ? 1u : 0u);
-                umma_commit(smem_u32(pv_done + (cp.gb & 1u)));
-                umma_commit(smem_u32(kv_empty + s));
-                if (cp.j == cp.nb - 1) umma_commit(smem_u32(o_final + (kSplit ? (cp.k & 1) : 0)));
-                advance(cp);
+                    for (int kk = 0; kk < BN / 16; ++kk)   // V: 16 keys further = 16 rows x 128 bytes
+                        umma_bf16_ts(o_tmem, p_tmem + (uint32_t)(kk * 8), vd + (uint64_t)(kk * (2048 >> 4)), idesc_pv,
+                                     (c.j > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(smem_u32(pv_done + (c.gb & 1u)));
+                    umma_commit(smem_u32(kv_empty + s));   // Q K^T of the block, the stage's other reader, completed long ago
+                    if (c.j == c.nb - 1) umma_commit(smem_u32(o_final + (kSplit ? (c.k & 1) : 0)));
+                    advance(c);
+                }
             }
         }
         __syncwarp();
