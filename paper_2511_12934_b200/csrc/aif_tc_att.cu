@@ -559,297 +559,6 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
     if (warp == C::kMmaWarp) tmem_dealloc(tmem_base, 512);
 }
 
-// ---- long sequences ------------------------------------------------------------------------------------------
-// Variant for tiles with many key blocks (d = 128, one CTA per tile, 320 threads).  Two softmax groups of four warps
-// take the even and the odd key blocks, each with its own running maximum, sum and O accumulator in TMEM (merged
-// once at the end), so that the exponentials of one group (XU pipe) overlap the other arithmetic of the other.  The
-// MMA lane issues whichever product is ready: Q K^T of block j + 2 once P V of block j has been issued (P aliases the
-// score buffer), P V as soon as the probabilities are written.  A key/value stage stays occupied from its load until
-// P V of its block, a span that covers two blocks in softmax, so the ring has six stages.
-constexpr int kAtt2Threads = 320;
-constexpr int kAtt2MmaWarp = 8;
-constexpr int kAtt2Stages = 6;
-constexpr size_t kAtt2Smem = 1024 + 32768 + kAtt2Stages * 32768 + 512;
-
-__global__ void __launch_bounds__(kAtt2Threads, 1) k_att_tc_long(const __grid_constant__ CUtensorMap tmapS, const AttParams p)
-{
-    constexpr int D = 128, BN = 128, kS = kAtt2Stages, kKvBytes = 32768, kKvChunkBytes = 16384, kTmemO = 256;
-    extern __shared__ unsigned char smem_dyn[];
-    unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-    unsigned char *smQ = base;
-    unsigned char *smKV = smQ + 32768;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smKV + kS * kKvBytes);
-    uint64_t *kv_full = bars, *kv_empty = bars + kS;
-    uint64_t *s_full = bars + 2 * kS, *p_full = s_full + 2, *pv_done = p_full + 2;
-    uint64_t *q_full = pv_done + 2, *o_final = q_full + 1, *merge_bar = o_final + 1;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(merge_bar + 1);
-    volatile uint32_t *abort_flag = tmem_slot + 1;
-    float *ml_s = reinterpret_cast<float *>(smQ);   // [group][m, l][128 rows]; the queries are no longer needed once O is final
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) {
-        for (int s = 0; s < kS; ++s) {
-            mbar_init(smem_u32(kv_full + s), 1);
-            mbar_init(smem_u32(kv_empty + s), 1);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(s_full + b), 1);
-            mbar_init(smem_u32(p_full + b), 128);
-            mbar_init(smem_u32(pv_done + b), 1);
-        }
-        mbar_init(smem_u32(q_full), 256);
-        mbar_init(smem_u32(o_final), 1);
-        mbar_init(smem_u32(merge_bar), 256);
-        *abort_flag = 0u;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == kAtt2MmaWarp) tmem_alloc(smem_u32(tmem_slot), 512);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-    grid_dep_launch();
-    grid_dep_wait();
-    const AttTile t = att_tile<BN>(p, blockIdx.x);
-    const int L = t.L, nb = t.nb;
-
-    if (warp < kAtt2MmaWarp) {
-        // ===================== queries, softmax, output =====================
-        const int grp = warp >> 2;                    // key blocks j with j % 2 == grp; score buffer and O accumulator grp
-        const int row = (warp & 3) * 32 + lane;       // TMEM lane = candidate row
-        {   // gather the tile's item rows: 8 threads per row, 16 bytes each per 128-byte chunk, 128B-swizzled K-major
-            const int sub = tid & 7, r0 = tid >> 3;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int r = r0 + 32 * i;
-                int id = -1;
-                if (r < t.cnt) {
-                    id = p.sl.ids[t.pos0 + r];
-                    if (id < 0 || (int64_t)id >= p.M) id = -1;
-                }
-                const uint8_t *g = p.E + (id >= 0 ? (size_t)id * (D * 2) + sub * 16 : 0);
-                const uint32_t dst = smem_u32(smQ) + (uint32_t)(r * 128) + (uint32_t)((sub ^ (r & 7)) << 4);
-                cp_async16(dst, g, id >= 0 ? 16u : 0u);
-                cp_async16(dst + 16384, g + 128, id >= 0 ? 16u : 0u);
-            }
-            cp_async_arrive_noinc(smem_u32(q_full));
-        }
-        const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-        const uint32_t ts = lane_base + (uint32_t)(grp * BN);
-        const uint32_t o_col = (uint32_t)(kTmemO + grp * D);
-        const float k2 = p.scale_log2;
-        float m_used = -INFINITY, l_sum = 0.f;
-        bool ok = true;
-        for (int j = grp; j < nb; j += 2) {
-            const uint32_t ph = (uint32_t)((j >> 1) & 1);
-            const int valid_cols = min(BN, L - j * BN);
-            if (!mbar_wait(smem_u32(s_full + grp), ph, abort_flag)) {
-                ok = false;
-                break;
-            }
-            tc_fence_after();
-            uint32_t sc[BN];
-#pragma unroll
-            for (int c0 = 0; c0 < BN; c0 += 32) tmem_ld32(ts + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[32]>(&sc[c0]));
-            tmem_ld_wait();
-            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            if (valid_cols == BN) {
-#pragma unroll
-                for (int i = 0; i < BN; i += 8) {   // three-input maxima: two scores per instruction
-                    mx4[0] = fmax3(mx4[0], __uint_as_float(sc[i]), __uint_as_float(sc[i + 1]));
-                    mx4[1] = fmax3(mx4[1], __uint_as_float(sc[i + 2]), __uint_as_float(sc[i + 3]));
-                    mx4[2] = fmax3(mx4[2], __uint_as_float(sc[i + 4]), __uint_as_float(sc[i + 5]));
-                    mx4[3] = fmax3(mx4[3], __uint_as_float(sc[i + 6]), __uint_as_float(sc[i + 7]));
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < BN; ++i)
-                    if (i < valid_cols) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sc[i]));
-            }
-            const float mt = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * k2;
-            if (j < 2) {
-                m_used = mt;
-            } else {
-                const bool need = mt > m_used + 8.0f;
-                if (__any_sync(0xffffffffu, need)) {   // raise the running maximum, rescale this warp's rows of O (rare)
-                    const float m_new = need ? mt : m_used;
-                    const float f = fast_exp2(m_used - m_new);
-                    l_sum *= f;
-                    m_used = m_new;
-                    // this group's previous block (j - 2) must have been accumulated into its O
-                    if (!mbar_wait(smem_u32(pv_done + grp), ph ^ 1u, abort_flag)) {
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after();
-#pragma unroll 1
-                    for (int c0 = 0; c0 < D; c0 += 32) {
-                        uint32_t r[32];
-                        tmem_ld32(lane_base + o_col + (uint32_t)c0, r);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
-                        tmem_st32(lane_base + o_col + (uint32_t)c0, r);
-                    }
-                    tmem_st_wait();
-                }
-            }
-            float ls4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int c0 = 0; c0 < BN; c0 += 64) {
-                uint32_t packed[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    float p0 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i]), k2, -m_used));
-                    float p1 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i + 1]), k2, -m_used));
-                    if (valid_cols != BN) {
-                        if (c0 + 2 * i >= valid_cols) p0 = 0.f;
-                        if (c0 + 2 * i + 1 >= valid_cols) p1 = 0.f;
-                    }
-                    ls4[i & 3] += p0 + p1;
-                    const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                    packed[i] = *reinterpret_cast<const uint32_t *>(&h);
-                }
-                tmem_st32(ts + (uint32_t)(c0 >> 1), packed);
-            }
-            tmem_st_wait();
-            l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-            tc_fence_before();
-            mbar_arrive(smem_u32(p_full + grp));
-        }
-        // merge the groups: O = (sum_g 2^(m_g - m) O_g) / (sum_g 2^(m_g - m) l_g); each group stores half the columns
-        const bool final_ok = ok && mbar_wait(smem_u32(o_final), 0u, abort_flag);
-        if (final_ok) {
-            ml_s[(grp * 2 + 0) * 128 + row] = m_used;
-            ml_s[(grp * 2 + 1) * 128 + row] = l_sum;
-        }
-        mbar_arrive(smem_u32(merge_bar));
-        if (final_ok && mbar_wait(smem_u32(merge_bar), 0u, abort_flag)) {
-            tc_fence_after();
-            float fg[2], denom = 0.f;
-            const float m_all = fmaxf(ml_s[row], ml_s[2 * 128 + row]);
-#pragma unroll
-            for (int g = 0; g < 2; ++g) {
-                const bool used = g < nb;             // a group without key blocks never wrote its accumulator
-                fg[g] = used ? fast_exp2(ml_s[(g * 2) * 128 + row] - m_all) : 0.f;
-                denom += used ? fg[g] * ml_s[(g * 2 + 1) * 128 + row] : 0.f;
-            }
-            const float inv = 1.0f / denom;
-            bool good = false;
-            if (row < t.cnt) {
-                const int id = p.sl.ids[t.pos0 + row];
-                good = id >= 0 && (int64_t)id < p.M;
-            }
-#pragma unroll 1
-            for (int c0 = grp * (D / 2); c0 < (grp + 1) * (D / 2); c0 += 32) {
-                float acc[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) acc[i] = 0.f;
-#pragma unroll
-                for (int g = 0; g < 2; ++g) {
-                    if (g < nb) {
-                        uint32_t r[32];
-                        tmem_ld32(lane_base + (uint32_t)(kTmemO + g * D + c0), r);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) acc[i] = fmaf(__uint_as_float(r[i]), fg[g], acc[i]);
-                    }
-                }
-                if (row < t.cnt) {
-                    uint32_t packed[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(good ? acc[2 * i] * inv : 0.f, good ? acc[2 * i + 1] * inv : 0.f);
-                        packed[i] = *reinterpret_cast<const uint32_t *>(&h);
-                    }
-                    uint4 *dst = reinterpret_cast<uint4 *>(p.X + (size_t)(t.pos0 + row) * p.x_stride + c0);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-                }
-            }
-        }
-    } else if (warp == kAtt2MmaWarp) {
-        // ===================== MMA issuer =====================
-        if (lane == 0) {
-            constexpr uint32_t idesc_qk = umma_idesc_bf16(kTcTile, BN);
-            constexpr uint32_t idesc_pv = umma_idesc_bf16_bmn(kTcTile, D);
-            bool ok = mbar_wait(smem_u32(q_full), 0u, abort_flag);
-            fence_proxy_async();
-            tc_fence_after();
-            const uint64_t qdesc0 = umma_desc_sw128(smem_u32(smQ)), kdesc0 = umma_desc_sw128(smem_u32(smKV));
-            const uint64_t vdesc0 = umma_desc_mn_sw128(smem_u32(smKV), kKvChunkBytes);
-            auto ready = [&](uint64_t *bar, uint32_t parity) { return mbar_try_wait(smem_u32(bar), parity, 40u); };
-            int jq = 0, jp = 0;          // next Q K^T / next P V to issue
-            long long t_last = clock64();
-            while (ok && jp < nb) {
-                bool progress = false;
-                // P V of block jp: its probabilities are in tensor memory
-                if (jp < jq && ready(p_full + (jp & 1), (uint32_t)((jp >> 1) & 1))) {
-                    tc_fence_after();
-                    const int s = jp % kS;
-                    const uint32_t o_tmem = tmem_base + (uint32_t)(kTmemO + (jp & 1) * D);
-                    const uint32_t p_tmem = tmem_base + (uint32_t)((jp & 1) * BN);
-                    const uint64_t vd = vdesc0 + (uint64_t)(uint32_t)(s * (kKvBytes >> 4));
-#pragma unroll
-                    for (int kk = 0; kk < BN / 16; ++kk)
-                        umma_bf16_ts(o_tmem, p_tmem + (uint32_t)(kk * 8), vd + (uint64_t)(kk * (2048 >> 4)), idesc_pv,
-                                     (jp >= 2 || kk > 0) ? 1u : 0u);
-                    umma_commit(smem_u32(pv_done + (jp & 1)));
-                    umma_commit(smem_u32(kv_empty + s));
-                    ++jp;
-                    progress = true;
-                }
-                // Q K^T of block jq: its key block has landed, and P V of block jq - 2 (which reads the probabilities that
-                // alias this score buffer) has been issued before it
-                if (jq < nb && jq < jp + 2 && ready(kv_full + jq % kS, (uint32_t)((jq / kS) & 1))) {
-                    tc_fence_after();
-                    const int s = jq % kS;
-                    const uint32_t d_tmem = tmem_base + (uint32_t)((jq & 1) * BN);
-                    const uint64_t kd = kdesc0 + (uint64_t)(uint32_t)(s * (kKvBytes >> 4));
-                    umma_bf16(d_tmem, qdesc0, kd, idesc_qk, 0u);
-#pragma unroll
-                    for (int kk = 1; kk < D / 16; ++kk)
-                        umma_bf16_acc(d_tmem, qdesc0 + (uint64_t)((kk >> 2) * (16384 >> 4) + 2 * (kk & 3)),
-                                      kd + (uint64_t)((kk >> 2) * (kKvChunkBytes >> 4) + 2 * (kk & 3)), idesc_qk);
-                    umma_commit(smem_u32(s_full + (jq & 1)));
-                    ++jq;
-                    progress = true;
-                }
-                if (progress) {
-                    t_last = clock64();
-                } else if (*abort_flag || clock64() - t_last > kWaitCycles) {
-                    *abort_flag = 1u;
-                    ok = false;
-                }
-            }
-            if (ok) umma_commit(smem_u32(o_final));
-        }
-        __syncwarp();
-    } else {
-        // ===================== key/value producer (TMA) =====================
-        if (lane == 0) {
-            for (int j = 0; j < nb; ++j) {
-                const int s = j % kS;
-                if (!mbar_wait(smem_u32(kv_empty + s), (uint32_t)(((j / kS) & 1) ^ 1), abort_flag)) break;
-                mbar_expect_tx(smem_u32(kv_full + s), (uint32_t)kKvBytes);
-                tma_load_3d(smem_u32(smKV + s * kKvBytes), &tmapS, smem_u32(kv_full + s), 0, j * BN, t.slot);
-                tma_load_3d(smem_u32(smKV + s * kKvBytes + kKvChunkBytes), &tmapS, smem_u32(kv_full + s), 64, j * BN, t.slot);
-            }
-        }
-        __syncwarp();
-    }
-
-    if (*abort_flag) {
-        if (tid == 0) atomicOr(p.sl.status, AIF_STATUS_TIMEOUT);
-        const long long t0 = clock64();
-        while (clock64() - t0 < 2000000ll) __nanosleep(1000);
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == kAtt2MmaWarp) tmem_dealloc(tmem_base, 512);
-}
-
 struct AttPlan {
     CUtensorMap tmap;
     int bn = 0;
@@ -901,8 +610,6 @@ cudaError_t tc_att_prepare(aif_ctx *ctx)
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
-    if (c.d == 128 && (e = cudaFuncSetAttribute(k_att_tc_long, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtt2Smem)) != cudaSuccess)
-        return e;
     if (c.d == 128)
         e = cudaFuncSetAttribute(k_att_tc<128, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttCfg<128, 128>::kSmem);
     else
@@ -950,14 +657,10 @@ cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.d);
     // One CTA per SM walking over its tiles hides a tile's query gather and output behind its neighbours' key blocks:
     // 22 k against 31 k cycles per 8-block tile, which outweighs the static assignment's rounding (8.5 tiles per SM cost
-    // 9 tile times) as soon as some SM has two tiles.  Tiles of many key blocks have little to hide and lose only the
-    // rounding: up to 16 tiles per SM they get a CTA each, in the two-group kernel.
-    const bool long_tiles = c.d == 128 && sl.max_L >= 16 * 128 && sl.n_tiles < 148 * 16;
-    const int grid = sl.n_tiles > 148 && !long_tiles ? 148 : sl.n_tiles;
+    // 9 tile times) as soon as some SM has two tiles.
+    const int grid = sl.n_tiles > 148 ? 148 : sl.n_tiles;
     cudaError_t e;
-    if (long_tiles)
-        e = launch_pdl(k_att_tc_long, dim3(grid), dim3(kAtt2Threads), kAtt2Smem, st, pl->tmap, p);
-    else if (c.d == 128)
+    if (c.d == 128)
         e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(AttCfg<128, 128>::kThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, tmap_x, p);
     else
         e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(AttCfg<256, 64>::kThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, tmap_x, p);
@@ -981,12 +684,9 @@ cudaError_t launch_self_att_tc(const aif_ctx *ctx, int slot_index, int L, cudaSt
     CUtensorMap tmap_x;
     cudaError_t ex = encode_x_map(&tmap_x, pl->self_rows, c.d, (size_t)c.L_max + kTcTile);
     if (ex != cudaSuccess) return ex;
-    const bool long_tiles = c.d == 128 && sl.max_L >= 16 * 128 && sl.n_tiles < 148 * 16;   // as in launch_att_tc
-    const int grid = sl.n_tiles > 148 && !long_tiles ? 148 : sl.n_tiles;
+    const int grid = sl.n_tiles > 148 ? 148 : sl.n_tiles;
     cudaError_t e;
-    if (long_tiles)
-        e = launch_pdl(k_att_tc_long, dim3(grid), dim3(kAtt2Threads), kAtt2Smem, st, pl->tmap, p);
-    else if (c.d == 128)
+    if (c.d == 128)
         e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(AttCfg<128, 128>::kThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, tmap_x, p);
     else
         e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(AttCfg<256, 64>::kThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, tmap_x, p);
