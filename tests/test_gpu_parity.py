@@ -228,8 +228,8 @@ def test_full_size_c1_and_sampled_c2():
 def test_sharp_softmax_exercises_the_running_max_rescaling(base, L, s_scale):
     """Item vectors x32 and sequence rows x64 (exact in bf16) give scores with a standard deviation of about 5: the
     softmax is close to one-hot and the running maximum of the streaming kernels jumps by more than their rescaling
-    threshold between key blocks; x1024 gives scores of several hundred (L = 700 and, at d = 256, L = 300: the persistent
-    kernel; L = 2500: the two-group kernel for long sequences).  With L = 200 the single-launch kernel runs: its first
+    threshold between key blocks; x1024 gives scores of several hundred (L = 700 and 2500 at d = 128: two softmax warps per
+    row, which must agree on every raise; L = 300 at d = 256: one).  With L = 200 the single-launch kernel runs: its first
     softmax attempt subtracts no maximum, which holds at x64 and overflows at x1024, where the kernel must fall back to
     exact row maxima.  Activations are O(1) or more here instead of O(0.05), so the bf16 budget is scaled: bf16
     intermediates of magnitude A carry about 2^-9 A of rounding error."""
