@@ -279,6 +279,30 @@ def test_single_launch_scoring_at_the_sequence_lengths_around_its_key_blocks(L):
     srv.close()
 
 
+@pytest.mark.parametrize("L", [1, 40, 64, 65, 128, 129, 192, 193, 320, 321])
+def test_attention_kernel_at_the_sequence_lengths_around_its_half_blocks(L):
+    """d = 128 on the kernel-per-layer path at every length class (a first layer of 256 units is not a shape of the
+    single-launch kernel, so short sequences reach the attention kernel too).  Two softmax warps share each candidate row,
+    each with 64 of a block's 128 keys: the last block leaves the second warp no key at all (L mod 128 in 1..64), a single
+    key (65) or all of them (0), and both must still agree on the block maximum and the row sum.  Two requests in one
+    launch, ragged last tiles."""
+    wl = helpers.MINI["c2"].with_(name=f"att_L{L}", R=2, N=333, L=L, mini_batch=0, hidden=(256, 256))
+    weights, table, srv, oracle = _setup(wl, zero_bias=False)
+    sampler = synth.IdSampler(wl)
+    states, id_lists, wants = [], [], []
+    for r in range(wl.R):
+        rq = synth.make_request(wl, r)
+        ids = sampler.request_ids(r)
+        states.append(srv.precompute(3 + r, srv.upload_request(rq, B.USER_PROJECTED)))
+        id_lists.append(ids), wants.append(oracle.score(table, helpers.projected_request(wl, rq), ids))
+    _check_logits(srv.score_ids(states[0], id_lists[0]), wants[0], TOL["bf16"])
+    for o, w in zip(srv.score_many(states, id_lists), wants):
+        _check_logits(o, w, TOL["bf16"])
+    assert srv.ctx.get_stats().tensor_path == 1
+    assert srv.ctx.poll_status() == 0
+    srv.close()
+
+
 @pytest.mark.parametrize("L", [200, 300])
 def test_several_requests_with_mini_batches_in_one_launch(L):
     """Requests of different sizes, each cut into mini-batches of 500 (tiles never straddle a mini-batch), scored in one
