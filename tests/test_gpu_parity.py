@@ -303,6 +303,32 @@ def test_attention_kernel_at_the_sequence_lengths_around_its_half_blocks(L):
     srv.close()
 
 
+def test_one_launch_over_requests_of_different_sequence_lengths():
+    """More tiles than SMs on the kernel-per-layer path: every CTA of the attention kernel walks over several tiles, and
+    the sequences differ in length from request to request (1 to 321 keys: one to three key blocks, the last one with
+    its second half empty, partly filled or full), so consecutive tiles of a CTA have different block counts.  The oracle
+    checks a seeded sample of every request, first and last candidate included."""
+    Ls = [321, 1, 129, 64, 200, 257]
+    wl = helpers.MINI["c2"].with_(name="mixed_L", R=len(Ls), N=3400, L=max(Ls), mini_batch=0, hidden=(256, 256))
+    weights, table, srv, oracle = _setup(wl, zero_bias=False, max_batch_candidates=wl.R * wl.N)
+    sampler = synth.IdSampler(wl)
+    states, id_lists, reqs = [], [], []
+    for r, L in enumerate(Ls):
+        rq = synth.make_request(wl, r, L=L)
+        states.append(srv.precompute(r, srv.upload_request(rq, B.USER_PROJECTED)))
+        id_lists.append(sampler.request_ids(r)), reqs.append(helpers.projected_request(wl, rq))
+    outs = srv.score_many(states, id_lists)
+    assert srv.ctx.get_stats().tensor_path == 1
+    g = np.random.default_rng(23)
+    for r in range(wl.R):
+        ids = id_lists[r]
+        pick = np.unique(np.concatenate([[0, len(ids) - 1], g.choice(len(ids), 38, replace=False)]))
+        _check_logits(outs[r][pick], oracle.score(table, reqs[r], ids[pick]), TOL["bf16"])
+        assert np.isfinite(outs[r]).all()
+    assert srv.ctx.poll_status() == 0
+    srv.close()
+
+
 @pytest.mark.parametrize("L", [200, 300])
 def test_several_requests_with_mini_batches_in_one_launch(L):
     """Requests of different sizes, each cut into mini-batches of 500 (tiles never straddle a mini-batch), scored in one
