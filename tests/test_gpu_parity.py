@@ -303,13 +303,16 @@ def test_attention_kernel_at_the_sequence_lengths_around_its_half_blocks(L):
     srv.close()
 
 
-def test_one_launch_over_requests_of_different_sequence_lengths():
-    """More tiles than SMs on the kernel-per-layer path: every CTA of the attention kernel walks over several tiles, and
+@pytest.mark.parametrize("base", ["c2", "c5"])
+def test_one_launch_over_requests_of_different_sequence_lengths(base):
+    """d = 128 and d = 256.  More tiles than SMs on the kernel-per-layer path: every CTA of the attention kernel walks over several tiles, and
     the sequences differ in length from request to request (1 to 321 keys: one to three key blocks, the last one with
     its second half empty, partly filled or full), so consecutive tiles of a CTA have different block counts.  The oracle
     checks a seeded sample of every request, first and last candidate included."""
     Ls = [321, 1, 129, 64, 200, 257]
-    wl = helpers.MINI["c2"].with_(name="mixed_L", R=len(Ls), N=3400, L=max(Ls), mini_batch=0, hidden=(256, 256))
+    wl = helpers.MINI[base].with_(name=f"mixed_L_{base}", R=len(Ls), N=3400, L=max(Ls), mini_batch=0)
+    if base == "c2":
+        wl = wl.with_(hidden=(256, 256))   # not a shape of the single-launch kernel
     weights, table, srv, oracle = _setup(wl, zero_bias=False, max_batch_candidates=wl.R * wl.N)
     sampler = synth.IdSampler(wl)
     states, id_lists, reqs = [], [], []
