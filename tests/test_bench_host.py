@@ -24,7 +24,8 @@ plan = bench.replica_plan(world, rank)
 elapsed = 10.0 + 5.0 * rank                    # rank 1 is the slow one
 total = bench.reduce_max(elapsed, dist)
 dist.barrier()
-print(json.dumps({"rank": rank, "total": total, "plan": plan}))
+with open(os.path.join(os.environ["AIF_OUT"], f"rank{rank}.json"), "w") as fh:   # one file per rank: stdout of two ranks can interleave
+    json.dump({"rank": rank, "total": total, "plan": plan}, fh)
 dist.destroy_process_group()
 """
 
@@ -43,12 +44,12 @@ def test_flop_model_matches_the_scope_table():
 def test_replica_plan_and_max_over_ranks_with_two_gloo_ranks(tmp_path):
     script = tmp_path / "worker.py"
     script.write_text(WORKER)
-    env = dict(os.environ, AIF_ROOT=ROOT)
+    env = dict(os.environ, AIF_ROOT=ROOT, AIF_OUT=str(tmp_path))
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2", "--master-addr", "127.0.0.1",
            "--master-port", "29617", str(script)]
     r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=240)
     assert r.returncode == 0, r.stderr[-2000:]
-    lines = [json.loads(ln) for ln in r.stdout.splitlines() if ln.startswith("{")]
+    lines = [json.loads((tmp_path / f"rank{k}.json").read_text()) for k in range(2)]
     assert sorted(x["rank"] for x in lines) == [0, 1]
     for x in lines:
         assert x["total"] == 15.0                     # max over ranks, seen by every rank
