@@ -203,8 +203,8 @@ typedef struct {
  * Errors: AIF_ERR_ARG (NULL, struct_size), AIF_ERR_SHAPE (widths < 1, not multiples of 4), AIF_ERR_OOM. */
 int aif_load_item_weights(aif_ctx *ctx, const aif_item_weights *w, aif_stream stream);
 
-/* Item side, nearline, as a compute call (Section 3.2: "generating vectors for the full candidate set stored in an
- * indexing table", triggered by model or feature updates; Section 3.4: full and incremental updates): from raw item
+/* Item side, nearline, as a compute call (Section 3.2: the nearline job that fills the item table for every candidate,
+ * run again whenever the model or the features change; Section 3.4: full and incremental updates): from raw item
  * features to the table rows that aif_item_nearline_refresh would have been handed.
  *   I_raw  device [n x dI] storage type: concatenated item embeddings; gives the item vectors I^ (eq. 4)
  *   I_id   device [n x d] storage type or NULL: item id embeddings for the BEA weights (Algorithm 1 step 3); NULL: the

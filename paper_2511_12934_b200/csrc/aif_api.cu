@@ -559,6 +559,11 @@ int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *st
         tiles += tiles_for(ctx, n);
         AIF_CUDA(wait_user_ready(ctx->slots[(size_t)states[r]->index], st));
     }
+    if (ctx->tensor_path && (size_t)tiles > tc_tile_capacity(ctx)) {
+        snprintf(g_last_error, sizeof(g_last_error), "aif_score_batch: %d tiles exceed the tile table's %zu entries", tiles,
+                 tc_tile_capacity(ctx));
+        return AIF_ERR_SHAPE;
+    }
     AIF_CUDA(cudaMemcpyAsync(ring.dev[slot], ring.host[slot], sizeof(ReqDev) * (size_t)n_req, cudaMemcpyHostToDevice, st));
     ScoreLaunch sl{};
     sl.slots = ctx->slots_dev, sl.reqs = ring.dev[slot], sl.n_req = n_req, sl.n_tiles = tiles, sl.total = total, sl.max_L = max_L;

@@ -252,6 +252,7 @@ void nearline_destroy(aif_ctx *ctx);
 int check_user_state(aif_ctx *ctx, const aif_user_state *st);
 void set_last_error(const char *text);
 int tc_tiles_for(const aif_ctx *ctx, int n);
+size_t tc_tile_capacity(const aif_ctx *ctx);   // entries of the context's tile table (launches over several requests)
 cudaError_t launch_wait_selftest(const aif_ctx *ctx, long long limit_cycles, cudaStream_t st);
 
 }  // namespace aif

@@ -696,6 +696,11 @@ cudaError_t launch_user_network(const aif_ctx *ctx, HostSlot &hs, int slot_index
         if (e != cudaSuccess) return e;
     } else if (c.blocks & AIF_BLK_BEA) {
         const size_t smem = (size_t)(c.n_bridge * in->bea_m + c.n_bridge * c.d) * 4;
+        if (smem > 48 * 1024) {   // up to 80 KB at n_bridge = 16, bea_m = 1024, d = 256: beyond the default limit of a launch
+            e = c.dtype == AIF_F32 ? cudaFuncSetAttribute(k_bea_user<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                                   : cudaFuncSetAttribute(k_bea_user<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
         if (c.dtype == AIF_F32)
             k_bea_user<float><<<1, 256, smem, st>>>((const float *)ctx->bridges, (const float *)in->bea_U, (const float *)ctx->W_f, c.n_bridge,
                                                     in->bea_m, c.d, (float *)hs.dev.V);

@@ -679,6 +679,7 @@ struct TcPlan {
     __nv_bfloat16 *X = nullptr;
     uint16_t *xb = nullptr;              // cross-feature buckets [positions x F]
     TileDev *tiles = nullptr;            // tile table of a launch over several requests
+    size_t tiles_cap = 0;                // its entries
     bool maps_ready = false;
 };
 
@@ -716,6 +717,8 @@ bool tc_supported(const aif_config &c)
 }
 
 int tc_tiles_for(const aif_ctx *ctx, int n) { return tiles_of(n, kTcTile, ctx->cfg.mini_batch); }
+
+size_t tc_tile_capacity(const aif_ctx *ctx) { return reinterpret_cast<const TcPlan *>(ctx->tc_plan)->tiles_cap; }
 
 static TcPlan *plan_of(const aif_ctx *ctx) { return reinterpret_cast<TcPlan *>(ctx->tc_plan); }
 
@@ -771,7 +774,15 @@ cudaError_t tc_prepare_context(aif_ctx *ctx)
     }
     if (pl->x_cols && (e = alloc((void **)&pl->X, cap * pl->x_cols * 2)) != cudaSuccess) return e;
     if ((c.blocks & AIF_BLK_CROSS) && (e = alloc((void **)&pl->xb, cap * c.F * 2)) != cudaSuccess) return e;
-    if ((e = alloc((void **)&pl->tiles, (cap / kTcTile + (size_t)c.max_user_states * 8 + 64) * sizeof(TileDev))) != cudaSuccess) return e;
+    {
+        // Tiles never straddle a mini-batch, so every mini-batch rounds up by itself: a mini-batch of mb candidates is
+        // ceil(mb / 128) tiles, and the tail of every request adds at most as many again.
+        const size_t mb = (size_t)c.mini_batch;
+        const size_t tpm = mb ? (mb + kTcTile - 1) / kTcTile : 0;
+        const size_t body = mb ? ((size_t)c.max_batch_candidates / mb + 1) * tpm : (size_t)c.max_batch_candidates / kTcTile + 1;
+        pl->tiles_cap = body + (size_t)c.max_user_states * (mb ? tpm : 1) + 64;
+        if ((e = alloc((void **)&pl->tiles, pl->tiles_cap * sizeof(TileDev))) != cudaSuccess) return e;
+    }
     e = cudaFuncSetAttribute(k_layer_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LayerCfg<0>::kSmem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_layer_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LayerCfg<1>::kSmem);

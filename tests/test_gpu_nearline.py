@@ -158,11 +158,12 @@ def test_nearline_call_errors():
     srv.close()
 
 
-@pytest.mark.parametrize("name,m", [("c1", 5), ("c2", 37)])
-def test_user_side_of_algorithm_1_is_computed_when_only_U_is_given(name, m):
+@pytest.mark.parametrize("name,m,nb", [("c1", 5, 8), ("c2", 37, 8), ("c2", 1024, 16), ("c5", 1024, 16)])
+def test_user_side_of_algorithm_1_is_computed_when_only_U_is_given(name, m, nb):
     """aif_user_precompute with bea_U instead of bea_V: W = Softmax(B U^T / sqrt(d)), V_k = W_f (sum_j W_kj U_j) on the GPU,
-    against the oracle; then scoring with the BEA block on, where the item-side weights meet these vectors (step 4)."""
-    wl = helpers.MINI[name].with_(name=f"bea_user_{name}", blocks=helpers.ALL_BLOCKS, N=200, L=40,
+    against the oracle; then scoring with the BEA block on, where the item-side weights meet these vectors (step 4).
+    The largest sizes the header allows (1024 features, 16 bridges, d up to 256) are included."""
+    wl = helpers.MINI[name].with_(name=f"bea_user_{name}", blocks=helpers.ALL_BLOCKS, N=200, L=40, n_bridge=nb, R=1,
                                   lsh_din_norm=synth.NORM_MEAN, simtier_norm=synth.NORM_MEAN, emit_sigmoid=0)
     weights = synth.make_weights(wl)
     table = synth.make_item_table(wl)
