@@ -60,6 +60,8 @@ def kernel_flops(name: str, wl: synth.Workload, n: int) -> float:
         return f["total"] * n
     if name == "interact":
         return (f["attention"] + f["lsh_din"] + f["bea"]) * n
+    if name == "lsh":          # eq. 8's contraction; the match counts of eqs. 6-7 ride in the same kernel (see lsh_note)
+        return f["lsh_din"] * n
     if name == "buckets":
         return 0.0
     return f.get(name, 0.0) * n
@@ -402,6 +404,10 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
         roof = {"bound": "alu", "kernel": top, "achieved": kf / (kavg[top] * 1e-3) / 1e12, "peak": FP32_FMA_PEAK_TFLOPS,
                 "unit": "TFLOP/s", "peak_kind": "fp32 FMA: 148 SMs x 128 lanes x 2 x 1.965 GHz"}
     roof["frac"] = roof["achieved"] / roof["peak"]
+    if top == "lsh":
+        roof["lsh_note"] = (f"eqs. 6-7 need {wl.lsh_bits // 32} xor + popc on 32-bit words per (candidate, key) pair by the definition; "
+                            f"the kernel gets the counts from a +-1 fp8 product ({2 * wl.lsh_bits} tensor flop per pair, not counted "
+                            "in `achieved`) and spends about ten integer / fp32 instructions per pair on conversion and tiers")
     roof["traffic"] = NCU_TRAFFIC_BYTES.get((wl.name, top))
     roof["kernel_ms"] = kavg
 
@@ -445,7 +451,7 @@ def main():
     ap.add_argument("--workload", default="c2", choices=sorted(synth.SHORT))
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--also", default="c3,c4,c5", help="other workloads measured briefly after the main one ('' = none)")
+    ap.add_argument("--also", default="c3,c4,c4_lsh,c4_both,c5", help="other workloads measured briefly after the main one ('' = none)")
     # scaled copies of a workload, for profiler captures that must stay small (the defaults are the full sizes)
     ap.add_argument("--requests", type=int, default=0, help="override the number of requests per step")
     ap.add_argument("--rows", type=int, default=0, help="override the rows of the item table")

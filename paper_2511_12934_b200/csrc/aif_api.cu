@@ -224,7 +224,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     TRY(dev_alloc(ctx, (void **)&ctx->b_b, (size_t)c.d * 4, true));
 
     // user-state arena: fixed-size slots in one allocation
-    struct Off { size_t u, u32, S, T, V, sig, pu, pu_hl, prof, partial, ppart, end; } o{};
+    struct Off { size_t u, u32, S, T, V, sig, sigE, pu, pu_hl, prof, partial, ppart, end; } o{};
     size_t p = 0;
     auto take = [&](size_t bytes) { size_t at = p; p += align_up(bytes ? bytes : 16, 256); return at; };
     o.u = take((size_t)c.d * el);
@@ -233,6 +233,8 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     o.T = take((c.blocks & AIF_BLK_CROSS) ? (size_t)c.F * c.B * c.dc * el : 0);
     o.V = take((c.blocks & AIF_BLK_BEA) ? (size_t)c.n_bridge * c.d * el : 0);
     o.sig = take((c.blocks & (AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER)) ? (size_t)c.L_max * c.lsh_bits / 8 : 0);
+    const bool lsh_tc = ctx->tensor_path && tc_lsh_supported(c);
+    o.sigE = take(lsh_tc ? (size_t)c.L_max * c.lsh_bits : 0);
     o.pu = take((size_t)c.hidden[0] * 4);
     o.pu_hl = take((size_t)c.hidden[0] * 2 * 2);
     o.prof = take((size_t)c.d * 4);
@@ -250,6 +252,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
         HostSlot &hs = ctx->slots[(size_t)i];
         hs.dev.u = base + o.u, hs.dev.u32 = (const float *)(base + o.u32), hs.dev.S = base + o.S;
         hs.dev.T = base + o.T, hs.dev.V = base + o.V, hs.dev.sigS = (const uint8_t *)(base + o.sig);
+        hs.dev.sigE = lsh_tc ? (const uint8_t *)(base + o.sigE) : nullptr;
         hs.dev.p_u = (const float *)(base + o.pu), hs.dev.pu_hl = base + o.pu_hl, hs.dev.L = 0;
         hs.prof_hat = (float *)(base + o.prof), hs.partial = (float *)(base + o.partial), hs.ppart = (float *)(base + o.ppart);
         cudaError_t e = cudaEventCreateWithFlags(&hs.ev, cudaEventDisableTiming);

@@ -25,6 +25,7 @@ struct SlotDev {
     const void *T;          // [F x B x dc] storage type: cross pre-cache
     const void *V;          // [n_bridge x d] storage type
     const uint8_t *sigS;    // [L x lsh_bits/8]
+    const uint8_t *sigE;    // [L x lsh_bits] the same signatures with one E4M3 byte per bit, +1.0 / -1.0 (tensor-core LSH), or nullptr
     const float *p_u;       // [H1] fp32: W1[:, user columns] u + b1
     const void *pu_hl;      // [2][H1] bf16: p_u split into high parts and remainders (bias operand of the tensor cores)
     int32_t L;
@@ -163,6 +164,7 @@ struct aif_ctx {
     void *tc_att_plan = nullptr;      // tensor-core attention: tensor map over the arena's S regions
     void *nearline_plan = nullptr;    // item-side weights and scratch of aif_item_nearline_compute
     void *tc_fused_plan = nullptr;    // single-launch scoring: the second layer's bias split into two bf16 rows
+    void *tc_lsh_plan = nullptr;      // tensor-core LSH blocks: tensor maps over the arena's S and +-1 signature regions
     aif::PinnedRing ring;
 
     aif_stats stats{};
@@ -205,6 +207,13 @@ void tc_att_destroy(aif_ctx *ctx);
 // *rows_out: [L x d] bf16 in scratch of the attention plan, valid until the next call
 cudaError_t launch_self_att_tc(const aif_ctx *ctx, int slot_index, int L, cudaStream_t st, const void **rows_out);
 cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, void *X, int x_stride, size_t x_rows);
+// LSH similarity, LSH-DIN and SimTier on the tensor cores (aif_tc_lsh.cu)
+bool tc_lsh_supported(const aif_config &cfg);
+cudaError_t tc_lsh_prepare(aif_ctx *ctx);
+void tc_lsh_destroy(aif_ctx *ctx);
+cudaError_t launch_expand_signatures(const aif_ctx *ctx, const uint8_t *sig, int L, uint8_t *out, cudaStream_t st);
+cudaError_t launch_lsh_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, void *X, int x_stride, size_t x_rows, int x_din,
+                          int x_tier);
 // whole scoring pass of a tile in one CTA (aif_tc_fused.cu); the tensor maps it shares with the other kernels
 bool tc_fused_supported(const aif_config &cfg);
 cudaError_t tc_fused_prepare(aif_ctx *ctx);

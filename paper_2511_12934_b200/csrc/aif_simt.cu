@@ -714,6 +714,8 @@ cudaError_t launch_user_network(const aif_ctx *ctx, HostSlot &hs, int slot_index
     if (c.blocks & (AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER)) {
         e = cudaMemcpyAsync((void *)hs.dev.sigS, in->seq_sig, (size_t)L * (c.lsh_bits / 8), cudaMemcpyDeviceToDevice, st);
         if (e != cudaSuccess) return e;
+        // the form the tensor-core LSH kernel multiplies: one +-1 byte per signature bit
+        if (ctx->tc_lsh_plan && (e = launch_expand_signatures(ctx, in->seq_sig, L, const_cast<uint8_t *>(hs.dev.sigE), st)) != cudaSuccess) return e;
     }
     if (c.dtype == AIF_F32) return user_network_typed<float>(ctx, hs, slot_index, in, L, st);
     return user_network_typed<__nv_bfloat16>(ctx, hs, slot_index, in, L, st);

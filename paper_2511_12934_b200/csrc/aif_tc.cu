@@ -571,7 +571,7 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
 // ---- interaction blocks that feed dense columns (CUDA cores; one warp per candidate) ---------------------------
 // Writes, per candidate position, a bf16 row [ att (d) | v_bea (d) | lsh_din (d) | simtier (64, first n_tiers used) ]
 // holding only the enabled blocks.
-__global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl, __nv_bfloat16 *X, int x_stride, int att_done)
+__global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl, __nv_bfloat16 *X, int x_stride, int att_done, int lsh_done)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *qv = reinterpret_cast<float *>(smem_raw);                         // [8][d]
@@ -584,16 +584,26 @@ __global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl,
     int start, cnt;
     tile_range(blockIdx.x - rq.tile_begin, rq.n, kTcTile, md.mini_batch, start, cnt);
     const SlotDev slot = sl.slots[rq.slot];
-    // att_done: the attention columns were already written by the tensor-core attention kernel
-    const bool has_att = md.blocks & AIF_BLK_ATT, do_att = has_att && !att_done, do_bea = md.blocks & AIF_BLK_BEA, do_din = md.blocks & AIF_BLK_LSH_DIN,
-               do_tier = md.blocks & AIF_BLK_SIMTIER, do_lsh = do_din || do_tier;
+    // att_done / lsh_done: those columns were already written by the tensor-core attention / LSH kernels
+    const bool has_att = md.blocks & AIF_BLK_ATT, do_att = has_att && !att_done, do_bea = md.blocks & AIF_BLK_BEA;
+    const bool has_din = md.blocks & AIF_BLK_LSH_DIN, has_tier = md.blocks & AIF_BLK_SIMTIER;
+    const bool do_din = has_din && !lsh_done, do_tier = has_tier && !lsh_done, do_lsh = do_din || do_tier;
+    const int col_bea = has_att ? d : 0, col_din = col_bea + (do_bea ? d : 0), col_tier = col_din + (has_din ? d : 0);
     using T = __nv_bfloat16;
     for (int c = warp; c < cnt; c += 8) {
         const int64_t pos = rq.off + start + c;
         const int id = sl.ids[pos];
         T *xrow = X + (size_t)pos * x_stride;
         if (id < 0 || (int64_t)id >= md.M) {
-            for (int k = lane; k < x_stride; k += 32) xrow[k] = __float2bfloat16_rn(0.f);
+            // zero the columns this kernel owns; the tensor-core kernels zero theirs
+            const __nv_bfloat16 z = __float2bfloat16_rn(0.f);
+            for (int k = lane; k < d; k += 32) {
+                if (do_att) xrow[k] = z;
+                if (do_bea) xrow[col_bea + k] = z;
+                if (do_din) xrow[col_din + k] = z;
+            }
+            if (do_tier)
+                for (int k = lane; k < 64; k += 32) xrow[col_tier + k] = z;
             continue;
         }
         const T *e = reinterpret_cast<const T *>(md.E) + (size_t)id * d;
@@ -606,13 +616,13 @@ __global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl,
         if (do_att || do_lsh)
             warp_interact<T>(qv + warp * d, reinterpret_cast<const T *>(slot.S), slot.L, d, rsqrtf((float)d), do_att, do_lsh,
                              do_tier, sigq + warp * 8, slot.sigS, md.lsh_bits, md.n_tiers, tiers + warp * 16, att, din);
-        int col = (has_att && att_done) ? d : 0;
+        int col = 0;
         if (do_att) {
 #pragma unroll
             for (int q = 0; q < 8; ++q)
                 if (q < dq) xrow[col + lane + 32 * q] = __float2bfloat16_rn(att[q]);
-            col += d;
         }
+        if (has_att) col += d;
         if (do_bea) {
             const T *wh = reinterpret_cast<const T *>(md.bea_w) + (size_t)id * md.n_bridge;
             const T *V = reinterpret_cast<const T *>(slot.V);
@@ -628,8 +638,8 @@ __global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl,
 #pragma unroll
             for (int q = 0; q < 8; ++q)
                 if (q < dq) xrow[col + lane + 32 * q] = __float2bfloat16_rn(din[q] * nrm);
-            col += d;
         }
+        if (has_din) col += d;
         if (do_tier) {
             __syncwarp();
             const float nrm = md.simtier_norm == AIF_NORM_MEAN ? 1.0f / (float)slot.L : 1.0f;
@@ -809,6 +819,7 @@ cudaError_t tc_prepare_context(aif_ctx *ctx)
     pl->maps_ready = true;
     if (tc_att_supported(c) && (e = tc_att_prepare(ctx)) != cudaSuccess) return e;
     if (tc_fused_supported(c) && (e = tc_fused_prepare(ctx)) != cudaSuccess) return e;
+    if (tc_lsh_supported(c) && (e = tc_lsh_prepare(ctx)) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
@@ -817,6 +828,7 @@ const void *tc_weight_tmap(const aif_ctx *ctx, int k) { return &plan_of(ctx)->tm
 void tc_destroy_context(aif_ctx *ctx)
 {
     if (ctx->tc_att_plan) tc_att_destroy(ctx);
+    if (ctx->tc_lsh_plan) tc_lsh_destroy(ctx);
     delete plan_of(ctx);
     ctx->tc_plan = nullptr;
 }
@@ -980,11 +992,25 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl_in
         timing_mark(ctx, "attention", st);
         if (e != cudaSuccess) return e;
     }
-    const int other_dense = c.blocks & (AIF_BLK_BEA | AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER);
-    if (pl->x_cols && (!att_tc || other_dense)) {
+    const int lsh_blocks = c.blocks & (AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER);
+    const bool lsh_tc = lsh_blocks && ctx->tc_lsh_plan != nullptr;
+    if (lsh_tc) {
+        // columns of X: [ att | v_bea | lsh_din | simtier (64) ], enabled blocks only
+        int col = 0;
+        if (c.blocks & AIF_BLK_ATT) col += c.d;
+        if (c.blocks & AIF_BLK_BEA) col += c.d;
+        const int x_din = (c.blocks & AIF_BLK_LSH_DIN) ? col : -1;
+        if (c.blocks & AIF_BLK_LSH_DIN) col += c.d;
+        const int x_tier = (c.blocks & AIF_BLK_SIMTIER) ? col : -1;
+        cudaError_t e = launch_lsh_tc(ctx, sl, st, sc.X, pl->x_cols, sc.rows, x_din, x_tier);
+        timing_mark(ctx, "lsh", st);
+        if (e != cudaSuccess) return e;
+    }
+    const bool need_att = (c.blocks & AIF_BLK_ATT) && !att_tc, need_lsh = lsh_blocks && !lsh_tc;
+    if (pl->x_cols && (need_att || need_lsh || (c.blocks & AIF_BLK_BEA))) {
         const size_t smem = (size_t)8 * c.d * 4 + 64 * 4 + 128 * 4;
         cudaError_t e = launch_pdl(k_interact_x, dim3(sl.n_tiles), dim3(256), smem, st, md, sl, (__nv_bfloat16 *)sc.X, pl->x_cols,
-                                   att_tc ? 1 : 0);
+                                   att_tc ? 1 : 0, lsh_tc ? 1 : 0);
         count_launch();
         timing_mark(ctx, "interact", st);
         if (e != cudaSuccess) return e;

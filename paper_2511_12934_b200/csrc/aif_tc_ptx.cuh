@@ -163,6 +163,25 @@ __device__ __forceinline__ void umma_bf16_acc(uint32_t d_tmem, uint64_t adesc, u
         : "memory");
 }
 
+// Instruction descriptor of tcgen05.mma.kind::f8f6f4 with both operands E4M3 (format code 0 in [7,10) and [10,13)), K-major,
+// D fp32: one instruction covers K = 32 elements (32 bytes of a 128-byte swizzled row).
+__host__ __device__ constexpr uint32_t umma_idesc_e4m3(int m, int n)
+{
+    return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_e4m3(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // D (+)= A B with the A operand read from tensor memory (M lanes x K/2 columns, two bf16 per 32-bit column along K).
 __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
 {

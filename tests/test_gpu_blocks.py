@@ -166,3 +166,56 @@ def test_raw_user_precompute_at_long_sequences(base, L):
     _check(srv.score_ids(st, ids)[pick], want)
     assert srv.ctx.poll_status() == 0
     srv.close()
+
+
+@pytest.mark.parametrize("base,n_tiers,din_norm,tier_norm,blocks", [
+    ("c2", 8, synth.NORM_MEAN, synth.NORM_MEAN, helpers.ALL_BLOCKS),
+    ("c2", 16, synth.NORM_MEAN, synth.NORM_MEAN, synth.BLK_CROSS | LSH),
+    ("c2", 5, synth.NORM_NONE, synth.NORM_NONE, synth.BLK_ATT | synth.BLK_CROSS | LSH),
+    ("c2", 1, synth.NORM_MEAN, synth.NORM_NONE, synth.BLK_SIMTIER),
+    ("c2", 3, synth.NORM_MEAN, synth.NORM_MEAN, synth.BLK_CROSS | synth.BLK_LSH_DIN),
+    ("c5", 16, synth.NORM_MEAN, synth.NORM_MEAN, synth.BLK_CROSS | LSH),
+    ("c5", 7, synth.NORM_NONE, synth.NORM_MEAN, helpers.ALL_BLOCKS)])
+def test_lsh_blocks_run_on_the_tensor_cores_for_every_tier_count_and_norm(base, n_tiers, din_norm, tier_norm, blocks):
+    """The LSH similarity, LSH-DIN and SimTier kernel (signature products in fp8, counts times S in bf16): tier counts 1 to
+    16 (tier edges that do and do not divide d'), raw and mean-normalised outputs, either block alone, sequence lengths that
+    leave the last key block nearly empty, half full and full, identical signatures (every match count = d', the closed
+    last tier) and complementary ones (0 matches).  The kernel list of the call must name the tensor-core kernel."""
+    exact = din_norm == synth.NORM_MEAN and tier_norm == synth.NORM_MEAN
+    # raw sums and counts (eq. 8 and eq. 9 as printed) grow with the sequence: kept to lengths whose counts bf16 still holds
+    # exactly (<= 256), since the MLP input is stored in bf16
+    Ls = [1, 63, 64, 65, 127, 128, 129, 700 if exact else 256]
+    wl = helpers.MINI[base].with_(name=f"lsh_tc_{base}_{n_tiers}", R=len(Ls), N=300, L=max(Ls), mini_batch=0, blocks=blocks,
+                                  n_tiers=n_tiers, lsh_din_norm=din_norm, simtier_norm=tier_norm)
+    weights = synth.make_weights(wl, zero_bias=False)
+    table = synth.make_item_table(wl)
+    sampler = synth.IdSampler(wl)
+    id_lists = [sampler.request_ids(r) for r in range(wl.R)]
+    rqs = [synth.make_request(wl, r, L=L) for r, L in enumerate(Ls)]
+    # request 3: every sequence item carries the signature of the request's first candidate, request 4 its complement
+    rqs[3]["sig_seq"][:] = table["sig"][id_lists[3][0]]
+    rqs[4]["sig_seq"][:] = ~table["sig"][id_lists[4][0]]
+    srv = serving.Server(wl, weights, table, path=B.PATH_TENSOR)
+    oracle = helpers.make_oracle(wl, weights, M=table["E"].shape[0])
+    states = [srv.precompute(r, srv.upload_request(rq, B.USER_PROJECTED)) for r, rq in enumerate(rqs)]
+    srv.ctx.set_kernel_timing(True)
+    outs = srv.score_many(states, id_lists)
+    assert "lsh" in srv.ctx.get_kernel_timing()
+    srv.ctx.set_kernel_timing(False)
+    # With mean-normalised outputs every MLP input is below 1 and the tolerance is the plain 2e-3.  Raw sums and counts are
+    # inputs of magnitude A >> 1 that the kernel chain stores in bf16 (relative rounding 2^-9), and so are the hidden
+    # activations they produce: the tolerance scales with A.  That only checks the plumbing of the unnormalised option; the
+    # counts and sums themselves are checked by the normalised cases, which differ by one multiplication.
+    def tol_for(x):
+        return TOL * (1.0 if exact else max(1.0, float(np.nanmax(np.abs(x)))))
+
+    for r in range(wl.R):
+        want, x = oracle.score(table, helpers.projected_request(wl, rqs[r]), id_lists[r], return_inputs=True)
+        _check(outs[r], want, tol_for(x))
+    # one request alone, with ids outside the table: NaN logits, status bit, neighbours untouched
+    ids = id_lists[7].copy()
+    ids[3], ids[130] = -1, table["E"].shape[0]
+    want, x = oracle.score(table, helpers.projected_request(wl, rqs[7]), ids, return_inputs=True)
+    _check(srv.score_ids(states[7], ids), want, tol_for(x))
+    assert srv.ctx.poll_status() == B.STATUS_BAD_ID
+    srv.close()
