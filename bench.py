@@ -33,9 +33,24 @@ METRIC = "candidates scored/s (p50 latency per request reported beside it), 1 B2
 UNIT = "candidates/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # CUDA-core kernels: SMs x lanes x 2 x max clock
+NOMINAL_BF16_TFLOPS = 2250.0                               # dense bf16, the data-sheet figure
+NOMINAL_HBM_GBS = 8000.0
 
-# DRAM traffic per launch of the dominant kernel from the committed ncu summary (profiles/), bytes; None = not captured.
-NCU_TRAFFIC_BYTES = {("c2_paper_shaped", "score_fused"): 4867840}      # profiles/scoring_step_c2.md
+
+def ncu_traffic_table():
+    """DRAM read + write bytes of the scoring kernels as ncu counted them: {(workload, kernel): (unit, bytes)} with unit
+    "per_launch" (captured on the benchmark's own workload) or "per_candidate" (captured on a scaled copy of it; the
+    traffic of these kernels grows with the candidates).  The table is a text file kept beside the ncu summaries."""
+    out = {}
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return out
+    with open(path) as fh:
+        for ln in fh:
+            parts = ln.split()
+            if len(parts) == 4 and not ln.startswith("#"):
+                out[(parts[0], parts[1])] = (parts[2], float(parts[3]))
+    return out
 
 
 # ----------------------------------------------------------------------------------------------------------------
@@ -224,7 +239,8 @@ def run_ours(args, wl):
         for name in args.also.split(","):
             o = measure(args, synth.SHORT[name], 20, 3, None, 1, 0, full=False)
             others[name] = {k: o[k] for k in ("value", "unit", "ms_per_step", "p50_ms_per_request", "p99_ms_per_request",
-                                              "flops_per_candidate", "config", "roofline", "step_tflops")}
+                                              "latency_samples", "flops_per_candidate", "config", "roofline", "step_tflops",
+                                              "step_frac", "e2e")}
         line["other_workloads"] = others
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl)
@@ -301,13 +317,16 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
     total_ms = reduce_max(sum(times), dist)
 
     # end to end: host ids in, host logits out, through aif_score_host (one call per request)
-    host_ids = [torch.from_numpy(x).pin_memory() for x in id_lists]
-    host_out = [torch.empty(len(x), dtype=torch.float32).pin_memory() for x in id_lists]
+    if batch:
+        host_ids = [torch.from_numpy(np.concatenate(id_lists)).pin_memory()]
+        host_out = [torch.empty(cands, dtype=torch.float32).pin_memory()]
+    else:
+        host_ids = [torch.from_numpy(x).pin_memory() for x in id_lists]
+        host_out = [torch.empty(len(x), dtype=torch.float32).pin_memory() for x in id_lists]
 
     def step_e2e(i):
         if batch:
-            for r in range(wl.R):
-                srv.ctx.score_host(states[r], host_ids[r], host_out[r])
+            srv.ctx.score_batch_host(states, host_ids[0], offs, host_out[0])
         else:
             srv.ctx.score_host(states[i % pool], host_ids[i % pool], host_out[i % pool])
 
@@ -315,6 +334,13 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
     step_e2e(0)
     e2e_times = timed(e2e_steps, step_e2e)
     e2e_ms = reduce_max(sum(e2e_times), dist)
+
+    # per-request latency percentiles from a pass of their own, whatever --steps says: one sample per scoring call
+    # (a launch over R requests gives its time divided by R), L2 flushed before each
+    lat_calls = (1000 if full else 100) if not batch else max(20, min(1000 if full else 60, int(4000.0 / max(1e-3, float(np.mean(times))))))
+    if args.latency_calls >= 0:
+        lat_calls = max(2, args.latency_calls)
+    lat_times = timed(lat_calls, step)
     clocks = sampler_proc.stop()
 
     # per-kernel durations (events inside the library), for the roofline of the dominant kernel
@@ -341,7 +367,17 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
 
     gather_step(0)
     g_ms = float(np.median(timed(10, gather_step)))
-    del g_out
+    # the same over distinct rows (a seeded permutation of the table, at most 2^22 of them): no row is read twice, so L2
+    # cannot serve repeats and the figure is an HBM figure (the table is larger than L2 for every bf16 workload)
+    gd = int(min(gn, table["E"].shape[0]))
+    d_ids = torch.from_numpy(np.random.default_rng(8).permutation(table["E"].shape[0])[:gd].astype(np.int32)).cuda()
+
+    def gather_distinct(i):
+        srv.ctx.gather_rows(d_ids, g_out[:gd])
+
+    gather_distinct(0)
+    gd_ms = float(np.median(timed(10, gather_distinct)))
+    del g_out, d_ids
 
     # the user-side call (eqs. 1-3 from raw embeddings + pre-cache + p_u) on the side stream: the time a retrieval phase has
     # to cover; one extra arena slot is not available, so a state of the pool is recomputed in place of itself
@@ -389,10 +425,17 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
         del dev_it, saved
 
     peaks, peak_kind = load_peaks()
-    gather = {"rows": gn, "row_bytes": row_bytes, "ms": g_ms, "achieved": gn * (2 * row_bytes + 4) / (g_ms * 1e-3) / 1e9,
+    gather = {"rows": gd, "row_bytes": row_bytes, "ms": gd_ms, "achieved": gd * (2 * row_bytes + 4) / (gd_ms * 1e-3) / 1e9,
               "peak": float(peaks["hbm_gbs"]), "unit": "GB/s", "bound": "hbm", "peak_kind": f"copy bandwidth, {peak_kind}",
-              "ids": "drawn like the workload's candidates, repeats allowed"}
+              "ids": "distinct rows (seeded permutation of the table): every row comes from HBM once",
+              "table_bytes": int(table["E"].shape[0]) * row_bytes}
     gather["frac"] = gather["achieved"] / gather["peak"]
+    gather["frac_nominal"] = gather["achieved"] / NOMINAL_HBM_GBS
+    rep_gbs = gn * (2 * row_bytes + 4) / (g_ms * 1e-3) / 1e9
+    gather["with_repeats"] = {"rows": gn, "ms": g_ms, "achieved": rep_gbs, "frac": rep_gbs / float(peaks["hbm_gbs"]),
+                              "ids": "drawn like the workload's candidates (Zipf), repeats allowed: hot rows are served by L2"}
+    gt = ncu_traffic_table().get(("gather_stage", "k_gather_rows"))
+    gather["traffic"] = None if gt is None else int(gt[1] * (gd if gt[0] == "per_candidate" else 1))
     top = max(kavg, key=kavg.get)
     tensor = bool(srv.ctx.get_stats().tensor_path) and top != "interact"
     kf = kernel_flops(top, wl, cands)
@@ -408,11 +451,16 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
         roof["lsh_note"] = (f"eqs. 6-7 need {wl.lsh_bits // 32} xor + popc on 32-bit words per (candidate, key) pair by the definition; "
                             f"the kernel gets the counts from a +-1 fp8 product ({2 * wl.lsh_bits} tensor flop per pair, not counted "
                             "in `achieved`) and spends about ten integer / fp32 instructions per pair on conversion and tiers")
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get((wl.name, top))
+    if tensor:
+        roof["frac_nominal"] = roof["achieved"] / NOMINAL_BF16_TFLOPS
+        roof["peak_nominal"] = NOMINAL_BF16_TFLOPS
+    traffic = ncu_traffic_table().get((wl.name, top))
+    roof["traffic"] = None if traffic is None else int(traffic[1] * (cands if traffic[0] == "per_candidate" else 1))
+    roof["traffic_source"] = None if traffic is None else f"ncu dram bytes read + write, {traffic[0].replace('_', ' ')}"
     roof["kernel_ms"] = kavg
 
     value = world * cands * steps / (total_ms * 1e-3)
-    per_request_ms = [t / (wl.R if batch else 1) for t in times]
+    per_request_ms = [t / (wl.R if batch else 1) for t in lat_times]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": max(3, warmup),
         "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -424,8 +472,12 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
                    "request_pool": pool},
         "p50_ms_per_request": float(np.percentile(per_request_ms, 50)),
         "p99_ms_per_request": float(np.percentile(per_request_ms, 99)),
+        "latency_samples": {"scoring_calls": len(lat_times), "requests_per_call": wl.R if batch else 1},
         "flops_per_candidate": flops_per_candidate(wl)["total"],
         "step_tflops": flops_per_candidate(wl)["total"] * cands * steps / (total_ms * 1e-3) / 1e12,
+        "step_frac": {"of_measured_peak": flops_per_candidate(wl)["total"] * cands * steps / (total_ms * 1e-3) / 1e12 / float(peaks["bf16_tflops"]),
+                      "of_nominal_peak": flops_per_candidate(wl)["total"] * cands * steps / (total_ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS}
+        if wl.dtype == "bf16" else None,
         "e2e": {"value": world * cands * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * cands,
                 "d2h_bytes_per_step": 4 * cands, "steps": e2e_steps},
         "gpu_launches": int(launches),
@@ -453,6 +505,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--also", default="c3,c4,c4_lsh,c4_both,c5", help="other workloads measured briefly after the main one ('' = none)")
     # scaled copies of a workload, for profiler captures that must stay small (the defaults are the full sizes)
+    ap.add_argument("--latency-calls", type=int, default=-1, help="scoring calls of the latency pass (default: 1000, fewer for long steps)")
     ap.add_argument("--requests", type=int, default=0, help="override the number of requests per step")
     ap.add_argument("--rows", type=int, default=0, help="override the rows of the item table")
     args = ap.parse_args()

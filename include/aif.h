@@ -14,8 +14,9 @@
  * Conventions
  *   - Every function returns an int: AIF_OK (0) or a negative AIF_ERR_* code.  Nothing throws, aborts or
  *     traps the GPU.  Argument, shape and version errors are returned at once.  What only the GPU can
- *     see (a candidate id outside the table) sets a bit in a device status word, the affected logit is
- *     NaN, and aif_poll_status reports it.
+ *     see (a candidate id outside the table, a bounded device-side wait that ran out) sets a bit in a device status
+ *     word, the affected logits are NaN, and aif_poll_status reports it.  AIF_STATUS_TIMEOUT stays set until it is
+ *     polled, and while it is set the kernel-per-layer path answers NaN: poll after a timeout before scoring on.
  *   - "device" pointers are GPU global memory, "host" pointers are ordinary host memory; the comment of
  *     each argument says which.  The caller owns every buffer it passes; the context owns the item
  *     table, the weight copies, the user-state arena and its scratch memory.
@@ -250,7 +251,9 @@ int aif_score(aif_ctx *ctx, const aif_user_state *state, const int32_t *cand_ids
 
 /* Many requests in one launch.  states: host array [n_req]; offsets: host int64 [n_req + 1], ascending, request
  * r owns cand_ids[offsets[r] .. offsets[r+1]) and the same range of logits (both device).  The small request
- * table is staged through pinned memory owned by the context (one asynchronous copy per call). */
+ * table is staged through pinned memory owned by the context (one asynchronous copy per call).
+ * Errors: AIF_ERR_SHAPE also when the launch needs more 128-candidate tiles than the context's tile table holds (it is
+ * sized from max_batch_candidates, mini_batch and max_user_states, so only a call beyond those limits can get there). */
 int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *states, const int32_t *cand_ids,
                     const int64_t *offsets, float *logits, aif_stream stream);
 
@@ -262,6 +265,14 @@ int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *st
  * benchmark times. */
 int aif_score_host(aif_ctx *ctx, const aif_user_state *state, const int32_t *host_ids, int32_t n,
                    float *host_logits, aif_stream stream);
+
+/* aif_score_batch for callers whose buffers live in host memory (Section 3.1: the real-time phase is handed candidate ids
+ * by the retrieval service and hands scores back to it): host_ids (host int32, all requests concatenated) are copied to the
+ * device on `stream`, scored in one launch, and the logits copied back into host_logits (host fp32); returns after the
+ * stream has drained.  Page-locked buffers make both copies asynchronous transfers of the copy engine; pageable ones are
+ * staged by the runtime.  states, offsets: as for aif_score_batch.  Errors as for aif_score_batch. */
+int aif_score_batch_host(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *states, const int32_t *host_ids,
+                         const int64_t *offsets, float *host_logits, aif_stream stream);
 
 /* Scoring for callers that cannot allocate device memory.  (The paper has no counterpart to this call; it exists
  * for deployment reasons only.)  Some hosts of this library never get to call cudaMalloc after start-up: a plug-in

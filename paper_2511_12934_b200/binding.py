@@ -82,7 +82,7 @@ EXPORTS = [
     "aif_input_width", "aif_mix64", "aif_create", "aif_destroy", "aif_load_weights", "aif_item_nearline_refresh",
     "aif_load_item_weights", "aif_item_nearline_compute",
     "aif_user_precompute", "aif_user_release", "aif_user_request_key", "aif_user_state_export", "aif_user_state_export_bea", "aif_score",
-    "aif_score_batch", "aif_score_host", "aif_score_noalloc", "aif_gather_rows", "aif_gather_sidecars", "aif_poll_status", "aif_get_stats",
+    "aif_score_batch", "aif_score_host", "aif_score_batch_host", "aif_score_noalloc", "aif_gather_rows", "aif_gather_sidecars", "aif_poll_status", "aif_get_stats",
     "aif_set_kernel_timing", "aif_get_kernel_timing", "aif_kernel_launches", "aif_selftest_bounded_wait", "aif_strerror", "aif_last_error",
 ]
 
@@ -115,6 +115,7 @@ def load_library(path: Optional[str] = None):
     lib.aif_score.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.aif_score_batch.argtypes = [vp, i32, C.POINTER(vp), vp, C.POINTER(i64), vp, vp]
     lib.aif_score_host.argtypes = [vp, vp, vp, i32, vp, vp]
+    lib.aif_score_batch_host.argtypes = [vp, i32, C.POINTER(vp), vp, C.POINTER(i64), vp, vp]
     lib.aif_score_noalloc.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.aif_gather_rows.argtypes = [vp, vp, i64, vp, vp]
     lib.aif_gather_sidecars.argtypes = [vp, vp, i64, vp, vp, vp]
@@ -337,6 +338,16 @@ class Aif:
         assert not host_ids.is_cuda and not host_logits.is_cuda
         _check(self.lib.aif_score_host(self.h, state.handle, C.c_void_p(host_ids.data_ptr()), host_ids.numel(),
                                        C.c_void_p(host_logits.data_ptr()), _stream(stream)), "aif_score_host")
+
+    def score_batch_host(self, states: Sequence[UserState], host_ids: torch.Tensor, offsets: Sequence[int],
+                         host_logits: torch.Tensor, stream=None):
+        """aif_score_batch with CPU tensors (int32 ids of all requests concatenated, float32 logits)."""
+        assert not host_ids.is_cuda and not host_logits.is_cuda
+        n = len(states)
+        hs = (C.c_void_p * n)(*[s.handle for s in states])
+        off = (C.c_int64 * (n + 1))(*[int(o) for o in offsets])
+        _check(self.lib.aif_score_batch_host(self.h, n, hs, C.c_void_p(host_ids.data_ptr()), off,
+                                             C.c_void_p(host_logits.data_ptr()), _stream(stream)), "aif_score_batch_host")
 
     # -- status ----------------------------------------------------------------------------------
     def poll_status(self) -> int:

@@ -613,6 +613,25 @@ int aif_score_host(aif_ctx *ctx, const aif_user_state *state, const int32_t *hos
     return AIF_OK;
 }
 
+int aif_score_batch_host(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *states, const int32_t *host_ids,
+                         const int64_t *offsets, float *host_logits, aif_stream stream)
+{
+    if (!ctx || !states || !offsets || n_req < 0) return AIF_ERR_ARG;
+    if (n_req == 0) return AIF_OK;
+    const int64_t total = offsets[n_req];
+    if (total < 0 || total > ctx->cfg.max_batch_candidates) return AIF_ERR_SHAPE;
+    if (total == 0) return AIF_OK;
+    if (!host_ids || !host_logits) return AIF_ERR_ARG;
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = as_stream(stream);
+    AIF_CUDA(cudaMemcpyAsync(ctx->ids_stage, host_ids, (size_t)total * 4, cudaMemcpyHostToDevice, st));
+    const int rc = aif_score_batch(ctx, n_req, states, ctx->ids_stage, offsets, ctx->logits_stage, stream);
+    if (rc != AIF_OK) return rc;
+    AIF_CUDA(cudaMemcpyAsync(host_logits, ctx->logits_stage, (size_t)total * 4, cudaMemcpyDeviceToHost, st));
+    AIF_CUDA(cudaStreamSynchronize(st));
+    return AIF_OK;
+}
+
 int aif_gather_rows(aif_ctx *ctx, const int32_t *ids, int64_t n, void *rows_out, aif_stream stream)
 {
     if (!ctx || n < 0) return AIF_ERR_ARG;

@@ -231,6 +231,9 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
         unsigned char *stg = out_stage + warp * (C::kSlabs * 2048);
         uint32_t slab = 0;
         int it = 0;
+        // a wait that ran out in an earlier kernel of this call left its outputs unwritten: logits computed from them are
+        // replaced by NaN
+        const bool poisoned = p.epi == EPI_DOT && (*reinterpret_cast<volatile const uint32_t *>(p.sl.status) & AIF_STATUS_TIMEOUT) != 0u;
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
             const int grp = item / n_ncg, nc = (item - grp * n_ncg) * NB + (NB == 2 ? a : 0), n0 = nc * p.n_cols;
             const int buf = kAcc == 1 ? (it & 1) : a;
@@ -244,13 +247,15 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
                 }
             }
             named_bar_sync(1 + a, 128);
-            if (!mbar_wait(smem_u32(acc_full + buf), ph, abort_flag)) break;
+            // a wait that ran out is carried to the barrier at the end of the item, so that the four warps of an
+            // accumulator leave together and none is left waiting there
+            const bool got = __all_sync(0xffffffffu, mbar_wait(smem_u32(acc_full + buf), ph, abort_flag));
             tc_fence_after();
             const bool valid = row < t.cnt;
             const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(buf * 256);
             float dot = 0.f;
             const float floor_v = p.linear_out ? -INFINITY : 0.f;
-            if (t.cnt > 0) {
+            if (got && t.cnt > 0) {
                 for (int c0 = 0; c0 < p.n_cols; c0 += 32) {
                     uint32_t r[32];
                     tmem_ld32(taddr + (uint32_t)c0, r);
@@ -321,15 +326,17 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(acc_empty + buf));
+            if (got && lane == 0) mbar_arrive(smem_u32(acc_empty + buf));
             if (p.epi == EPI_DOT && valid) {
                 float logit = dot + p.b_out[0];
                 if (p.emit_sigmoid) logit = 1.0f / (1.0f + expf(-logit));
                 const int id = p.sl.ids[t.pos0 + row];
-                if (id < 0 || (int64_t)id >= p.M) logit = __int_as_float(0x7fc00000);
+                // no number for an id outside the table, nor for a tile whose inputs never arrived (here or in an
+                // earlier kernel of the call: the status word says so)
+                if (id < 0 || (int64_t)id >= p.M || !got || poisoned) logit = __int_as_float(0x7fc00000);
                 p.sl.logits[t.pos0 + row] = logit;
             }
-            named_bar_sync(1 + a, 128);
+            if (named_bar_or(1 + a, 128, !got)) break;
         }
         if (lane == 0) bulk_wait<0>();   // all tile stores of this warp have reached global memory
     } else if (warp == C::kMmaWarp) {
@@ -419,10 +426,13 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
             }
             pend = id;
         };
-        auto publish = [&](int buf, int pend) {
-            named_bar_sync(9, C::kProdThreads);   // every producer thread is done reading what this buffer held
+        // returns true if some producer thread's wait ran out: they all learn it here and leave together, so that none
+        // is left waiting at this barrier
+        auto publish = [&](int buf, int pend, bool failed) {
+            const bool any = named_bar_or(9, C::kProdThreads, failed);   // every producer thread is done reading what this buffer held
             ids_s[(buf * G + gt) * 128 + lp] = pend;
             named_bar_sync(9, C::kProdThreads);
+            return any;
         };
         // bucket of this thread's rows in the field its slot of chunk kc belongs to (cross chunks only); rows outside
         // the tile read other candidates' entries or stale scratch, which rowmask discards
@@ -488,20 +498,24 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
         for (int i = 0; i < 8; ++i) off[i] = 0, raw[i] = 0;
         if ((int)blockIdx.x < n_items) {
             load_rows(blockIdx.x, cur, pend);
-            publish(0, pend);
+            publish(0, pend, false);
             resolve(0, cur, ids_s + gt * 128, raw, false, bp, off, mask, tma_x, tma_y);
             if (deep) fetch(1, cur, raw);
         }
         nxt = cur;
-        for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, buf ^= 1) {
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x, buf ^= 1) {
             const int next_item = item + gridDim.x;
             const bool has_next = next_item < n_items;
             const int *ids_cur = ids_s + (buf * G + gt) * 128, *ids_nxt = ids_s + ((buf ^ 1) * G + gt) * 128;
             if (has_next) load_rows(next_item, nxt, pend);   // the id load lands while chunk 0 is copied
+            bool all_out = false;
             for (int kc = 0; kc < p.n_k; ++kc) {
-                if (!mbar_wait(smem_u32(empty_a + s), ph ^ 1u, abort_flag)) {
-                    ok = false;
-                    break;
+                // a thread whose wait ran out keeps walking (no copies, no arrivals) until the next publish barrier
+                if (ok && !mbar_wait(smem_u32(empty_a + s), ph ^ 1u, abort_flag)) ok = false;
+                if (!ok) {
+                    if (kc == 0 && has_next) all_out = publish(buf ^ 1, pend, true);
+                    if (all_out) break;
+                    continue;
                 }
                 if (tma_x == -1) {
                     const uint32_t dst0 = smem_u32(smA + s * C::kAStage) + a_off;
@@ -517,7 +531,10 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
                 // the stage's barrier receives this thread's arrival when its copies have landed: no thread waits for them
                 cp_async_arrive_noinc(smem_u32(full_a + s));
                 if (++s == kSA) s = 0, ph ^= 1u;
-                if (kc == 0 && has_next) publish(buf ^ 1, pend);
+                if (kc == 0 && has_next && publish(buf ^ 1, pend, false)) {
+                    all_out = true;
+                    break;
+                }
                 // sources of the next chunk from the buckets fetched one iteration ago; then start the fetch for the
                 // chunk after it, so that its latency is covered by a whole iteration
                 if (kc + 1 < p.n_k) resolve(kc + 1, cur, ids_cur, raw, deep, bp, off, mask, tma_x, tma_y);
@@ -527,6 +544,7 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
                     else if (has_next) fetch(kc + 2 - p.n_k, nxt, raw);
                 }
             }
+            if (all_out) break;
             cur = nxt;
         }
         cp_async_wait_all();

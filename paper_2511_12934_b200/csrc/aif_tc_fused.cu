@@ -360,11 +360,11 @@ __global__ void __launch_bounds__(kFThreads, 1) k_request_fused(const __grid_con
             dot = (d4[0] + d4[1]) + (d4[2] + d4[3]);
         }
         if (g == 1) dot_s[row] = dot;
-        named_bar_sync(1, 256);
-        if (g == 0 && ok && row < cnt) {
+        const bool all_ok = !named_bar_or(1, 256, !ok);   // also orders dot_s; a wait that ran out anywhere in these warps
+        if (g == 0 && row < cnt) {
             float logit = dot + dot_s[row] + b_out;
             if (p.emit_sigmoid) logit = 1.0f / (1.0f + expf(-logit));
-            if (!good) logit = __int_as_float(0x7fc00000);
+            if (!good || !all_ok) logit = __int_as_float(0x7fc00000);   // no number for a bad id, nor for a tile whose wait ran out
             p.sl.logits[pos0 + row] = logit;
         }
     } else if (warp == kFMmaWarp) {

@@ -15,16 +15,20 @@
 //
 // One CTA per SM walks over the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Warps at d = 128 (512 threads; d = 256 in
 // brackets, 256 threads):
-//   0-7 [0-3]  per key block: read the score row from tensor memory, write 2 matches back into the same columns as
-//              packed bf16 pairs (A operand of the second product, never in shared memory), count the tiers.  A thread
-//              owns a candidate row; at d = 128 two warps share each quarter of the rows, each with half of a block's
-//              keys.  At the end of a tile the SimTier columns are written.
+//   0-7 [0-3]  per key block: read the score row from tensor memory, write 2 matches as packed bf16 pairs into the P
+//              buffer (A operand of the second product, never in shared memory), count the tiers.  A thread owns a
+//              candidate row; at d = 128 two warps share each quarter of the rows and take alternate key blocks.  At the
+//              end of a tile the SimTier columns are written.
 //   8  [4]     allocates tensor memory; one lane issues the signature products, up to two blocks ahead
-//   9  [5]     one lane streams the key blocks with TMA: the +-1 signatures and the rows of S
+//   9  [5]     one lane streams the key blocks with TMA, the +-1 signatures (ahead) and the rows of S through rings of their own
 //   10 [6]     expands the item signatures of the next tile into one of two operand buffers
 //   11 [7]     one lane issues O += P S
 //   12-15      d = 128 only: scale the finished tile's O accumulator and store the LSH-DIN rows while the other warps are
-//              on the next tile
+//              on the next tile's first blocks
+// Tensor memory: two score buffers, two P buffers, one O accumulator.  P has columns of its own, so that the signature
+// product of block j + 2 waits only until the scores of block j are in registers and not for the product that reads P_j:
+// with P written over the scores, a block's period was the sum of both products, both conversions' latencies and four
+// barrier round trips, divided by two buffers (1470 cycles per 128-key block at d = 128 with next to no conversion work).
 // Every wait is bounded.
 #include "aif_device.cuh"
 #include "aif_internal.h"
@@ -44,7 +48,6 @@ struct LshParams {
     int32_t x_din;           // first LSH-DIN column of X, or -1: block off
     int32_t x_tier;          // first SimTier column of X (64 columns, the first n_tiers used), or -1
     int32_t n_tiers;
-    uint32_t tier_mul, tier_add;   // tier = ((bits of (score + d' + 2^23)) * tier_mul + tier_add) >> 24, see launch_lsh_tc
     int32_t din_mean, tier_mean;   // divide by the sequence length
     __nv_bfloat16 *X;
 };
@@ -54,14 +57,19 @@ struct LshCfg {
     static constexpr int kQChunks = D / 128;             // 128-byte chunks of a +-1 signature row (one byte per bit)
     static constexpr int kQBytes = kQChunks * 128 * 128;
     static constexpr int kQBufs = 2;
-    static constexpr int kStages = 3;
+    // key blocks arrive through two rings: the +-1 signatures (needed two blocks ahead, by the first product) and the rows
+    // of S (needed by the second product, and held until it completes)
+    static constexpr int kStagesG = D <= 128 ? 4 : 3, kStagesV = 3;
     static constexpr int kVChunks = D / 64;              // 64-column (128-byte) chunks of a row of S
     static constexpr int kVChunkBytes = BN * 128;
     static constexpr int kVBytes = kVChunks * kVChunkBytes;
     static constexpr int kGChunkBytes = BN * 128;        // one 128-bit chunk of a key block's signatures
     static constexpr int kGBytes = kQChunks * kGChunkBytes;
-    static constexpr int kStageBytes = kVBytes + kGBytes;
-    static constexpr int kTmemO = 2 * BN;
+    // tensor memory: two score buffers, two P buffers of their own (BN / 2 columns of packed bf16 pairs each: the next
+    // signature product only waits until the scores are in registers, not for the product that reads P), one O accumulator
+    static constexpr int kTmemP = 2 * BN;
+    static constexpr int kTmemO = D <= 128 ? 384 : 256;
+    static_assert(kTmemP + BN <= kTmemO && kTmemO + D <= 512, "tensor memory");
     static constexpr bool kSplitEpi = D <= 128;
     static constexpr int kHalves = D <= 128 ? 2 : 1;
     static constexpr int kConvWarps = 4 * kHalves;
@@ -71,7 +79,7 @@ struct LshCfg {
     // tier counters [tile parity][half][tier][row] (two parities only where two warps share a row)
     static constexpr int kTierBufs = kHalves == 2 ? 2 : 1;
     static constexpr int kTierBytes = kTierBufs * kHalves * kTierSlots * 128 * 4;
-    static constexpr size_t kSmem = 1024 + kQBufs * kQBytes + kStages * kStageBytes + 512 + kTierBytes;
+    static constexpr size_t kSmem = 1024 + kQBufs * kQBytes + kStagesG * kGBytes + kStagesV * kVBytes + 512 + kTierBytes;
     static_assert(kSmem <= 227 * 1024, "shared memory");
     static_assert(kQBytes >= 16384, "output staging lives in the signature buffer");
 };
@@ -115,11 +123,78 @@ __device__ __forceinline__ uint4 expand16(uint32_t b0, uint32_t b1)
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-__device__ __forceinline__ uint32_t shl_clamped(uint32_t v, uint32_t by)   // 0 once `by` reaches 32, as PTX defines shl
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 {
     uint32_t r;
-    asm("shl.b32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(by));
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
     return r;
+}
+
+// A chunk of a candidate row's scores against a key block: 32 scores (2 matches - d', exact integers in fp32) -> P = 2 matches as packed
+// bf16 pairs, and the tier counts in 8-bit counters (tier t in byte t & 3 of cnt[t >> 2]), 32 keys at a time.
+//
+// Tier of a pair (eq. 9, equal-width tiers, the last one closed): n = floor(matches N / d').  d' is a power of two here, so
+// 2 matches * (N / 2 d') is exact in fp32 and a fused multiply-add that rounds towards minus infinity onto 1.5 * 2^23 leaves
+// n in the low mantissa bits (fp32 counts in ones between 2^23 and 2^24).  An integer multiply by 0x1111 copies n into the
+// four low nibbles.  Up to eight tiers: adding 0x0123 makes nibble p equal to n + 3 - p, which is 3 exactly where p = n and 7
+// where p + 4 = n, never carries (n <= 8) and has bit 3 set (the byte permute's sign-replicating mode: zero for these
+// pools) when it is 8 or more; byte permutes with that selector over a pool whose byte 3, or byte 7, is 0x01 yield the
+// increments 1 << 8 n of the two packed counters.  More than eight tiers: the nibbles are xor-ed with their positions
+// instead (p ^ n is zero only where p = n) and n is capped at 15.  matches = d' gives n = N, one past the last tier: those
+// pairs land in no counted slot and the last tier is derived from the total.  The per-thread work here is what bounds
+// the kernel (about seven instructions per pair with SimTier on), so every instruction counts.
+template <int D, bool TIERS, bool WIDE>
+__device__ __forceinline__ void lsh_convert(const uint32_t (&sc)[32], float c1, float n_cap, uint32_t p_col, uint32_t (&cnt)[4])
+{
+    uint32_t packed[16];
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        const float p0 = __uint_as_float(sc[i]) + (float)D, p1 = __uint_as_float(sc[i + 1]) + (float)D;   // 2 matches
+        if (TIERS) {
+            float w0 = __fmaf_rd(p0, c1, 12582912.0f), w1 = __fmaf_rd(p1, c1, 12582912.0f);
+            if (WIDE) {
+                w0 = fminf(w0, n_cap), w1 = fminf(w1, n_cap);
+                const uint32_t r0 = __float_as_uint(w0) * 0x1111u, r1 = __float_as_uint(w1) * 0x1111u;
+                cnt[0] += prmt(1u, 0u, r0 ^ 0x3210u) + prmt(1u, 0u, r1 ^ 0x3210u);
+                cnt[1] += prmt(0u, 1u, r0 ^ 0x3210u) + prmt(0u, 1u, r1 ^ 0x3210u);
+                cnt[2] += prmt(1u, 0u, r0 ^ 0xBA98u) + prmt(1u, 0u, r1 ^ 0xBA98u);
+                cnt[3] += prmt(0u, 1u, r0 ^ 0xBA98u) + prmt(0u, 1u, r1 ^ 0xBA98u);
+            } else {
+                const uint32_t s0 = __float_as_uint(w0) * 0x1111u + 0x0123u, s1 = __float_as_uint(w1) * 0x1111u + 0x0123u;
+                cnt[0] += prmt(0x01000000u, 0u, s0) + prmt(0x01000000u, 0u, s1);
+                cnt[1] += prmt(0u, 0x01000000u, s0) + prmt(0u, 0x01000000u, s1);
+            }
+        }
+        const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+        packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
+    }
+    tmem_st16(p_col, packed);
+}
+
+// One key block of a candidate row: BN scores from the score buffer at s_col -> P at p_col and the packed tier counts,
+// 32 columns at a time with the load of the next chunk in flight while one is converted.  Returns after the last load
+// has landed and `s_free` has been told so; the stores may still be in flight.
+// Columns beyond the sequence need no special case: their signatures and their rows of S are zero (the user side pads
+// both to the key block), so they add nothing to O, and their score of 0 (matches = d' / 2) lands in tier floor(N / 2),
+// from which the caller takes them out again.
+template <int D, int BN, bool TIERS, bool WIDE>
+__device__ __forceinline__ void lsh_block(uint32_t s_col, uint32_t p_col, float c1, float n_cap, uint32_t s_free_bar, uint32_t (&cnt)[4])
+{
+    uint32_t ra[32], rb[32];
+    tmem_ld32(s_col, ra);
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += 64) {
+        tmem_ld_wait();
+        tmem_ld32(s_col + (uint32_t)(c0 + 32), rb);
+        lsh_convert<D, TIERS, WIDE>(ra, c1, n_cap, p_col + (uint32_t)(c0 >> 1), cnt);
+        tmem_ld_wait();
+        if (c0 + 64 < BN) tmem_ld32(s_col + (uint32_t)(c0 + 64), ra);
+        else {   // all scores are in registers: the signature product of block gb + 2 may overwrite the buffer
+            tc_fence_before();
+            mbar_arrive(s_free_bar);
+        }
+        lsh_convert<D, TIERS, WIDE>(rb, c1, n_cap, p_col + (uint32_t)((c0 + 32) >> 1), cnt);
+    }
 }
 
 template <int D, int BN>
@@ -128,17 +203,18 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
                                                                          const __grid_constant__ CUtensorMap tmapX, const LshParams p)
 {
     using C = LshCfg<D, BN>;
-    constexpr int kS = C::kStages, kQB = C::kQBufs;
+    constexpr int kSG = C::kStagesG, kSV = C::kStagesV, kQB = C::kQBufs;
     constexpr bool kSplit = C::kSplitEpi;
-    constexpr int kH = C::kHalves, CW = BN / kH;
+    constexpr int kH = C::kHalves;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
     unsigned char *smQ = base;
-    unsigned char *smKV = smQ + kQB * C::kQBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smKV + kS * C::kStageBytes);
-    uint64_t *kv_full = bars, *kv_empty = bars + kS;
-    uint64_t *s_full = bars + 2 * kS, *p_full = s_full + 2, *pv_done = p_full + 2;
-    uint64_t *q_full = pv_done + 2, *q_empty = q_full + 2, *o_final = q_empty + 2, *o_free = o_final + 2;
+    unsigned char *smV = smQ + kQB * C::kQBytes;
+    unsigned char *smG = smV + kSV * C::kVBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smG + kSG * C::kGBytes);
+    uint64_t *v_full = bars, *v_empty = bars + kSV, *g_full = v_empty + kSV, *g_empty = g_full + kSG;
+    uint64_t *s_full = g_empty + kSG, *p_full = s_full + 2, *pv_done = p_full + 2, *s_free = pv_done + 2;
+    uint64_t *q_full = s_free + 2, *q_empty = q_full + 2, *o_final = q_empty + 2, *o_free = o_final + 2;
     uint64_t *q_first = o_free + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_first + 1);
     volatile uint32_t *abort_flag = tmem_slot + 1;
@@ -147,14 +223,19 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
-        for (int s = 0; s < kS; ++s) {
-            mbar_init(smem_u32(kv_full + s), 1);
-            mbar_init(smem_u32(kv_empty + s), 1);
+        for (int s = 0; s < kSV; ++s) {
+            mbar_init(smem_u32(v_full + s), 1);
+            mbar_init(smem_u32(v_empty + s), 1);
+        }
+        for (int s = 0; s < kSG; ++s) {
+            mbar_init(smem_u32(g_full + s), 1);
+            mbar_init(smem_u32(g_empty + s), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(s_full + b), 1);
-            mbar_init(smem_u32(p_full + b), C::kConvWarps * 32);
+            mbar_init(smem_u32(p_full + b), 128);
             mbar_init(smem_u32(pv_done + b), 1);
+            mbar_init(smem_u32(s_free + b), 128);
             mbar_init(smem_u32(q_full + b), 32);
             mbar_init(smem_u32(q_empty + b), 5);   // the tenant's last signature product, and the four output warps' staging
             mbar_init(smem_u32(o_final + b), 1);
@@ -193,8 +274,8 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
     auto tile_epilogue = [&](int k, const LshTile &t, int wq, int lane) {
         const int row = wq * 32 + lane;
         const uint32_t lane_base = tmem_base + ((uint32_t)(wq * 32) << 16);
-        const uint32_t o_col = (uint32_t)(C::kTmemO + (kSplit ? (k & 1) * D : 0));
-        uint64_t *o_free_k = o_free + (kSplit ? (k & 1) : 0);
+        const uint32_t o_col = (uint32_t)C::kTmemO;
+        uint64_t *o_free_k = o_free;
         const float scale = (0.5f / (float)D) * (p.din_mean ? 1.0f / (float)t.L : 1.0f);
         bool good = false;
         if (row < t.cnt) {
@@ -269,8 +350,9 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
         const int wq = warp & 3, half = warp >> 2;
         const int row = wq * 32 + lane;
         const uint32_t lane_base = tmem_base + ((uint32_t)(wq * 32) << 16);
-        const float magic = (float)D + 8388608.0f;   // score + magic has 2 matches in its low mantissa bits
-        const bool wide = p.n_tiers > 8;
+        const bool tiers = p.x_tier >= 0, wide = p.n_tiers > 8;
+        // constants of the tier arithmetic (lsh_convert)
+        const float tc1 = (float)p.n_tiers / (float)(2 * D), n_cap = 12582912.0f + 15.0f;
         bool ok = true;
         uint32_t gb = 0;
         int k = 0;
@@ -295,92 +377,66 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
             const LshTile t = lsh_tile<BN>(p, tile);
             const int L = t.L;
             uint32_t *tc = tier_s + (((kH == 2 ? (k & 1) * kH : 0) + half) * kTierSlots) * 128 + row;   // this thread's counters, stride 128
-            int n_valid = 0;
+            int n_valid = 0, n_pad = 0;   // keys this thread has counted, and columns beyond the sequence it has converted
             for (int j = 0; j < t.nb; ++j, ++gb) {
+                // d = 128: the two warps of a row quarter take alternate key blocks (block gb, and with it score and P buffer
+                // gb & 1, belongs to warp half gb & 1), so that one converts while the other sits in its waits
+                if (kH == 2 && (int)(gb & 1u) != half) continue;
                 const int b = (int)(gb & 1u);
-                const int valid_cols = min(BN, L - j * BN);
-                const int vc = max(0, min(CW, valid_cols - half * CW));   // this warp's keys of the block that exist
-                const bool got = __all_sync(0xffffffffu, mbar_wait(smem_u32(s_full + b), (gb >> 1) & 1u, abort_flag));
-                const uint32_t ts = lane_base + (uint32_t)(b * BN);
-                uint32_t sc[CW];
-                if (got) {
-                    tc_fence_after();
-#pragma unroll
-                    for (int c0 = 0; c0 < CW; c0 += 32)
-                        tmem_ld32(ts + (uint32_t)(half * CW + c0), *reinterpret_cast<uint32_t(*)[32]>(&sc[c0]));
-                    tmem_ld_wait();
-                }
-                if (kH == 2) {
-                    // orders this warp's score loads before the partner's stores, which for the second half land in the
-                    // first half's columns; a failed wait is carried through the barrier so that both warps leave together
-                    tc_fence_before();
-                    const bool bad = named_bar_or(1 + wq, 64, !got);
-                    tc_fence_after();
-                    if (bad) {
-                        ok = false;
-                        break;
-                    }
-                } else if (!got) {
+                const int vc = min(BN, L - j * BN);   // keys of the block that exist
+                if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(s_full + b), (gb >> 1) & 1u, abort_flag))) {
                     ok = false;
                     break;
                 }
-                // 8-bit counters of this block (at most 64 keys per thread), tier t in byte t of c01 (t < 8) or c23
-                uint32_t c0r = 0u, c1r = 0u, c2r = 0u, c3r = 0u;
-#pragma unroll
-                for (int c0 = 0; c0 < CW; c0 += 64) {
-                    uint32_t packed[32];
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float s0 = __uint_as_float(sc[c0 + 2 * i]), s1 = __uint_as_float(sc[c0 + 2 * i + 1]);
-                        float p0 = s0 + (float)D, p1 = s1 + (float)D;          // 2 matches
-                        uint32_t sh0 = ((__float_as_uint(s0 + magic) * p.tier_mul + p.tier_add) >> 21) & 0xF8u;   // 8 tier
-                        uint32_t sh1 = ((__float_as_uint(s1 + magic) * p.tier_mul + p.tier_add) >> 21) & 0xF8u;
-                        if (vc != CW) {
-                            if (c0 + 2 * i >= vc) p0 = 0.f, sh0 = 255u;
-                            if (c0 + 2 * i + 1 >= vc) p1 = 0.f, sh1 = 255u;
-                        }
-                        c0r += shl_clamped(1u, sh0) + shl_clamped(1u, sh1);
-                        c1r += shl_clamped(1u, sh0 - 32u) + shl_clamped(1u, sh1 - 32u);
-                        if (wide) {
-                            c2r += shl_clamped(1u, sh0 - 64u) + shl_clamped(1u, sh1 - 64u);
-                            c3r += shl_clamped(1u, sh0 - 96u) + shl_clamped(1u, sh1 - 96u);
-                        }
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                        packed[i] = *reinterpret_cast<const uint32_t *>(&h);
-                    }
-                    tmem_st32(ts + (uint32_t)((half * CW + c0) >> 1), packed);
+                tc_fence_after();
+                // P buffer b was last read by the product of block gb - 2
+                if (gb >= 2 && !__all_sync(0xffffffffu, mbar_wait(smem_u32(pv_done + b), ((gb - 2) >> 1) & 1u, abort_flag))) {
+                    ok = false;
+                    break;
                 }
+                tc_fence_after();
+                const uint32_t s_col = lane_base + (uint32_t)(b * BN), p_col = lane_base + (uint32_t)(C::kTmemP + b * (BN / 2));
+                uint32_t cnt[4] = {0u, 0u, 0u, 0u};
+                if (!tiers) lsh_block<D, BN, false, false>(s_col, p_col, tc1, n_cap, smem_u32(s_free + b), cnt);
+                else if (!wide) lsh_block<D, BN, true, false>(s_col, p_col, tc1, n_cap, smem_u32(s_free + b), cnt);
+                else lsh_block<D, BN, true, true>(s_col, p_col, tc1, n_cap, smem_u32(s_free + b), cnt);
                 tmem_st_wait();
                 tc_fence_before();
                 mbar_arrive(smem_u32(p_full + b));
-                // the block's counts into the tile's 32-bit counters
-                n_valid += vc;
-                if (p.x_tier >= 0) {
+                n_valid += vc, n_pad += BN - vc;
+                // the block's packed counts (at most 128 per slot) into the tile's 32-bit counters
+                if (tiers) {
 #pragma unroll
                     for (int t4 = 0; t4 < 4; ++t4) {
-                        tc[t4 * 128] += (c0r >> (8 * t4)) & 0xFFu;
-                        tc[(4 + t4) * 128] += (c1r >> (8 * t4)) & 0xFFu;
+                        tc[t4 * 128] += (cnt[0] >> (8 * t4)) & 0xFFu;
+                        tc[(4 + t4) * 128] += (cnt[1] >> (8 * t4)) & 0xFFu;
                     }
                     if (wide) {
 #pragma unroll
                         for (int t4 = 0; t4 < 4; ++t4) {
-                            tc[(8 + t4) * 128] += (c2r >> (8 * t4)) & 0xFFu;
-                            tc[(12 + t4) * 128] += (c3r >> (8 * t4)) & 0xFFu;
+                            tc[(8 + t4) * 128] += (cnt[2] >> (8 * t4)) & 0xFFu;
+                            tc[(12 + t4) * 128] += (cnt[3] >> (8 * t4)) & 0xFFu;
                         }
                     }
                 }
             }
-            if (!ok) break;
             // ---- SimTier columns of the tile (eq. 9): 64 bf16 per row, the first n_tiers used
             if (p.x_tier >= 0) {
                 if (kH == 2) {
-                    tc[15 * 128] = (uint32_t)n_valid;   // slot 15 is free: the last tier is derived from the total
-                    named_bar_sync(1 + wq, 64);
-                }
+                    // the two warps of a row quarter meet here once per tile; a failed wait is carried through the barrier so
+                    // that both leave together
+                    // slot 15 is free (the last tier is derived from the total): this warp's totals for its partner
+                    tc[15 * 128] = (uint32_t)n_valid | ((uint32_t)n_pad << 24);
+                    if (named_bar_or(1 + wq, 64, !ok)) {
+                        ok = false;
+                        break;
+                    }
+                } else if (!ok)
+                    break;
                 if (half == 0) {
                     uint32_t *tc1 = tc + kTierSlots * 128;   // the partner's counters
-                    int total = n_valid;
-                    if (kH == 2) total += (int)tc1[15 * 128];
+                    int total = n_valid, pads = n_pad;
+                    if (kH == 2) total += (int)(tc1[15 * 128] & 0xFFFFFFu), pads += (int)(tc1[15 * 128] >> 24);
                     bool good = false;
                     if (row < t.cnt) {
                         const int id = p.sl.ids[t.pos0 + row];
@@ -395,6 +451,7 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
                         int cnt_t = (int)tc[tt * 128] + (kH == 2 ? (int)tc1[tt * 128] : 0);
                         tc[tt * 128] = 0u;
                         if (kH == 2) tc1[tt * 128] = 0u;
+                        if (tt == (p.n_tiers >> 1)) cnt_t -= pads;        // columns beyond the sequence scored 0: matches = d' / 2
                         if (tt == p.n_tiers - 1) cnt_t = total - below;   // the closed last tier takes matches = d' as well
                         below += cnt_t;
                         const float v = (good && tt < p.n_tiers) ? (float)cnt_t * nrm : 0.f;
@@ -413,6 +470,7 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
                     }
                 }
             }
+            if (!ok) break;
             if (!kSplit) {
                 if (!mbar_wait(smem_u32(o_final), (uint32_t)(k & 1), abort_flag)) {
                     ok = false;
@@ -451,7 +509,7 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
             bool ok = true;
             if (warp == C::kMmaWarp) {
                 // scores of block gb (2 matches - d') into buffer gb & 1
-                const uint64_t qdesc0 = umma_desc_sw128(smem_u32(smQ)), gdesc0 = umma_desc_sw128(smem_u32(smKV + C::kVBytes));
+                const uint64_t qdesc0 = umma_desc_sw128(smem_u32(smQ)), gdesc0 = umma_desc_sw128(smem_u32(smG));
                 while (ok && c.tile < n_tiles) {
                     const int qb = c.k % kQB;
                     if (c.j == 0) {
@@ -459,42 +517,43 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
                                       : mbar_wait(smem_u32(q_full + qb), (uint32_t)(((c.k - 1) / kQB) & 1), abort_flag);
                         if (!ok) break;
                     }
-                    const int s = (int)(c.gb % kS);
-                    if (!mbar_wait(smem_u32(kv_full + s), (c.gb / kS) & 1u, abort_flag)) break;
-                    // the buffer's previous content, the counts of block gb - 2, must have been consumed by its product
-                    if (c.gb >= 2 && !mbar_wait(smem_u32(pv_done + (c.gb & 1u)), ((c.gb - 2) >> 1) & 1u, abort_flag)) break;
+                    const int s = (int)(c.gb % kSG);
+                    if (!mbar_wait(smem_u32(g_full + s), (c.gb / kSG) & 1u, abort_flag)) break;
+                    // the buffer's previous content, the scores of block gb - 2, must have been read
+                    if (c.gb >= 2 && !mbar_wait(smem_u32(s_free + (c.gb & 1u)), ((c.gb - 2) >> 1) & 1u, abort_flag)) break;
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + (uint32_t)((c.gb & 1u) * BN);
                     const uint64_t qd = qdesc0 + (uint64_t)(uint32_t)(qb * (C::kQBytes >> 4));
-                    const uint64_t gd = gdesc0 + (uint64_t)(uint32_t)(s * (C::kStageBytes >> 4));
+                    const uint64_t gd = gdesc0 + (uint64_t)(uint32_t)(s * (C::kGBytes >> 4));
 #pragma unroll
                     for (int kk = 0; kk < D / 32; ++kk)   // K = 32 signature bits per instruction, 32 bytes of a chunk row
                         umma_e4m3(d_tmem, qd + (uint64_t)((kk >> 2) * (16384 >> 4) + 2 * (kk & 3)),
                                   gd + (uint64_t)((kk >> 2) * (C::kGChunkBytes >> 4) + 2 * (kk & 3)), idesc_sig, kk > 0 ? 1u : 0u);
                     umma_commit(smem_u32(s_full + (c.gb & 1u)));
+                    umma_commit(smem_u32(g_empty + s));
                     if (c.j == c.nb - 1) umma_commit(smem_u32(q_empty + qb));
                     advance(c);
                 }
             } else {
                 // O += P S of block gb as soon as its counts are in tensor memory
-                const uint64_t vdesc0 = umma_desc_mn_sw128(smem_u32(smKV), C::kVChunkBytes);
+                const uint64_t vdesc0 = umma_desc_mn_sw128(smem_u32(smV), C::kVChunkBytes);
                 while (ok && c.tile < n_tiles) {
+                    const int s = (int)(c.gb % kSV);
+                    if (!mbar_wait(smem_u32(v_full + s), (c.gb / kSV) & 1u, abort_flag)) break;
                     if (!mbar_wait(smem_u32(p_full + (c.gb & 1u)), (c.gb >> 1) & 1u, abort_flag)) break;
-                    if (c.j == 0 && (kSplit ? c.k >= 2 && !mbar_wait(smem_u32(o_free + (c.k & 1)), (uint32_t)(((c.k - 2) >> 1) & 1), abort_flag)
-                                            : c.k > 0 && !mbar_wait(smem_u32(o_free), (uint32_t)((c.k - 1) & 1), abort_flag)))
-                        break;
+                    // the first product of a tile overwrites O: the previous tile's rows must have been read
+                    if (c.j == 0 && c.k > 0 && !mbar_wait(smem_u32(o_free), (uint32_t)((c.k - 1) & 1), abort_flag)) break;
                     tc_fence_after();
-                    const int s = (int)(c.gb % kS);
-                    const uint32_t o_tmem = tmem_base + (uint32_t)(C::kTmemO + (kSplit ? (c.k & 1) * D : 0));
-                    const uint32_t p_tmem = tmem_base + (uint32_t)((c.gb & 1u) * BN);
-                    const uint64_t vd = vdesc0 + (uint64_t)(uint32_t)(s * (C::kStageBytes >> 4));
+                    const uint32_t o_tmem = tmem_base + (uint32_t)C::kTmemO;
+                    const uint32_t p_tmem = tmem_base + (uint32_t)(C::kTmemP + (c.gb & 1u) * (BN / 2));
+                    const uint64_t vd = vdesc0 + (uint64_t)(uint32_t)(s * (C::kVBytes >> 4));
 #pragma unroll
                     for (int kk = 0; kk < BN / 16; ++kk)
                         umma_bf16_ts(o_tmem, p_tmem + (uint32_t)(kk * 8), vd + (uint64_t)(kk * (2048 >> 4)), idesc_pv,
                                      (c.j > 0 || kk > 0) ? 1u : 0u);
                     umma_commit(smem_u32(pv_done + (c.gb & 1u)));
-                    umma_commit(smem_u32(kv_empty + s));
-                    if (c.j == c.nb - 1) umma_commit(smem_u32(o_final + (kSplit ? (c.k & 1) : 0)));
+                    umma_commit(smem_u32(v_empty + s));
+                    if (c.j == c.nb - 1) umma_commit(smem_u32(o_final));
                     advance(c);
                 }
             }
@@ -503,25 +562,49 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
     } else if (warp == C::kTmaWarp) {
         // ===================== key blocks: rows of S and +-1 signatures (TMA) =====================
         if (lane == 0) {
-            uint32_t gb = 0;
+            // two cursors over the same sequence of key blocks: the signature stream runs up to three blocks ahead of the
+            // stream of S rows, which is held back by the products that still read its stages
+            struct Stream {
+                int tile, j, nb, slot;
+                uint32_t gb;
+            };
+            auto open = [&](Stream &c) {
+                if (c.tile < n_tiles) {
+                    const LshTile t = lsh_tile<BN>(p, c.tile);
+                    c.nb = t.nb, c.slot = t.slot;
+                }
+            };
+            auto step = [&](Stream &c) {
+                ++c.gb;
+                if (++c.j == c.nb) {
+                    c.j = 0, c.tile += gridDim.x;
+                    open(c);
+                }
+            };
+            Stream g{(int)blockIdx.x, 0, 0, 0, 0u}, v{(int)blockIdx.x, 0, 0, 0, 0u};
+            open(g), open(v);
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
-                const LshTile t = lsh_tile<BN>(p, tile);
-                for (int j = 0; j < t.nb; ++j, ++gb) {
-                    const int s = (int)(gb % kS);
-                    if (!mbar_wait(smem_u32(kv_empty + s), ((gb / kS) & 1u) ^ 1u, abort_flag)) {
+            while (ok && v.tile < n_tiles) {
+                while (ok && g.tile < n_tiles && g.gb < v.gb + (uint32_t)(kSG - 1)) {
+                    const int s = (int)(g.gb % kSG);
+                    if (!mbar_wait(smem_u32(g_empty + s), ((g.gb / kSG) & 1u) ^ 1u, abort_flag)) {
                         ok = false;
                         break;
                     }
-                    mbar_expect_tx(smem_u32(kv_full + s), (uint32_t)C::kStageBytes);
-                    unsigned char *st = smKV + s * C::kStageBytes;
+                    mbar_expect_tx(smem_u32(g_full + s), (uint32_t)C::kGBytes);
 #pragma unroll
                     for (int c = 0; c < C::kQChunks; ++c)
-                        tma_load_3d(smem_u32(st + C::kVBytes + c * C::kGChunkBytes), &tmapG, smem_u32(kv_full + s), c * 128, j * BN, t.slot);
-#pragma unroll
-                    for (int c = 0; c < C::kVChunks; ++c)
-                        tma_load_3d(smem_u32(st + c * C::kVChunkBytes), &tmapS, smem_u32(kv_full + s), c * 64, j * BN, t.slot);
+                        tma_load_3d(smem_u32(smG + s * C::kGBytes + c * C::kGChunkBytes), &tmapG, smem_u32(g_full + s), c * 128, g.j * BN, g.slot);
+                    step(g);
                 }
+                if (!ok) break;
+                const int s = (int)(v.gb % kSV);
+                if (!mbar_wait(smem_u32(v_empty + s), ((v.gb / kSV) & 1u) ^ 1u, abort_flag)) break;
+                mbar_expect_tx(smem_u32(v_full + s), (uint32_t)C::kVBytes);
+#pragma unroll
+                for (int c = 0; c < C::kVChunks; ++c)
+                    tma_load_3d(smem_u32(smV + s * C::kVBytes + c * C::kVChunkBytes), &tmapS, smem_u32(v_full + s), c * 64, v.j * BN, v.slot);
+                step(v);
             }
         }
         __syncwarp();
@@ -531,8 +614,7 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
         int k = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++k) {
             const LshTile t = lsh_tile<BN>(p, tile);
-            const int b = k & 1;
-            if (!mbar_wait(smem_u32(o_final + b), (uint32_t)((k >> 1) & 1), abort_flag)) break;
+            if (!mbar_wait(smem_u32(o_final), (uint32_t)(k & 1), abort_flag)) break;
             tc_fence_after();
             tile_epilogue(k, t, wq, lane);
         }
@@ -646,7 +728,13 @@ cudaError_t launch_expand_signatures(const aif_ctx *ctx, const uint8_t *sig, int
     const int grid = (int)((total + 255) / 256 < 592 ? (total + 255) / 256 : 592);
     k_expand_signatures<<<grid, 256, 0, st>>>(sig, L, ctx->cfg.lsh_bits, out);
     count_launch();
-    return cudaGetLastError();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    // zero bytes from the sequence's end to the end of its last 128-key block: the kernel relies on a score of exactly 0
+    // for the columns beyond the sequence (rows beyond L_max are zero-filled by the tensor map)
+    const int L_pad = (L + 127) / 128 * 128 < ctx->cfg.L_max ? (L + 127) / 128 * 128 : ctx->cfg.L_max;
+    if (L_pad > L) e = cudaMemsetAsync(out + (size_t)L * ctx->cfg.lsh_bits, 0, (size_t)(L_pad - L) * ctx->cfg.lsh_bits, st);
+    return e;
 }
 
 // LSH-DIN rows into columns [x_din, x_din + d) and SimTier rows into [x_tier, x_tier + 64) of X; a negative column turns
@@ -671,13 +759,6 @@ cudaError_t launch_lsh_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
     p.x_stride = x_stride, p.x_din = x_din, p.x_tier = x_tier, p.X = (__nv_bfloat16 *)X;
     p.n_tiers = (c.blocks & AIF_BLK_SIMTIER) ? c.n_tiers : 1;
     p.din_mean = c.lsh_din_norm == AIF_NORM_MEAN, p.tier_mean = c.simtier_norm == AIF_NORM_MEAN;
-    // Tier of a pair from q = 2 matches (an integer in [0, 2 d']): floor(q N / (2 d')) as (q N m) >> 24 with
-    // m = floor(2^24 / (2 d')) + 1, exact while q N (m 2 d' - 2^24) < 2^24, i.e. for every q N <= 8192 and d' <= 256.  The
-    // kernel has q in the low mantissa bits of the float score + d' + 2^23, whose bit pattern is 0x4B000000 + q: the
-    // constant part is taken out by the addend (arithmetic modulo 2^32).
-    const uint32_t m = (1u << 24) / (uint32_t)(2 * c.lsh_bits) + 1u;
-    p.tier_mul = (uint32_t)p.n_tiers * m;
-    p.tier_add = 0u - 0x4B000000u * p.tier_mul;
     const int grid = sl.n_tiles > 148 ? 148 : sl.n_tiles;
     cudaError_t e;
     if (c.d == 128)

@@ -113,8 +113,10 @@ C5_MIXED = C5.with_(name="c5_wide_mixed", N=10_000, mixed_sizes=(1000, 10_000))
 # the long-sequence shape with the LSH blocks (eqs. 6-9) in place of, and beside, the dense target attention
 C4_LSH = C4.with_(name="c4_long_sequence_lsh", blocks=BLK_CROSS | BLK_LSH_DIN | BLK_SIMTIER)
 C4_BOTH = C4.with_(name="c4_long_sequence_att_lsh", blocks=BLK_ATT | BLK_CROSS | BLK_LSH_DIN | BLK_SIMTIER)
-CONFIGS = {w.name: w for w in (C1, C2, C3, C4, C5, C5_MIXED, C4_LSH, C4_BOTH)}
-SHORT = {"c1": C1, "c2": C2, "c3": C3, "c4": C4, "c5": C5, "c5a": C5, "c5b": C5_MIXED, "c4_lsh": C4_LSH, "c4_both": C4_BOTH}
+C4_DIN = C4.with_(name="c4_long_sequence_lsh_din", blocks=BLK_CROSS | BLK_LSH_DIN)
+CONFIGS = {w.name: w for w in (C1, C2, C3, C4, C5, C5_MIXED, C4_LSH, C4_BOTH, C4_DIN)}
+SHORT = {"c1": C1, "c2": C2, "c3": C3, "c4": C4, "c5": C5, "c5a": C5, "c5b": C5_MIXED, "c4_lsh": C4_LSH, "c4_both": C4_BOTH,
+         "c4_din": C4_DIN}
 
 
 def _seed(*keys) -> np.random.Generator:

@@ -467,3 +467,34 @@ def test_score_host_with_pinned_and_with_pageable_buffers():
         assert np.array_equal(h_out.numpy(), ref)
     assert srv.ctx.poll_status() == 0
     srv.close()
+
+
+def test_score_batch_host_gives_the_device_buffer_result():
+    """aif_score_batch_host (host ids in, host logits out, several requests in one launch) equals aif_score_batch on
+    device buffers bit for bit, with page-locked and with pageable buffers, and matches the oracle."""
+    wl = helpers.MINI["c3"].with_(name="hostbatch", R=3, N=333)
+    weights, table, srv, oracle = _setup(wl)
+    sampler = synth.IdSampler(wl)
+    states, id_lists, wants = [], [], []
+    for r in range(wl.R):
+        rq = synth.make_request(wl, r)
+        states.append(srv.precompute(r, srv.upload_request(rq, B.USER_PROJECTED)))
+        id_lists.append(sampler.request_ids(r, 333 - 100 * r))
+        wants.append(oracle.score(table, helpers.projected_request(wl, rq), id_lists[-1]))
+    ref = np.concatenate(srv.score_many(states, id_lists))
+    offs = np.zeros(wl.R + 1, dtype=np.int64)
+    offs[1:] = np.cumsum([len(x) for x in id_lists])
+    for pinned in (True, False):
+        h_ids = torch.from_numpy(np.concatenate(id_lists))
+        h_out = torch.full((int(offs[-1]),), float("nan"), dtype=torch.float32)
+        if pinned:
+            h_ids, h_out = h_ids.pin_memory(), h_out.pin_memory()
+        srv.ctx.score_batch_host(states, h_ids, offs, h_out)
+        assert np.array_equal(h_out.numpy(), ref)
+    _check_logits(ref, np.concatenate(wants), TOL["bf16"])
+    with pytest.raises(B.AifError) as e:     # more candidates than the context was sized for
+        big = torch.zeros(wl.R * wl.N + 1, dtype=torch.int32)
+        srv.ctx.score_batch_host(states[:1], big, [0, len(big)], torch.zeros(len(big)))
+    assert e.value.code == B.ERR_SHAPE
+    assert srv.ctx.poll_status() == 0
+    srv.close()
