@@ -49,6 +49,8 @@ typedef struct {
     int32_t lsh_din_norm; /* ORC_NORM_NONE: eq. 8 as printed (a sum); ORC_NORM_MEAN: divided by l */
     int32_t simtier_norm; /* ORC_NORM_NONE: raw counts (eq. 9); ORC_NORM_MEAN: counts divided by l */
     int32_t emit_sigmoid;
+    int32_t n_categories; /* 0: the interaction blocks see the whole sequence; > 0: only the sub-sequence of the
+                             candidate's category (Section 3.3, SIM-hard) */
 } orc_cfg;
 
 typedef struct {
@@ -105,6 +107,12 @@ int64_t orc_bucket(int64_t id, int field, int B, int mode)
     if (mode == ORC_BUCKET_MOD) return id % B;
     return (int64_t)(orc_mix64((uint64_t)id, (uint64_t)field) % (uint64_t)B);
 }
+
+/* Category of an item (Section 3.3: SIM-hard selects sub-sequences "based on the candidate items' category").
+ * Reading: like the cross-feature attribute, the category is derived from the id, with the bucket function applied
+ * to a field number of its own. */
+enum { ORC_CATEGORY_FIELD = 3239 };
+int64_t orc_category(int64_t id, int n_categories, int mode) { return orc_bucket(id, ORC_CATEGORY_FIELD, n_categories, mode); }
 
 /* ---------------------------------------------------------------------------------------------
  * LSH signatures (Section 4.2).
@@ -415,6 +423,8 @@ typedef struct {
     const void *T;          /* [F x B x dc] user-side part of the cross features, or NULL */
     const void *V;          /* [n x d] user-side BEA vectors (Algorithm 1 line 2), or NULL */
     const uint8_t *sig_seq; /* [l x d'/8] signatures of the sequence items, or NULL */
+    const int32_t *seq_cat; /* [l] category of every sequence item (the parsed <user, category, sub_sequence> form of
+                               Section 3.3), or NULL when n_categories = 0 */
 } orc_request;
 
 void orc_build_input(const orc_cfg *cfg, const orc_request *rq, int64_t id, double *x)
@@ -424,8 +434,32 @@ void orc_build_input(const orc_cfg *cfg, const orc_request *rq, int64_t id, doub
     for (int c = 0; c < d; ++c) x[o++] = rq->u[c];
     double *e = x + o;
     for (int c = 0; c < d; ++c) x[o++] = ld(rq->E, id * d + c, dt);
+    /* Section 3.3 (SIM-hard): with categories on, the sequence the interaction blocks see is the sub-sequence of the
+     * user's behaviours whose category is the candidate's, in their original order.  Reading for an empty sub-sequence
+     * (the paper is silent): attention output, LSH-DIN output and tier counts are all zero. */
+    const double *S = rq->S;
+    const uint8_t *sig_seq = rq->sig_seq;
+    int l = rq->l;
+    double *S_sub = NULL;
+    uint8_t *sig_sub = NULL;
+    if (cfg->n_categories > 0) {
+        const int64_t cat = orc_category(id, cfg->n_categories, cfg->bucket_mode);
+        const int nbytes = cfg->lsh_bits / 8;
+        S_sub = (double *)malloc(sizeof(double) * (size_t)(rq->l > 0 ? rq->l : 1) * (size_t)d);
+        if (rq->sig_seq) sig_sub = (uint8_t *)malloc((size_t)(rq->l > 0 ? rq->l : 1) * (size_t)(nbytes > 0 ? nbytes : 1));
+        l = 0;
+        for (int j = 0; j < rq->l; ++j)
+            if (rq->seq_cat[j] == cat) {
+                memcpy(S_sub + (int64_t)l * d, rq->S + (int64_t)j * d, sizeof(double) * (size_t)d);
+                if (sig_sub) memcpy(sig_sub + (int64_t)l * nbytes, rq->sig_seq + (int64_t)j * nbytes, (size_t)nbytes);
+                l += 1;
+            }
+        S = S_sub, sig_seq = sig_sub;
+    }
     if (cfg->blocks & ORC_BLK_ATT) {
-        orc_attention(e, rq->S, rq->l, d, x + o);
+        if (l > 0) orc_attention(e, S, l, d, x + o);
+        else
+            for (int c = 0; c < d; ++c) x[o + c] = 0.0;
         o += d;
     }
     if (cfg->blocks & ORC_BLK_CROSS) {
@@ -445,24 +479,30 @@ void orc_build_input(const orc_cfg *cfg, const orc_request *rq, int64_t id, doub
         free(wh);
     }
     if (cfg->blocks & (ORC_BLK_LSH_DIN | ORC_BLK_SIMTIER)) {
-        int nbytes = cfg->lsh_bits / 8, l = rq->l;
-        int *matches = (int *)malloc(sizeof(int) * (size_t)l);
-        double *sim = (double *)malloc(sizeof(double) * (size_t)l);
+        int nbytes = cfg->lsh_bits / 8;
+        int *matches = (int *)malloc(sizeof(int) * (size_t)(l > 0 ? l : 1));
+        double *sim = (double *)malloc(sizeof(double) * (size_t)(l > 0 ? l : 1));
         for (int j = 0; j < l; ++j) {
-            matches[j] = orc_lsh_matches(rq->sig + id * nbytes, rq->sig_seq + (int64_t)j * nbytes, nbytes, 1);
+            matches[j] = orc_lsh_matches(rq->sig + id * nbytes, sig_seq + (int64_t)j * nbytes, nbytes, 1);
             sim[j] = (double)matches[j] / (double)cfg->lsh_bits;
         }
         if (cfg->blocks & ORC_BLK_LSH_DIN) {
-            orc_lsh_din(sim, rq->S, l, d, cfg->lsh_din_norm, x + o);
+            if (l > 0) orc_lsh_din(sim, S, l, d, cfg->lsh_din_norm, x + o);
+            else
+                for (int c = 0; c < d; ++c) x[o + c] = 0.0;
             o += d;
         }
         if (cfg->blocks & ORC_BLK_SIMTIER) {
-            orc_simtier(matches, l, cfg->lsh_bits, cfg->n_tiers, cfg->simtier_norm, x + o);
+            if (l > 0) orc_simtier(matches, l, cfg->lsh_bits, cfg->n_tiers, cfg->simtier_norm, x + o);
+            else
+                for (int t = 0; t < cfg->n_tiers; ++t) x[o + t] = 0.0;
             o += cfg->n_tiers;
         }
         free(matches);
         free(sim);
     }
+    free(S_sub);
+    free(sig_sub);
 }
 
 /* The shallow scoring MLP on the full concatenated input (Section 1): ReLU hidden layers, linear

@@ -32,6 +32,8 @@ def lib():
         _lib.orc_mix64.argtypes = [C.c_uint64, C.c_uint64]
         _lib.orc_bucket.restype = C.c_int64
         _lib.orc_bucket.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
+        _lib.orc_category.restype = C.c_int64
+        _lib.orc_category.argtypes = [C.c_int64, C.c_int, C.c_int]
         _lib.orc_mlp.restype = C.c_double
         _lib.orc_num_threads.restype = C.c_int
     return _lib
@@ -42,7 +44,7 @@ class _Cfg(C.Structure):
         ("dtype", C.c_int32), ("M", C.c_int64), ("d", C.c_int32), ("F", C.c_int32), ("B", C.c_int32),
         ("dc", C.c_int32), ("n_hidden", C.c_int32), ("hidden", C.c_int32 * 4), ("bucket_mode", C.c_int32),
         ("blocks", C.c_int32), ("n_bridge", C.c_int32), ("lsh_bits", C.c_int32), ("n_tiers", C.c_int32),
-        ("lsh_din_norm", C.c_int32), ("simtier_norm", C.c_int32), ("emit_sigmoid", C.c_int32),
+        ("lsh_din_norm", C.c_int32), ("simtier_norm", C.c_int32), ("emit_sigmoid", C.c_int32), ("n_categories", C.c_int32),
     ]
 
 
@@ -58,7 +60,7 @@ class _UserW(C.Structure):
 class _Req(C.Structure):
     _fields_ = [("E", C.c_void_p), ("bea_w", C.c_void_p), ("sig", C.c_void_p), ("u", C.c_void_p),
                 ("S", C.c_void_p), ("l", C.c_int32), ("T", C.c_void_p), ("V", C.c_void_p),
-                ("sig_seq", C.c_void_p)]
+                ("sig_seq", C.c_void_p), ("seq_cat", C.c_void_p)]
 
 
 @dataclasses.dataclass
@@ -78,12 +80,13 @@ class OracleConfig:
     lsh_din_norm: int = NORM_NONE
     simtier_norm: int = NORM_NONE
     emit_sigmoid: int = 0
+    n_categories: int = 0
 
     def c(self) -> _Cfg:
         h = list(self.hidden) + [0] * (4 - len(self.hidden))
         return _Cfg(self.dtype, self.M, self.d, self.F, self.B, self.dc, len(self.hidden), (C.c_int32 * 4)(*h),
                     self.bucket_mode, self.blocks, self.n_bridge, self.lsh_bits, self.n_tiers,
-                    self.lsh_din_norm, self.simtier_norm, self.emit_sigmoid)
+                    self.lsh_din_norm, self.simtier_norm, self.emit_sigmoid, self.n_categories)
 
     def input_width(self) -> int:
         cfg = self.c()
@@ -124,6 +127,13 @@ def mix64(id_: int, field: int) -> int:
 
 def bucket(id_: int, field: int, B: int, mode: int) -> int:
     return int(lib().orc_bucket(id_, field, B, mode))
+
+
+def category(id_: int, n_categories: int, mode: int) -> int:
+    return int(lib().orc_category(id_, n_categories, mode))
+
+
+CATEGORY_FIELD = 3239
 
 
 def pack_bits(bits: np.ndarray) -> np.ndarray:
@@ -328,7 +338,8 @@ class Oracle:
                                 ("sig", table, lambda a: np.ascontiguousarray(a, dtype=np.uint8)),
                                 ("T", request, lambda a: _store(a, dt)),
                                 ("V", request, lambda a: _store(a, dt)),
-                                ("sig_seq", request, lambda a: np.ascontiguousarray(a, dtype=np.uint8))):
+                                ("sig_seq", request, lambda a: np.ascontiguousarray(a, dtype=np.uint8)),
+                                ("seq_cat", request, lambda a: np.ascontiguousarray(a, dtype=np.int32))):
             a = src.get(name)
             if a is not None:
                 a = conv(a)
@@ -343,9 +354,12 @@ class Oracle:
         """Logits (or probabilities when emit_sigmoid) of the candidates `ids` of one request.
 
         table: E [M x d] (+ bea_w [M x n], sig [M x d'/8]); request: u [d], S [l x d] (float64, or any
-        array convertible to it exactly), T [F x B x dc], V [n x d], sig_seq [l x d'/8]."""
+        array convertible to it exactly), T [F x B x dc], V [n x d], sig_seq [l x d'/8], seq_cat [l] (int32, needed
+        when the configuration has categories)."""
         cfg = self.cfg.c()
         rq, keep = self._request(table, request)
+        if self.cfg.n_categories > 0:
+            assert request.get("seq_cat") is not None and len(request["seq_cat"]) == rq.l
         ids = np.ascontiguousarray(ids, dtype=np.int32)
         out = np.zeros(ids.size)
         x = np.zeros((ids.size, self.cfg.input_width())) if return_inputs else None

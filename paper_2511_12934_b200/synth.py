@@ -70,6 +70,7 @@ class Workload:
     emit_sigmoid: int = 0
     dU: int = 0                     # width of the raw user embeddings (0: same as d)
     n_cross_tables: int = 0         # distinct cross tables generated and cycled over requests (0: one per request)
+    n_categories: int = 0           # item categories; > 0: the interaction blocks see the candidate's category's sub-sequence
 
     @property
     def raw_dU(self) -> int:
@@ -292,7 +293,8 @@ def make_request(wl: Workload, r: int, L: Optional[int] = None) -> dict:
 
     "profile" [dU] and "seq" [L x dU] are the raw embeddings for the user-side network; "u" [d] and "S"
     [L x d] are a combined user vector and a projected sequence for callers that supply them directly.
-    "T" [F x B x dc], "V" [n x d], "sig_seq" [L x d'/8] as enabled."""
+    "T" [F x B x dc], "V" [n x d], "sig_seq" [L x d'/8] as enabled; "seq_cat" [L] the category of every sequence item
+    when the workload has categories."""
     t = _tag(wl.name)
     L = L or wl.L
     dU = wl.raw_dU
@@ -309,4 +311,9 @@ def make_request(wl: Workload, r: int, L: Optional[int] = None) -> dict:
         rq["V"] = normal_rows(wl.n_bridge, wl.d, wl.sigma, wl.dtype, t, 25, r)
     if wl.blocks & (BLK_LSH_DIN | BLK_SIMTIER):
         rq["sig_seq"] = _signatures(L, wl.lsh_bits // 8, t, 26, r, protos=signature_prototypes(wl))
+    if wl.n_categories > 0:
+        # a user's behaviours are skewed towards a few categories: weights 1 / (rank + 1) over a per-request order
+        g = _seed(t, 27, r)
+        w = 1.0 / (1.0 + g.permutation(wl.n_categories))
+        rq["seq_cat"] = g.choice(wl.n_categories, size=L, p=w / w.sum()).astype(np.int32)
     return rq

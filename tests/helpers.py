@@ -10,7 +10,7 @@ def oracle_config(wl: synth.Workload, M=None) -> orc.OracleConfig:
         dtype=orc.F32 if wl.dtype == "f32" else orc.BF16, M=M or wl.M, d=wl.d, F=wl.F, B=wl.B, dc=wl.dc,
         hidden=tuple(wl.hidden), bucket_mode=wl.bucket_mode, blocks=wl.blocks, n_bridge=wl.n_bridge,
         lsh_bits=wl.lsh_bits, n_tiers=wl.n_tiers, lsh_din_norm=wl.lsh_din_norm, simtier_norm=wl.simtier_norm,
-        emit_sigmoid=wl.emit_sigmoid)
+        emit_sigmoid=wl.emit_sigmoid, n_categories=wl.n_categories)
 
 
 def make_oracle(wl: synth.Workload, weights: dict, M=None) -> orc.Oracle:
@@ -21,7 +21,7 @@ def projected_request(wl: synth.Workload, rq: dict) -> dict:
     """Request dict for Oracle.score when the caller supplies u and S directly."""
     out = {"u": synth.as_f32(rq["u"], wl.dtype).astype(np.float64),
            "S": synth.as_f32(rq["S"], wl.dtype).astype(np.float64)}
-    for k in ("T", "V", "sig_seq"):
+    for k in ("T", "V", "sig_seq", "seq_cat"):
         if k in rq:
             out[k] = rq[k]
     return out
@@ -31,7 +31,7 @@ def raw_request(oracle: orc.Oracle, rq: dict) -> dict:
     """Request dict for Oracle.score with u and S computed by the oracle's user-side network (eqs. 1-3)."""
     u, S = oracle.user_state(rq["profile"], rq["seq"])
     out = {"u": u, "S": S}
-    for k in ("T", "V", "sig_seq"):
+    for k in ("T", "V", "sig_seq", "seq_cat"):
         if k in rq:
             out[k] = rq[k]
     return out

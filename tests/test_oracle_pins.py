@@ -620,3 +620,103 @@ def test_bea_user_side_and_the_whole_of_algorithm_1():
     V0, _ = orc.bea_user(orc.F32, Bm[:1], U, Wf)
     w0 = orc.item_nearline(orc.F32, I_id=I, bridges=Bm[:1])["w_hat"]
     assert np.array_equal(w0, np.ones((b, 1))) and np.allclose(orc.bea(w0[3], V0), V0[0], atol=0)
+
+
+# ------------------------------------------------------------------------------------------------
+# Category sub-sequences (Section 3.3, SIM-hard): the interaction blocks restricted to the behaviours whose category is
+# the candidate's
+# ------------------------------------------------------------------------------------------------
+def _sim_setup(n_categories, L=40, N=60, blocks=helpers.ALL_BLOCKS, seed=0, dtype="f32"):
+    base = synth.C1 if dtype == "f32" else synth.C2
+    wl = base.with_(name=f"sim_pin_{n_categories}_{seed}", N=N, M=500, L=L, blocks=blocks, n_categories=n_categories,
+                    lsh_din_norm=synth.NORM_MEAN, simtier_norm=synth.NORM_MEAN, emit_sigmoid=0, hidden=(32, 16), F=2, B=8, dc=8)
+    weights = synth.make_weights(wl, zero_bias=False)
+    table = synth.make_item_table(wl)
+    rq = synth.make_request(wl, seed)
+    ids = synth.IdSampler(wl).request_ids(seed)
+    return wl, weights, table, rq, ids
+
+
+def test_category_is_the_bucket_function_on_its_own_field():
+    for i in (0, 1, 17, 4242, 2**31 - 1):
+        for C_ in (1, 7, 100):
+            assert orc.category(i, C_, orc.BUCKET_MOD) == i % C_
+            assert orc.category(i, C_, orc.BUCKET_HASH) == orc.mix64(i, orc.CATEGORY_FIELD) % C_
+            assert orc.category(i, C_, orc.BUCKET_HASH) == orc.bucket(i, orc.CATEGORY_FIELD, C_, orc.BUCKET_HASH)
+
+
+def test_one_category_is_the_whole_sequence():
+    wl, weights, table, rq, ids = _sim_setup(1)
+    assert (rq["seq_cat"] == 0).all()
+    with_cat = helpers.make_oracle(wl, weights).score(table, helpers.projected_request(wl, rq), ids)
+    plain_wl = wl.with_(n_categories=0)
+    plain = helpers.make_oracle(plain_wl, weights).score(table, helpers.projected_request(plain_wl, rq), ids)
+    assert np.array_equal(with_cat, plain)
+
+
+def test_every_behaviour_in_the_candidates_category_is_the_whole_sequence_and_none_is_all_zeros():
+    wl, weights, table, rq, ids = _sim_setup(5)
+    oracle = helpers.make_oracle(wl, weights)
+    plain_wl = wl.with_(n_categories=0)
+    plain, xp = helpers.make_oracle(plain_wl, weights).score(table, helpers.projected_request(plain_wl, rq), ids, return_inputs=True)
+    d = wl.d
+    for i in (0, 7, 31):
+        cat = orc.category(int(ids[i]), 5, wl.bucket_mode)
+        rq_all = dict(rq, seq_cat=np.full(wl.L, cat, dtype=np.int32))
+        got, x = oracle.score(table, helpers.projected_request(wl, rq_all), ids[i:i + 1], return_inputs=True)
+        assert got[0] == plain[i] and np.array_equal(x[0], xp[i])
+        rq_none = dict(rq, seq_cat=np.full(wl.L, (cat + 1) % 5, dtype=np.int32))
+        _, x0 = oracle.score(table, helpers.projected_request(wl, rq_none), ids[i:i + 1], return_inputs=True)
+        assert np.all(x0[0, 2 * d:3 * d] == 0.0)                       # attention
+        tail = x0[0, 3 * d + wl.F * wl.dc + d:]                        # [lsh_din | simtier] after cross and v_bea
+        assert tail.shape[0] == d + wl.n_tiers and np.all(tail == 0.0)
+        assert np.array_equal(x0[0, :2 * d], xp[i, :2 * d])            # u and e do not depend on the sequence
+
+
+def test_a_sub_sequence_of_one_item_gives_that_item():
+    wl, weights, table, rq, ids = _sim_setup(3)
+    oracle = helpers.make_oracle(wl, weights)
+    i = 4
+    cat = orc.category(int(ids[i]), 3, wl.bucket_mode)
+    seq_cat = np.full(wl.L, (cat + 1) % 3, dtype=np.int32)
+    seq_cat[11] = cat
+    _, x = oracle.score(table, helpers.projected_request(wl, dict(rq, seq_cat=seq_cat)), ids[i:i + 1], return_inputs=True)
+    d = wl.d
+    S = synth.as_f32(rq["S"], wl.dtype).astype(np.float64)
+    assert np.allclose(x[0, 2 * d:3 * d], S[11], rtol=0, atol=1e-15)   # softmax over one key is 1
+    k = orc.lsh_matches(table["sig"][ids[i]], rq["sig_seq"][11])
+    off = 3 * d + wl.F * wl.dc + d
+    assert np.allclose(x[0, off:off + d], (k / wl.lsh_bits) * S[11], rtol=0, atol=1e-15)   # mean over one item
+    tiers = x[0, off + d:]
+    assert tiers.sum() == 1.0 and tiers[orc.tier_of(k, wl.lsh_bits, wl.n_tiers)] == 1.0
+
+
+def test_sub_sequences_against_explicit_selection_and_under_a_permutation_of_the_sequence():
+    wl, weights, table, rq, ids = _sim_setup(4, L=57, seed=2)
+    oracle = helpers.make_oracle(wl, weights)
+    req = helpers.projected_request(wl, rq)
+    want, x = oracle.score(table, req, ids, return_inputs=True)
+    S = req["S"]
+    d = wl.d
+    E = synth.as_f32(table["E"], wl.dtype).astype(np.float64)
+    for i in range(0, len(ids), 9):
+        cat = int(ids[i]) % 4 if wl.bucket_mode == synth.BUCKET_MOD else orc.mix64(int(ids[i]), orc.CATEGORY_FIELD) % 4
+        sel = np.flatnonzero(rq["seq_cat"] == cat)
+        if len(sel) == 0:
+            assert np.all(x[i, 2 * d:3 * d] == 0.0)
+            continue
+        # plain numpy: softmax(e S_c^T / sqrt(d)) S_c over the selected rows
+        s = S[sel] @ E[ids[i]] / math.sqrt(d)
+        a = np.exp(s - s.max())
+        a /= a.sum()
+        assert np.allclose(x[i, 2 * d:3 * d], a @ S[sel], rtol=0, atol=1e-14)
+        k = np.array([orc.lsh_matches(table["sig"][ids[i]], rq["sig_seq"][j]) for j in sel])
+        off = 3 * d + wl.F * wl.dc + d
+        assert np.allclose(x[i, off:off + d], (k / wl.lsh_bits) @ S[sel] / len(sel), rtol=0, atol=1e-14)
+        hist = np.bincount([orc.tier_of(int(v), wl.lsh_bits, wl.n_tiers) for v in k], minlength=wl.n_tiers) / len(sel)
+        assert np.allclose(x[i, off + d:], hist, rtol=0, atol=1e-15)
+    # the order of the behaviours does not matter, as long as every row keeps its category and its signature
+    perm = np.random.default_rng(4).permutation(wl.L)
+    rq_p = dict(rq, S=rq["S"][perm], sig_seq=rq["sig_seq"][perm], seq_cat=rq["seq_cat"][perm])
+    got = oracle.score(table, helpers.projected_request(wl, rq_p), ids)
+    assert np.abs(got - want).max() < 1e-12
