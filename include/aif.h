@@ -103,6 +103,11 @@ typedef struct {
     int32_t path;                  /* AIF_PATH_AUTO: tensor-core kernels when dtype and shapes allow, else
                                       the CUDA-core kernels; _SIMT / _TENSOR force one (TENSOR: AIF_ERR_SHAPE
                                       if unsupported) */
+    int32_t n_categories;          /* 0: the sequence blocks (attention, LSH-DIN, SimTier) see the whole behaviour
+                                      sequence.  1..4096: they see only the sub-sequence of the candidate's category
+                                      (Section 3.3, SIM-hard: <user, category, sub-sequence>), see aif_category.  Needs
+                                      the tensor-core kernels (AIF_ERR_SHAPE otherwise); mini_batch is then ignored
+                                      (scores do not depend on it) */
     int64_t max_batch_candidates;  /* upper bound of the candidates of one aif_score / aif_score_batch call;
                                       sizes the context's scratch memory */
 } aif_config;
@@ -141,6 +146,9 @@ typedef struct {
                                 byte 0 (Section 4.2); NULL if both LSH blocks are off */
     const void *bea_U;       /* [bea_m x d] user-side feature embeddings U of Algorithm 1: with bea_V == NULL the call
                                 computes W = Softmax(B U^T / sqrt(d)) and V from them (needs bridges and W_f) */
+    const int32_t *seq_cat;  /* int32 [L]: category in [0, n_categories) of every sequence item, the parsed form of the
+                                long-term sequence (Section 3.3); required iff n_categories > 0.  An entry outside the
+                                range drops that item from every sub-sequence and sets AIF_STATUS_BAD_ID */
     int32_t bea_m;           /* 1 <= bea_m <= 1024 */
 } aif_user_inputs;
 
@@ -159,6 +167,12 @@ int aif_input_width(const aif_config *cfg);
 /* The 64-bit mix behind AIF_BUCKET_HASH: the splitmix64 output function applied to
  * id * 0x9E3779B97F4A7C15 + field.  Host function; the kernels compute the same value. */
 uint64_t aif_mix64(uint64_t id, uint64_t field);
+
+/* Category of an item when n_categories > 0 (Section 3.3 selects sub-sequences by the candidate's category; like the
+ * cross-feature attribute it is derived from the id here): id % n_categories (AIF_BUCKET_MOD) or
+ * aif_mix64(id, AIF_CATEGORY_FIELD) % n_categories (AIF_BUCKET_HASH).  Host function; the kernels compute the same. */
+#define AIF_CATEGORY_FIELD 3239
+int64_t aif_category(int64_t id, int32_t n_categories, int32_t bucket_mode);
 
 /* Creates a context on the current CUDA device: allocates the item table (M x d, plus M x n_bridge BEA
  * weights and M x lsh_bits/8 signature bytes when those blocks are on), the user-state arena, the status
@@ -221,7 +235,10 @@ int aif_item_nearline_compute(aif_ctx *ctx, const int32_t *ids, int64_t n, const
 /* User side, online-asynchronous (Section 3.1 eqs. 1-3, Section 3.3 "User-Side Pre-Processing").  Takes a free
  * slot of the arena and fills it on `side_stream`: u, S = U^_seq [L x d], the cross pre-cache T, V, the
  * sequence signatures, and p_u = W1[:, user columns] u + b1 (fp32), so that the real-time phase never touches
- * the user columns of the first layer again.  Records a "ready" event that aif_score waits on.
+ * the user columns of the first layer again.  With categories on it also lays the projected sequence (and its
+ * signatures) out a second time grouped by category, every sub-sequence padded with zero rows to a multiple of 128:
+ * this is the pre-cache of parsed sub-sequences for all of the user's categories that Section 3.3 builds in parallel
+ * with retrieval.  Records a "ready" event that aif_score waits on.
  * in: host struct of device pointers; the inputs must stay valid until the work on side_stream is done.
  * request_key: the caller's request identity (Section 3.4 keys the cached state by request), kept in the handle.
  * Calls with AIF_USER_RAW inputs share scratch of the context (the attention rows of eq. 2): issue them on one side

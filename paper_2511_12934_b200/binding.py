@@ -41,7 +41,7 @@ class aif_config(C.Structure):
         ("hidden", C.c_int32 * 4), ("bucket_mode", C.c_int32), ("blocks", C.c_int32), ("n_bridge", C.c_int32),
         ("lsh_bits", C.c_int32), ("n_tiers", C.c_int32), ("lsh_din_norm", C.c_int32), ("simtier_norm", C.c_int32),
         ("emit_sigmoid", C.c_int32), ("max_user_states", C.c_int32), ("mini_batch", C.c_int32), ("path", C.c_int32),
-        ("max_batch_candidates", C.c_int64),
+        ("n_categories", C.c_int32), ("max_batch_candidates", C.c_int64),
     ]
 
 
@@ -63,7 +63,8 @@ class aif_item_weights(C.Structure):
 class aif_user_inputs(C.Structure):
     _fields_ = [
         ("struct_size", C.c_uint32), ("mode", C.c_int32), ("profile", C.c_void_p), ("seq", C.c_void_p),
-        ("cross_raw", C.c_void_p), ("bea_V", C.c_void_p), ("seq_sig", C.c_void_p), ("bea_U", C.c_void_p), ("bea_m", C.c_int32),
+        ("cross_raw", C.c_void_p), ("bea_V", C.c_void_p), ("seq_sig", C.c_void_p), ("bea_U", C.c_void_p), ("seq_cat", C.c_void_p),
+        ("bea_m", C.c_int32),
     ]
 
 
@@ -79,7 +80,7 @@ class aif_stats(C.Structure):
 
 # every symbol include/aif.h declares
 EXPORTS = [
-    "aif_input_width", "aif_mix64", "aif_create", "aif_destroy", "aif_load_weights", "aif_item_nearline_refresh",
+    "aif_input_width", "aif_mix64", "aif_category", "aif_create", "aif_destroy", "aif_load_weights", "aif_item_nearline_refresh",
     "aif_load_item_weights", "aif_item_nearline_compute",
     "aif_user_precompute", "aif_user_release", "aif_user_request_key", "aif_user_state_export", "aif_user_state_export_bea", "aif_score",
     "aif_score_batch", "aif_score_host", "aif_score_batch_host", "aif_score_noalloc", "aif_gather_rows", "aif_gather_sidecars", "aif_poll_status", "aif_get_stats",
@@ -101,6 +102,7 @@ def load_library(path: Optional[str] = None):
     vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
     lib.aif_input_width.argtypes = [C.POINTER(aif_config)]
     lib.aif_mix64.argtypes, lib.aif_mix64.restype = [u64, u64], u64
+    lib.aif_category.argtypes, lib.aif_category.restype = [i64, i32, i32], i64
     lib.aif_create.argtypes = [C.POINTER(aif_config), C.POINTER(vp)]
     lib.aif_destroy.argtypes = [vp]
     lib.aif_load_weights.argtypes = [vp, C.POINTER(aif_weights), vp]
@@ -176,11 +178,11 @@ def _stream(s) -> C.c_void_p:
 def make_config(*, dtype, M, d, L_max, hidden: Sequence[int], F=0, B=1, dc=0, dU=0, bucket_mode=BUCKET_HASH,
                 blocks=BLK_ATT | BLK_CROSS, n_bridge=8, lsh_bits=0, n_tiers=8, lsh_din_norm=NORM_MEAN,
                 simtier_norm=NORM_MEAN, emit_sigmoid=0, max_user_states=4, mini_batch=0, path=PATH_AUTO,
-                max_batch_candidates=16384) -> aif_config:
+                max_batch_candidates=16384, n_categories=0) -> aif_config:
     h = list(hidden) + [0] * (4 - len(hidden))
     return aif_config(C.sizeof(aif_config), dtype, M, d, dU or d, L_max, F, B, dc, len(hidden), (C.c_int32 * 4)(*h),
                       bucket_mode, blocks, n_bridge, lsh_bits or d, n_tiers, lsh_din_norm, simtier_norm,
-                      emit_sigmoid, max_user_states, mini_batch, path, max_batch_candidates)
+                      emit_sigmoid, max_user_states, mini_batch, path, n_categories, max_batch_candidates)
 
 
 class UserState:
@@ -296,16 +298,17 @@ class Aif:
 
     # -- user side -------------------------------------------------------------------------------
     def user_precompute(self, request_key: int, *, mode: int, profile: torch.Tensor, seq: torch.Tensor,
-                        cross_raw=None, bea_V=None, seq_sig=None, bea_U=None, stream=None) -> UserState:
+                        cross_raw=None, bea_V=None, seq_sig=None, bea_U=None, seq_cat=None, stream=None) -> UserState:
         inp = aif_user_inputs(C.sizeof(aif_user_inputs), mode, profile.data_ptr(), seq.data_ptr(),
                               None if cross_raw is None else cross_raw.data_ptr(),
                               None if bea_V is None else bea_V.data_ptr(),
                               None if seq_sig is None else seq_sig.data_ptr(),
-                              None if bea_U is None else bea_U.data_ptr(), 0 if bea_U is None else bea_U.shape[0])
+                              None if bea_U is None else bea_U.data_ptr(), None if seq_cat is None else seq_cat.data_ptr(),
+                              0 if bea_U is None else bea_U.shape[0])
         out = C.c_void_p()
         _check(self.lib.aif_user_precompute(self.h, request_key, C.byref(inp), seq.shape[0], C.byref(out),
                                             _stream(stream)), "aif_user_precompute")
-        return UserState(self, out.value, (profile, seq, cross_raw, bea_V, seq_sig, bea_U))
+        return UserState(self, out.value, (profile, seq, cross_raw, bea_V, seq_sig, bea_U, seq_cat))
 
     def user_state_export(self, state: UserState, L: int, stream=None):
         u = torch.empty(self.cfg.d, dtype=torch.float32, device="cuda")

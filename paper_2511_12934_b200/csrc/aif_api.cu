@@ -65,6 +65,8 @@ int check_config(const aif_config *c)
     }
     if (c->max_user_states < 1 || c->mini_batch < 0 || c->max_batch_candidates < 1) return AIF_ERR_SHAPE;
     if (c->path < AIF_PATH_AUTO || c->path > AIF_PATH_TENSOR) return AIF_ERR_ARG;
+    if (c->n_categories < 0 || c->n_categories > 4096) return AIF_ERR_SHAPE;
+    if (c->n_categories > 0 && c->bucket_mode != AIF_BUCKET_MOD && c->bucket_mode != AIF_BUCKET_HASH) return AIF_ERR_ARG;
     return AIF_OK;
 }
 
@@ -162,6 +164,13 @@ int aif_input_width(const aif_config *c)
     return w;
 }
 
+int64_t aif_category(int64_t id, int32_t n_categories, int32_t bucket_mode)
+{
+    if (n_categories < 1) return 0;
+    if (bucket_mode == AIF_BUCKET_MOD) return id % n_categories;
+    return (int64_t)(aif_mix64((uint64_t)id, (uint64_t)AIF_CATEGORY_FIELD) % (uint64_t)n_categories);
+}
+
 uint64_t aif_mix64(uint64_t id, uint64_t field)
 {
     uint64_t z = id * 0x9E3779B97F4A7C15ull + field;
@@ -191,6 +200,18 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
         return AIF_ERR_SHAPE;
     }
     ctx->tensor_path = c.path != AIF_PATH_SIMT && tc_supported(c);
+    if (c.n_categories > 0) {
+        // sub-sequences by category are a feature of the tensor-core kernels: every sequence block that is on must be one
+        // of theirs
+        const bool att_ok = !(c.blocks & AIF_BLK_ATT) || tc_att_supported(c);
+        const bool lsh_ok = !(c.blocks & (AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER)) || tc_lsh_supported(c);
+        if (!ctx->tensor_path || !att_ok || !lsh_ok) {
+            delete ctx;
+            set_last_error("n_categories > 0 needs bf16 storage and d = 128 or 256 (tensor-core attention and LSH kernels)");
+            return AIF_ERR_SHAPE;
+        }
+        ctx->grouped_rows = sim_grouped_rows(c.L_max, c.n_categories);
+    }
 
 #define TRY(x)                 \
     do {                       \
@@ -224,7 +245,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     TRY(dev_alloc(ctx, (void **)&ctx->b_b, (size_t)c.d * 4, true));
 
     // user-state arena: fixed-size slots in one allocation
-    struct Off { size_t u, u32, S, T, V, sig, sigE, pu, pu_hl, prof, partial, ppart, end; } o{};
+    struct Off { size_t u, u32, S, T, V, sig, sigE, pu, pu_hl, prof, partial, ppart, Sg, sigEg, cat_off, cat_len, cat_map, cat_hist, end; } o{};
     size_t p = 0;
     auto take = [&](size_t bytes) { size_t at = p; p += align_up(bytes ? bytes : 16, 256); return at; };
     o.u = take((size_t)c.d * el);
@@ -240,6 +261,13 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     o.prof = take((size_t)c.d * 4);
     o.partial = take((size_t)kUserPartials * c.d * 4);
     o.ppart = take((size_t)kProfParts * (c.d + 2) * 4);
+    const bool sim = c.n_categories > 0;
+    o.Sg = take(sim ? ctx->grouped_rows * c.d * el : 0);
+    o.sigEg = take(sim && lsh_tc ? ctx->grouped_rows * c.lsh_bits : 0);
+    o.cat_off = take(sim ? (size_t)c.n_categories * 4 : 0);
+    o.cat_len = take(sim ? (size_t)c.n_categories * 4 : 0);
+    o.cat_map = take(sim ? (size_t)c.L_max * 4 : 0);
+    o.cat_hist = take(sim ? (size_t)((c.L_max + 1023) / 1024) * c.n_categories * 4 : 0);
     o.end = p;
     ctx->slot_bytes = o.end;
     TRY(dev_alloc(ctx, (void **)&ctx->arena, ctx->slot_bytes * (size_t)c.max_user_states, true));
@@ -255,6 +283,11 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
         hs.dev.sigE = lsh_tc ? (const uint8_t *)(base + o.sigE) : nullptr;
         hs.dev.p_u = (const float *)(base + o.pu), hs.dev.pu_hl = base + o.pu_hl, hs.dev.L = 0;
         hs.prof_hat = (float *)(base + o.prof), hs.partial = (float *)(base + o.partial), hs.ppart = (float *)(base + o.ppart);
+        if (sim) {
+            hs.dev.Sg = base + o.Sg, hs.dev.sigEg = lsh_tc ? (const uint8_t *)(base + o.sigEg) : nullptr;
+            hs.dev.cat_off = (const int32_t *)(base + o.cat_off), hs.dev.cat_len = (const int32_t *)(base + o.cat_len);
+            hs.cat_map = (int32_t *)(base + o.cat_map), hs.cat_hist = (int32_t *)(base + o.cat_hist);
+        }
         cudaError_t e = cudaEventCreateWithFlags(&hs.ev, cudaEventDisableTiming);
         if (e != cudaSuccess) {
             aif_destroy(ctx);
@@ -312,6 +345,7 @@ int aif_destroy(aif_ctx *ctx)
         if (ctx->ring.host[i]) cudaFreeHost(ctx->ring.host[i]);
         if (ctx->ring.ev[i]) cudaEventDestroy(ctx->ring.ev[i]);
     }
+    if (ctx->sim_plan) sim_destroy(ctx);
     if (ctx->tc_plan) tc_destroy_context(ctx);
     if (ctx->nearline_plan) nearline_destroy(ctx);
     for (void *p : ctx->allocations) cudaFree(p);
@@ -426,6 +460,7 @@ int aif_user_precompute(aif_ctx *ctx, uint64_t request_key, const aif_user_input
         if (!ctx->bea_user_weights) return AIF_ERR_NOT_READY;
     }
     if ((c.blocks & (AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER)) && !in->seq_sig) return AIF_ERR_ARG;
+    if (c.n_categories > 0 && !in->seq_cat) return AIF_ERR_ARG;
     int idx = -1;
     for (int i = 0; i < (int)ctx->slots.size(); ++i)
         if (!ctx->slots[(size_t)i].in_use) {
@@ -437,6 +472,7 @@ int aif_user_precompute(aif_ctx *ctx, uint64_t request_key, const aif_user_input
     HostSlot &hs = ctx->slots[(size_t)idx];
     cudaStream_t st = as_stream(side_stream);
     AIF_CUDA(launch_user_network(ctx, hs, idx, in, L, st));
+    if (c.n_categories > 0) AIF_CUDA(sim_group_sequence(ctx, hs, in->seq_cat, L, st));
     AIF_CUDA(cudaEventRecord(hs.ev, st));
     hs.ev_seen_done = false;
     hs.in_use = true, hs.ready = true, hs.L = L, hs.key = request_key, hs.model_version = ctx->model_version;
@@ -562,7 +598,7 @@ int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *st
         tiles += tiles_for(ctx, n);
         AIF_CUDA(wait_user_ready(ctx->slots[(size_t)states[r]->index], st));
     }
-    if (ctx->tensor_path && (size_t)tiles > tc_tile_capacity(ctx)) {
+    if (ctx->tensor_path && ctx->cfg.n_categories == 0 && (size_t)tiles > tc_tile_capacity(ctx)) {
         snprintf(g_last_error, sizeof(g_last_error), "aif_score_batch: %d tiles exceed the tile table's %zu entries", tiles,
                  tc_tile_capacity(ctx));
         return AIF_ERR_SHAPE;

@@ -28,6 +28,12 @@ struct SlotDev {
     const uint8_t *sigE;    // [L x lsh_bits] the same signatures with one E4M3 byte per bit, +1.0 / -1.0 (tensor-core LSH), or nullptr
     const float *p_u;       // [H1] fp32: W1[:, user columns] u + b1
     const void *pu_hl;      // [2][H1] bf16: p_u split into high parts and remainders (bias operand of the tensor cores)
+    // categories on: the sequence a second time, grouped by category, every sub-sequence padded with zero rows to a multiple
+    // of 128 (the pre-cache of parsed sub-sequences, Section 3.3)
+    const void *Sg;         // [Lg x d] storage type, Lg = grouped_rows(L_max, n_categories)
+    const uint8_t *sigEg;   // [Lg x lsh_bits] +-1 bytes, or nullptr
+    const int32_t *cat_off; // [n_categories] first row of every sub-sequence in Sg
+    const int32_t *cat_len; // [n_categories] items of every sub-sequence
     int32_t L;
     int32_t pad_;
 };
@@ -62,8 +68,9 @@ struct TileDev {
     int32_t slot;
     int32_t cnt;     // candidates in the tile
     int64_t pos0;    // position of its first candidate in ids / logits
-    int32_t L;       // sequence length of the tile's request
-    int32_t pad_[3];
+    int32_t L;       // keys of the tile: the request's sequence length, or the length of its category's sub-sequence
+    int32_t key0;    // first key row (0, or where the category's sub-sequence begins in the grouped sequence)
+    int32_t pad_[2];
 };
 
 struct ScoreLaunch {
@@ -78,6 +85,12 @@ struct ScoreLaunch {
     float *logits;
     uint32_t *status;
     const TileDev *tiles;   // [n_tiles] (tensor-core tiles), or nullptr: search `reqs` per tile
+    // categories on: tiles are formed on the device from the candidates grouped by (request, category).  n_tiles above is
+    // then an upper bound that sizes grids, the count is read from n_tiles_dev; ids are the grouped candidates, and
+    // out_index[p] is where the logit of grouped position p belongs in the caller's array.
+    const int32_t *n_tiles_dev;
+    const int32_t *out_index;
+    int32_t grouped;        // 1: key blocks come from the grouped sequence
 };
 
 struct HostSlot {
@@ -93,6 +106,8 @@ struct HostSlot {
     float *prof_hat = nullptr;   // [d]
     float *partial = nullptr;    // [kUserPartials x d]
     float *ppart = nullptr;      // [kProfParts x (d + 2)]: per key slice, unnormalised attention row, maximum, sum
+    int32_t *cat_map = nullptr;  // [L_max]: row of every sequence item in the grouped sequence (scratch of the grouping)
+    int32_t *cat_hist = nullptr; // [ceil(L_max / 1024) x n_categories]: per 1024-item block, items of every category
 };
 
 constexpr int kUserPartials = 1184;
@@ -165,6 +180,8 @@ struct aif_ctx {
     void *nearline_plan = nullptr;    // item-side weights and scratch of aif_item_nearline_compute
     void *tc_fused_plan = nullptr;    // single-launch scoring: the second layer's bias split into two bf16 rows
     void *tc_lsh_plan = nullptr;      // tensor-core LSH blocks: tensor maps over the arena's S and +-1 signature regions
+    void *sim_plan = nullptr;         // categories on: scratch of the grouping passes (aif_sim.cu)
+    size_t grouped_rows = 0;          // rows of a slot's grouped sequence
     aif::PinnedRing ring;
 
     aif_stats stats{};
@@ -214,6 +231,15 @@ void tc_lsh_destroy(aif_ctx *ctx);
 cudaError_t launch_expand_signatures(const aif_ctx *ctx, const uint8_t *sig, int L, uint8_t *out, cudaStream_t st);
 cudaError_t launch_lsh_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_t st, void *X, int x_stride, size_t x_rows, int x_din,
                           int x_tier);
+// category sub-sequences (aif_sim.cu): the user-side grouping of a sequence, and the grouping of a launch's candidates by
+// (request, category) into tiles
+size_t sim_grouped_rows(int L_max, int n_categories);
+cudaError_t sim_prepare(aif_ctx *ctx);
+void sim_destroy(aif_ctx *ctx);
+size_t sim_tile_capacity(const aif_ctx *ctx);
+cudaError_t sim_group_sequence(const aif_ctx *ctx, HostSlot &hs, const int32_t *seq_cat, int L, cudaStream_t st);
+// fills sl (ids, tiles, n_tiles upper bound, n_tiles_dev, out_index) for a launch whose original ids are sl.ids
+cudaError_t sim_group_candidates(const aif_ctx *ctx, ScoreLaunch &sl, cudaStream_t st);
 // whole scoring pass of a tile in one CTA (aif_tc_fused.cu); the tensor maps it shares with the other kernels
 bool tc_fused_supported(const aif_config &cfg);
 cudaError_t tc_fused_prepare(aif_ctx *ctx);

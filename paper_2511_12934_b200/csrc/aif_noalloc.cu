@@ -65,6 +65,10 @@ extern "C" int aif_score_noalloc(aif_ctx *ctx, const aif_user_state *state, cons
         set_last_error("aif_score_noalloc: this context runs the CUDA-core kernel, which has no scratch; use aif_score");
         return AIF_ERR_SHAPE;
     }
+    if (ctx->cfg.n_categories > 0) {
+        set_last_error("aif_score_noalloc: contexts with category sub-sequences group their candidates in allocated scratch; use aif_score");
+        return AIF_ERR_SHAPE;
+    }
     if (tc_scratch_row_bytes(ctx) > (size_t)kRowBytes) {
         char msg[200];
         snprintf(msg, sizeof(msg), "aif_score_noalloc: model needs %zu scratch bytes per candidate, limit is %d",

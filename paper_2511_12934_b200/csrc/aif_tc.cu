@@ -100,10 +100,10 @@ struct TileInfo {
     int64_t pos0;   // position of the tile's first candidate in the launch (ids / logits / dense rows)
 };
 
-__device__ __forceinline__ TileInfo decode_tile(const LayerParams &p, int tile)
+__device__ __forceinline__ TileInfo decode_tile(const LayerParams &p, int tile, int n_tiles)
 {
     TileInfo t;
-    if (tile >= p.sl.n_tiles) {   // the second tile of the last group may not exist
+    if (tile >= n_tiles) {   // the second tile of the last group may not exist
         t.rq = ReqDev{0, 0, 0, 0, 0};
         t.start = 0, t.cnt = 0, t.pos0 = 0;
         return t;
@@ -193,9 +193,6 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
     int *ids_s = reinterpret_cast<int *>(wout_s + kAcc * 256);   // [2][G][128] validated ids of the current / next item
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n_groups = (p.sl.n_tiles + G - 1) / G;
-    const int n_ncg = p.n_nchunks / NB;             // groups of output slices
-    const int n_items = n_groups * n_ncg;
 
     if (tid == 0) {
         for (int s = 0; s < kSA; ++s) {
@@ -220,6 +217,11 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
     const uint32_t tmem_base = *tmem_slot;
     grid_dep_launch();
     grid_dep_wait();   // everything above overlapped the tail of the previous kernel; from here on its results are read
+    // tiles formed on the device (candidates grouped by category): their number is read here
+    const int n_tiles = p.sl.n_tiles_dev ? *p.sl.n_tiles_dev : p.sl.n_tiles;
+    const int n_groups = (n_tiles + G - 1) / G;
+    const int n_ncg = p.n_nchunks / NB;             // groups of output slices
+    const int n_items = n_groups * n_ncg;
 
     if (warp < C::kEpiWarps) {
         // ===================== epilogue =====================
@@ -238,7 +240,7 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
             const int grp = item / n_ncg, nc = (item - grp * n_ncg) * NB + (NB == 2 ? a : 0), n0 = nc * p.n_cols;
             const int buf = kAcc == 1 ? (it & 1) : a;
             const uint32_t ph = kAcc == 1 ? (uint32_t)((it >> 1) & 1) : (uint32_t)(it & 1);
-            const TileInfo t = decode_tile(p, grp * G + g);
+            const TileInfo t = decode_tile(p, grp * G + g, n_tiles);
             if (t.cnt > 0) {
                 const float *bias = p.bias_from_slot ? p.sl.slots[t.rq.slot].p_u : p.bias;
                 for (int j = row; j < p.n_cols; j += 128) {
@@ -334,7 +336,7 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
                 // no number for an id outside the table, nor for a tile whose inputs never arrived (here or in an
                 // earlier kernel of the call: the status word says so)
                 if (id < 0 || (int64_t)id >= p.M || !got || poisoned) logit = __int_as_float(0x7fc00000);
-                p.sl.logits[t.pos0 + row] = logit;
+                p.sl.logits[p.sl.out_index ? (int64_t)p.sl.out_index[t.pos0 + row] : t.pos0 + row] = logit;
             }
             if (named_bar_or(1 + a, 128, !got)) break;
         }
@@ -411,7 +413,7 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
         };
         const uint32_t xb_step = (uint32_t)(16 * p.F);   // elements between the bucket rows of rows r0 + 16 i and r0 + 16 (i + 1)
         auto load_rows = [&](int item, Rows &R, int &pend) {
-            const TileInfo t = decode_tile(p, (item / n_ncg) * G + gt);
+            const TileInfo t = decode_tile(p, (item / n_ncg) * G + gt, n_tiles);
             const int nrows = t.cnt > r0 ? (t.cnt - r0 + 15) >> 4 : 0;
             R.rowmask = (1u << nrows) - 1u, R.pos0 = (uint32_t)t.pos0;
             R.Tt = t.cnt > 0 ? reinterpret_cast<const uint8_t *>(p.sl.slots[t.rq.slot].T) : p.E;
@@ -598,10 +600,20 @@ __global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl,
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, d = md.d, dq = d >> 5;
     grid_dep_launch();
     grid_dep_wait();
-    const ReqDev rq = find_request(sl, blockIdx.x);
-    int start, cnt;
-    tile_range(blockIdx.x - rq.tile_begin, rq.n, kTcTile, md.mini_batch, start, cnt);
-    const SlotDev slot = sl.slots[rq.slot];
+    // the tile: from the launch's tile table when it has one that was formed on the device, else from the request table
+    int slot_index, cnt;
+    int64_t pos0;
+    if (sl.n_tiles_dev) {
+        if ((int)blockIdx.x >= *sl.n_tiles_dev) return;
+        const TileDev t = sl.tiles[blockIdx.x];
+        slot_index = t.slot, cnt = t.cnt, pos0 = t.pos0;
+    } else {
+        const ReqDev rq = find_request(sl, blockIdx.x);
+        int start;
+        tile_range(blockIdx.x - rq.tile_begin, rq.n, kTcTile, md.mini_batch, start, cnt);
+        slot_index = rq.slot, pos0 = rq.off + start;
+    }
+    const SlotDev slot = sl.slots[slot_index];
     // att_done / lsh_done: those columns were already written by the tensor-core attention / LSH kernels
     const bool has_att = md.blocks & AIF_BLK_ATT, do_att = has_att && !att_done, do_bea = md.blocks & AIF_BLK_BEA;
     const bool has_din = md.blocks & AIF_BLK_LSH_DIN, has_tier = md.blocks & AIF_BLK_SIMTIER;
@@ -609,7 +621,7 @@ __global__ void __launch_bounds__(256) k_interact_x(ModelDev md, ScoreLaunch sl,
     const int col_bea = has_att ? d : 0, col_din = col_bea + (do_bea ? d : 0), col_tier = col_din + (has_din ? d : 0);
     using T = __nv_bfloat16;
     for (int c = warp; c < cnt; c += 8) {
-        const int64_t pos = rq.off + start + c;
+        const int64_t pos = pos0 + c;
         const int id = sl.ids[pos];
         T *xrow = X + (size_t)pos * x_stride;
         if (id < 0 || (int64_t)id >= md.M) {
@@ -838,6 +850,7 @@ cudaError_t tc_prepare_context(aif_ctx *ctx)
     if (tc_att_supported(c) && (e = tc_att_prepare(ctx)) != cudaSuccess) return e;
     if (tc_fused_supported(c) && (e = tc_fused_prepare(ctx)) != cudaSuccess) return e;
     if (tc_lsh_supported(c) && (e = tc_lsh_prepare(ctx)) != cudaSuccess) return e;
+    if (c.n_categories > 0 && (e = sim_prepare(ctx)) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
@@ -984,12 +997,18 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl_in
     const ModelDev md = make_model(ctx);
     timing_begin(ctx, st);
     // a launch that fits the machine in one round of tiles: the whole pass in one kernel, one CTA per tile
-    if (sl.n_tiles <= kFusedMaxTiles && sl.max_L <= 256 && tc_fused_supported(c)) {
+    if (c.n_categories == 0 && sl.n_tiles <= kFusedMaxTiles && sl.max_L <= 256 && tc_fused_supported(c)) {
         cudaError_t e = launch_request_fused(ctx, sl, st);
         timing_mark(ctx, "score_fused", st);
         return e;
     }
-    if (sl.reqs && sc.tiles) {   // several requests: look every tile up once
+    if (c.n_categories > 0) {
+        // candidates grouped by (request, category): tiles, grouped ids and the way back to the caller's order
+        if (sc.rows < (size_t)sl.total + kTcTile || !ctx->sim_plan) return cudaErrorInvalidValue;
+        cudaError_t e = sim_group_candidates(ctx, sl, st);
+        timing_mark(ctx, "group", st);
+        if (e != cudaSuccess) return e;
+    } else if (sl.reqs && sc.tiles) {   // several requests: look every tile up once
         cudaError_t e = launch_pdl(k_tile_table, dim3((sl.n_tiles + 255) / 256), dim3(256), 0, st, sl, c.mini_batch, (TileDev *)sc.tiles);
         count_launch();
         if (e != cudaSuccess) return e;

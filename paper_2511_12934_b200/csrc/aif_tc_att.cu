@@ -67,6 +67,7 @@ struct AttCfg {
 // One tile of the launch as every role needs it.
 struct AttTile {
     int slot, cnt, nb, L;
+    int key0;   // first key row: 0, or where the tile's category's sub-sequence begins in the grouped sequence
     int64_t pos0;
 };
 
@@ -78,15 +79,16 @@ __device__ __forceinline__ AttTile att_tile(const AttParams &p, int tile)
         const int4 v = *reinterpret_cast<const int4 *>(p.sl.tiles + tile);   // slot, cnt, pos0
         t.slot = v.x, t.cnt = v.y;
         t.pos0 = ((int64_t)(uint32_t)v.w << 32) | (int64_t)(uint32_t)v.z;
-        t.L = p.sl.tiles[tile].L;
-        t.nb = (t.L + BN - 1) / BN;
+        t.L = p.sl.tiles[tile].L, t.key0 = p.sl.tiles[tile].key0;
+        // an empty sub-sequence still walks one key block, every column of it masked: the roles' hand-overs stay the same
+        t.nb = t.L > 0 ? (t.L + BN - 1) / BN : 1;
         return t;
     }
     const ReqDev rq = find_request(p.sl, tile);
     int start, cnt;
     tile_range(tile - rq.tile_begin, rq.n, kTcTile, p.mini_batch, start, cnt);
     t.slot = rq.slot, t.cnt = cnt, t.pos0 = rq.off + start;
-    t.L = p.sl.slots[rq.slot].L;
+    t.L = p.sl.slots[rq.slot].L, t.key0 = 0;
     t.nb = (t.L + BN - 1) / BN;
     return t;
 }
@@ -143,7 +145,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
     grid_dep_launch();
     grid_dep_wait();   // the set-up above overlapped the previous kernel; the request table and slots are read from here on
 
-    const int n_tiles = p.sl.n_tiles;
+    const int n_tiles = p.sl.n_tiles_dev ? *p.sl.n_tiles_dev : p.sl.n_tiles;
 
     // Normalises a finished tile's O accumulator and stores the attention rows.  Run by the softmax warps themselves
     // (d = 256) or by the epilogue warps (d = 128); wq = the warp's quarter of the TMEM lanes.
@@ -152,7 +154,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
         const uint32_t lane_base = tmem_base + ((uint32_t)(wq * 32) << 16);
         const uint32_t o_col = (uint32_t)(C::kTmemO + (kSplit ? (k & 1) * D : 0));
         uint64_t *o_free_k = o_free + (kSplit ? (k & 1) : 0);
-        const float inv = 1.0f / l_sum;
+        const float inv = l_sum > 0.f ? 1.0f / l_sum : 0.f;   // no key at all (an empty sub-sequence): a zero row
         bool good = false;
         if (row < t.cnt) {
             const int id = p.sl.ids[t.pos0 + row];
@@ -490,7 +492,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
 #pragma unroll
                     for (int c = 0; c < C::kQChunks; ++c)
                         tma_load_3d(smem_u32(smKV + s * C::kKvBytes + c * C::kKvChunkBytes), &tmapS, smem_u32(kv_full + s), c * 64,
-                                    j * BN, t.slot);
+                                    t.key0 + j * BN, t.slot);
                 }
             }
         }
@@ -561,6 +563,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
 
 struct AttPlan {
     CUtensorMap tmap;
+    CUtensorMap tmap_g;                   // categories on: over the grouped sequences
     int bn = 0;
     __nv_bfloat16 *self_rows = nullptr;   // [L_max + 128][d]: attention rows of eq. 2 for the user state being computed
     int32_t *iota = nullptr;              // 0, 1, 2, ...: the "candidate ids" of that launch are the sequence positions
@@ -595,6 +598,12 @@ cudaError_t tc_att_prepare(aif_ctx *ctx)
     CUresult r = enc(&pl->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    if (c.n_categories > 0) {
+        const cuuint64_t gdims[3] = {(cuuint64_t)c.d, (cuuint64_t)ctx->grouped_rows, (cuuint64_t)c.max_user_states};
+        r = enc(&pl->tmap_g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ctx->slots[0].dev.Sg), gdims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    }
     cudaError_t e;
     {   // scratch of the user-side self-attention
         const size_t rows = (size_t)c.L_max + kTcTile;
@@ -660,10 +669,11 @@ cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
     // 9 tile times) as soon as some SM has two tiles.
     const int grid = sl.n_tiles > 148 ? 148 : sl.n_tiles;
     cudaError_t e;
+    const CUtensorMap &tm = sl.grouped ? pl->tmap_g : pl->tmap;
     if (c.d == 128)
-        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(AttCfg<128, 128>::kThreads), AttCfg<128, 128>::kSmem, st, pl->tmap, tmap_x, p);
+        e = launch_pdl(k_att_tc<128, 128>, dim3(grid), dim3(AttCfg<128, 128>::kThreads), AttCfg<128, 128>::kSmem, st, tm, tmap_x, p);
     else
-        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(AttCfg<256, 64>::kThreads), AttCfg<256, 64>::kSmem, st, pl->tmap, tmap_x, p);
+        e = launch_pdl(k_att_tc<256, 64>, dim3(grid), dim3(AttCfg<256, 64>::kThreads), AttCfg<256, 64>::kSmem, st, tm, tmap_x, p);
     count_launch();
     return e;
 }

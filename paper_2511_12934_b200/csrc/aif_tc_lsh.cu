@@ -86,6 +86,7 @@ struct LshCfg {
 
 struct LshTile {
     int slot, cnt, nb, L;
+    int key0;   // first key row: 0, or where the tile's category's sub-sequence begins in the grouped sequence
     int64_t pos0;
 };
 
@@ -97,15 +98,16 @@ __device__ __forceinline__ LshTile lsh_tile(const LshParams &p, int tile)
         const int4 v = *reinterpret_cast<const int4 *>(p.sl.tiles + tile);
         t.slot = v.x, t.cnt = v.y;
         t.pos0 = ((int64_t)(uint32_t)v.w << 32) | (int64_t)(uint32_t)v.z;
-        t.L = p.sl.tiles[tile].L;
-        t.nb = (t.L + BN - 1) / BN;
+        t.L = p.sl.tiles[tile].L, t.key0 = p.sl.tiles[tile].key0;
+        // an empty sub-sequence still walks one key block (its outputs are forced to zero): the hand-overs stay the same
+        t.nb = t.L > 0 ? (t.L + BN - 1) / BN : 1;
         return t;
     }
     const ReqDev rq = find_request(p.sl, tile);
     int start, cnt;
     tile_range(tile - rq.tile_begin, rq.n, kTcTile, p.mini_batch, start, cnt);
     t.slot = rq.slot, t.cnt = cnt, t.pos0 = rq.off + start;
-    t.L = p.sl.slots[rq.slot].L;
+    t.L = p.sl.slots[rq.slot].L, t.key0 = 0;
     t.nb = (t.L + BN - 1) / BN;
     return t;
 }
@@ -254,7 +256,7 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
     grid_dep_launch();
     grid_dep_wait();
 
-    const int n_tiles = p.sl.n_tiles;
+    const int n_tiles = p.sl.n_tiles_dev ? *p.sl.n_tiles_dev : p.sl.n_tiles;
 
     // A row's item signature as +-1 bytes in the operand layout (128-byte swizzled K-major chunks): 8 threads per row,
     // 16 bits (two signature bytes) each per 128-bit chunk.
@@ -278,7 +280,7 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
         uint64_t *o_free_k = o_free;
         const float scale = (0.5f / (float)D) * (p.din_mean ? 1.0f / (float)t.L : 1.0f);
         bool good = false;
-        if (row < t.cnt) {
+        if (row < t.cnt && t.L > 0) {   // an empty sub-sequence gives zero rows
             const int id = p.sl.ids[t.pos0 + row];
             good = id >= 0 && (int64_t)id < p.M;
         }
@@ -438,7 +440,7 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
                     int total = n_valid, pads = n_pad;
                     if (kH == 2) total += (int)(tc1[15 * 128] & 0xFFFFFFu), pads += (int)(tc1[15 * 128] >> 24);
                     bool good = false;
-                    if (row < t.cnt) {
+                    if (row < t.cnt && L > 0) {
                         const int id = p.sl.ids[t.pos0 + row];
                         good = id >= 0 && (int64_t)id < p.M;
                     }
@@ -565,13 +567,13 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
             // two cursors over the same sequence of key blocks: the signature stream runs up to three blocks ahead of the
             // stream of S rows, which is held back by the products that still read its stages
             struct Stream {
-                int tile, j, nb, slot;
+                int tile, j, nb, slot, key0;
                 uint32_t gb;
             };
             auto open = [&](Stream &c) {
                 if (c.tile < n_tiles) {
                     const LshTile t = lsh_tile<BN>(p, c.tile);
-                    c.nb = t.nb, c.slot = t.slot;
+                    c.nb = t.nb, c.slot = t.slot, c.key0 = t.key0;
                 }
             };
             auto step = [&](Stream &c) {
@@ -581,7 +583,7 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
                     open(c);
                 }
             };
-            Stream g{(int)blockIdx.x, 0, 0, 0, 0u}, v{(int)blockIdx.x, 0, 0, 0, 0u};
+            Stream g{(int)blockIdx.x, 0, 0, 0, 0, 0u}, v{(int)blockIdx.x, 0, 0, 0, 0, 0u};
             open(g), open(v);
             bool ok = true;
             while (ok && v.tile < n_tiles) {
@@ -594,7 +596,8 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
                     mbar_expect_tx(smem_u32(g_full + s), (uint32_t)C::kGBytes);
 #pragma unroll
                     for (int c = 0; c < C::kQChunks; ++c)
-                        tma_load_3d(smem_u32(smG + s * C::kGBytes + c * C::kGChunkBytes), &tmapG, smem_u32(g_full + s), c * 128, g.j * BN, g.slot);
+                        tma_load_3d(smem_u32(smG + s * C::kGBytes + c * C::kGChunkBytes), &tmapG, smem_u32(g_full + s), c * 128,
+                                    g.key0 + g.j * BN, g.slot);
                     step(g);
                 }
                 if (!ok) break;
@@ -603,7 +606,8 @@ __global__ void __launch_bounds__((LshCfg<D, BN>::kThreads), 1) k_lsh_tc(const _
                 mbar_expect_tx(smem_u32(v_full + s), (uint32_t)C::kVBytes);
 #pragma unroll
                 for (int c = 0; c < C::kVChunks; ++c)
-                    tma_load_3d(smem_u32(smV + s * C::kVBytes + c * C::kVChunkBytes), &tmapS, smem_u32(v_full + s), c * 64, v.j * BN, v.slot);
+                    tma_load_3d(smem_u32(smV + s * C::kVBytes + c * C::kVChunkBytes), &tmapS, smem_u32(v_full + s), c * 64,
+                                v.key0 + v.j * BN, v.slot);
                 step(v);
             }
         }
@@ -673,6 +677,7 @@ __global__ void __launch_bounds__(256) k_expand_signatures(const uint8_t *__rest
 
 struct LshPlan {
     CUtensorMap tmap_s, tmap_g;
+    CUtensorMap tmap_sg, tmap_gg;   // categories on: the same over the grouped sequences
     int bn = 0;
 };
 
@@ -708,6 +713,22 @@ cudaError_t tc_lsh_prepare(aif_ctx *ctx)
         const cuuint64_t strides[2] = {(cuuint64_t)c.lsh_bits, (cuuint64_t)ctx->slot_bytes};
         const cuuint32_t box[3] = {128, (cuuint32_t)pl->bn, 1};
         if (enc(&pl->tmap_g, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>(ctx->slots[0].dev.sigE), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    if (c.n_categories > 0) {
+        const cuuint64_t dims[3] = {(cuuint64_t)c.d, (cuuint64_t)ctx->grouped_rows, (cuuint64_t)c.max_user_states};
+        const cuuint64_t strides[2] = {(cuuint64_t)c.d * 2, (cuuint64_t)ctx->slot_bytes};
+        const cuuint32_t box[3] = {64, (cuuint32_t)pl->bn, 1};
+        if (enc(&pl->tmap_sg, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ctx->slots[0].dev.Sg), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+        const cuuint64_t gdims[3] = {(cuuint64_t)c.lsh_bits, (cuuint64_t)ctx->grouped_rows, (cuuint64_t)c.max_user_states};
+        const cuuint64_t gstrides[2] = {(cuuint64_t)c.lsh_bits, (cuuint64_t)ctx->slot_bytes};
+        const cuuint32_t gbox[3] = {128, (cuuint32_t)pl->bn, 1};
+        if (enc(&pl->tmap_gg, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>(ctx->slots[0].dev.sigEg), gdims, gstrides, gbox, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
@@ -761,10 +782,11 @@ cudaError_t launch_lsh_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
     p.din_mean = c.lsh_din_norm == AIF_NORM_MEAN, p.tier_mean = c.simtier_norm == AIF_NORM_MEAN;
     const int grid = sl.n_tiles > 148 ? 148 : sl.n_tiles;
     cudaError_t e;
+    const CUtensorMap &ts = sl.grouped ? pl->tmap_sg : pl->tmap_s, &tg = sl.grouped ? pl->tmap_gg : pl->tmap_g;
     if (c.d == 128)
-        e = launch_pdl(k_lsh_tc<128, 128>, dim3(grid), dim3(LshCfg<128, 128>::kThreads), LshCfg<128, 128>::kSmem, st, pl->tmap_s, pl->tmap_g, tmap_x, p);
+        e = launch_pdl(k_lsh_tc<128, 128>, dim3(grid), dim3(LshCfg<128, 128>::kThreads), LshCfg<128, 128>::kSmem, st, ts, tg, tmap_x, p);
     else
-        e = launch_pdl(k_lsh_tc<256, 64>, dim3(grid), dim3(LshCfg<256, 64>::kThreads), LshCfg<256, 64>::kSmem, st, pl->tmap_s, pl->tmap_g, tmap_x, p);
+        e = launch_pdl(k_lsh_tc<256, 64>, dim3(grid), dim3(LshCfg<256, 64>::kThreads), LshCfg<256, 64>::kSmem, st, ts, tg, tmap_x, p);
     count_launch();
     return e;
 }

@@ -21,7 +21,7 @@ def config_for(wl: synth.Workload, *, rows: Optional[int] = None, L_max: Optiona
         dU=wl.raw_dU, bucket_mode=wl.bucket_mode, blocks=wl.blocks, n_bridge=wl.n_bridge, lsh_bits=wl.lsh_bits,
         n_tiers=wl.n_tiers, lsh_din_norm=wl.lsh_din_norm, simtier_norm=wl.simtier_norm,
         emit_sigmoid=wl.emit_sigmoid, max_user_states=max_user_states or max(2, wl.R), mini_batch=wl.mini_batch,
-        path=path, max_batch_candidates=max_batch_candidates or max(1, wl.R * wl.N))
+        path=path, max_batch_candidates=max_batch_candidates or max(1, wl.R * wl.N), n_categories=wl.n_categories)
 
 
 class Server:
@@ -61,13 +61,14 @@ class Server:
         dev["bea_V"] = B.to_device(rq["V"], self.dt) if "V" in rq else None
         dev["bea_U"] = B.to_device(rq["bea_U"], self.dt) if "bea_U" in rq else None   # Algorithm 1's U: V is computed
         dev["seq_sig"] = torch.from_numpy(np.ascontiguousarray(rq["sig_seq"])).cuda() if "sig_seq" in rq else None
+        dev["seq_cat"] = torch.from_numpy(np.ascontiguousarray(rq["seq_cat"], dtype=np.int32)).cuda() if "seq_cat" in rq else None
         return dev
 
     def precompute(self, key: int, dev: dict, stream=None) -> B.UserState:
         """aif_user_precompute on the side stream (or `stream`)."""
         return self.ctx.user_precompute(key, mode=dev["mode"], profile=dev["profile"], seq=dev["seq"],
                                         cross_raw=dev["cross_raw"], bea_V=dev["bea_V"], seq_sig=dev["seq_sig"],
-                                        bea_U=dev.get("bea_U"), stream=stream or self.side)
+                                        bea_U=dev.get("bea_U"), seq_cat=dev.get("seq_cat"), stream=stream or self.side)
 
     def score_ids(self, state: B.UserState, ids: np.ndarray) -> np.ndarray:
         ids_t = torch.from_numpy(np.ascontiguousarray(ids, dtype=np.int32)).cuda()

@@ -36,9 +36,9 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_layouts_match_the_header(lib):
     # sizes follow from the header's field lists under the C ABI (natural alignment)
-    assert C.sizeof(B.aif_config) == 112
+    assert C.sizeof(B.aif_config) == 120
     assert C.sizeof(B.aif_weights) == 8 + 4 * 8 + 4 * 8 + 10 * 8
-    assert C.sizeof(B.aif_user_inputs) == 8 + 6 * 8 + 8
+    assert C.sizeof(B.aif_user_inputs) == 8 + 7 * 8 + 8
     assert C.sizeof(B.aif_item_weights) == 16 + 6 * 8
     cfg = B.make_config(dtype=B.BF16, M=1000, d=128, L_max=10, hidden=(512, 256), F=16, B=1024, dc=32)
     assert lib.aif_input_width(C.byref(cfg)) == 128 * 3 + 16 * 32
@@ -49,6 +49,9 @@ def test_host_hash_matches_oracle_hash(lib):
     for i in (0, 1, 2, 77, 123456789, 2**31 - 1):
         for f in (0, 1, 15, 63):
             assert B.mix64(i, f) == orc.mix64(i, f)
+        for n_cat in (1, 7, 100):
+            for mode in (B.BUCKET_MOD, B.BUCKET_HASH):
+                assert lib.aif_category(i, n_cat, mode) == orc.category(i, n_cat, mode)
 
 
 def test_argument_errors_without_a_device(lib):
