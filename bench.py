@@ -56,10 +56,13 @@ def ncu_traffic_table():
 # ----------------------------------------------------------------------------------------------------------------
 # algorithmic work (what the method itself has to do; padding and recomputation are not counted)
 # ----------------------------------------------------------------------------------------------------------------
-def flops_per_candidate(wl: synth.Workload) -> dict:
+def flops_per_candidate(wl: synth.Workload, keys=None) -> dict:
+    """keys: mean number of sequence items a candidate interacts with (the whole sequence unless the workload has
+    category sub-sequences)."""
     k1 = wl.input_width() - wl.d                       # the user columns are done once per request
-    f = {"attention": 4.0 * wl.L * wl.d if wl.blocks & synth.BLK_ATT else 0.0}
-    f["lsh_din"] = 2.0 * wl.L * wl.d if wl.blocks & synth.BLK_LSH_DIN else 0.0
+    keys = float(wl.L if keys is None else keys)
+    f = {"attention": 4.0 * keys * wl.d if wl.blocks & synth.BLK_ATT else 0.0}
+    f["lsh_din"] = 2.0 * keys * wl.d if wl.blocks & synth.BLK_LSH_DIN else 0.0
     f["bea"] = 2.0 * wl.n_bridge * wl.d if wl.blocks & synth.BLK_BEA else 0.0
     widths = [k1] + list(wl.hidden)
     for i in range(len(wl.hidden)):
@@ -69,15 +72,15 @@ def flops_per_candidate(wl: synth.Workload) -> dict:
     return f
 
 
-def kernel_flops(name: str, wl: synth.Workload, n: int) -> float:
-    f = flops_per_candidate(wl)
+def kernel_flops(name: str, wl: synth.Workload, n: int, keys=None) -> float:
+    f = flops_per_candidate(wl, keys)
     if name in ("score_simt", "score_fused"):
         return f["total"] * n
     if name == "interact":
         return (f["attention"] + f["lsh_din"] + f["bea"]) * n
     if name == "lsh":          # eq. 8's contraction; the match counts of eqs. 6-7 ride in the same kernel (see lsh_note)
         return f["lsh_din"] * n
-    if name == "buckets":
+    if name in ("buckets", "group"):
         return 0.0
     return f.get(name, 0.0) * n
 
@@ -101,7 +104,7 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", uuid, f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                          "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
 
@@ -267,10 +270,16 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
                          max_batch_candidates=wl.R * wl.N if batch else wl.N)
     sampler = synth.IdSampler(wl)
     states, id_lists = [], []
+    key_sum = 0.0
     for r in range(n_states):
         rq = synth.make_request(wl, r)
         states.append(srv.precompute(r, srv.upload_request(rq, B.USER_PROJECTED)))
         id_lists.append(sampler.request_ids(r))
+        if wl.n_categories:   # sequence items each candidate meets: the length of its category's sub-sequence
+            lens = np.bincount(rq["seq_cat"], minlength=wl.n_categories)
+            cats = np.array([srv.ctx.lib.aif_category(int(i), wl.n_categories, wl.bucket_mode) for i in id_lists[-1]])
+            key_sum += float(lens[cats].sum())
+    keys = key_sum / sum(len(x) for x in id_lists) if wl.n_categories else None
     torch.cuda.synchronize()
     if batch:
         offs = np.zeros(wl.R + 1, dtype=np.int64)
@@ -299,12 +308,15 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
         torch.cuda.synchronize()
         return [a.elapsed_time(b) for a, b in ev]
 
+    # the clock sampler starts before the warm-up so that it is running when the timed region begins; it stops after the
+    # latency pass
+    uuid = str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
+    sampler_proc = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    time.sleep(0.4)
     for i in range(max(3, warmup)):
         flush.zero_()
         step(i)
     torch.cuda.synchronize()
-    uuid = str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
-    sampler_proc = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
@@ -438,7 +450,7 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
     gather["traffic"] = None if gt is None else int(gt[1] * (gd if gt[0] == "per_candidate" else 1))
     top = max(kavg, key=kavg.get)
     tensor = bool(srv.ctx.get_stats().tensor_path) and top != "interact"
-    kf = kernel_flops(top, wl, cands)
+    kf = kernel_flops(top, wl, cands, keys)
     if tensor:
         peak = float(peaks["bf16_tflops"])
         roof = {"bound": "tensor", "kernel": top, "achieved": kf / (kavg[top] * 1e-3) / 1e12, "peak": peak,
@@ -469,14 +481,15 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
                    "L": wl.L, "F": wl.F, "hidden": list(wl.hidden), "mini_batch": wl.mini_batch,
                    "l2": "flushed between timed steps (256 MiB memset)", "parallelism": "replicas only" if world > 1 else "1 GPU",
                    "path": "tensor" if srv.ctx.get_stats().tensor_path else "cuda-core",
-                   "request_pool": pool},
+                   "request_pool": pool, "n_categories": wl.n_categories,
+                   "mean_keys_per_candidate": keys if keys is not None else wl.L},
         "p50_ms_per_request": float(np.percentile(per_request_ms, 50)),
         "p99_ms_per_request": float(np.percentile(per_request_ms, 99)),
         "latency_samples": {"scoring_calls": len(lat_times), "requests_per_call": wl.R if batch else 1},
-        "flops_per_candidate": flops_per_candidate(wl)["total"],
-        "step_tflops": flops_per_candidate(wl)["total"] * cands * steps / (total_ms * 1e-3) / 1e12,
-        "step_frac": {"of_measured_peak": flops_per_candidate(wl)["total"] * cands * steps / (total_ms * 1e-3) / 1e12 / float(peaks["bf16_tflops"]),
-                      "of_nominal_peak": flops_per_candidate(wl)["total"] * cands * steps / (total_ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS}
+        "flops_per_candidate": flops_per_candidate(wl, keys)["total"],
+        "step_tflops": flops_per_candidate(wl, keys)["total"] * cands * steps / (total_ms * 1e-3) / 1e12,
+        "step_frac": {"of_measured_peak": flops_per_candidate(wl, keys)["total"] * cands * steps / (total_ms * 1e-3) / 1e12 / float(peaks["bf16_tflops"]),
+                      "of_nominal_peak": flops_per_candidate(wl, keys)["total"] * cands * steps / (total_ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS}
         if wl.dtype == "bf16" else None,
         "e2e": {"value": world * cands * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * cands,
                 "d2h_bytes_per_step": 4 * cands, "steps": e2e_steps},
@@ -503,7 +516,7 @@ def main():
     ap.add_argument("--workload", default="c2", choices=sorted(synth.SHORT))
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--also", default="c3,c4,c4_lsh,c4_both,c5", help="other workloads measured briefly after the main one ('' = none)")
+    ap.add_argument("--also", default="c3,c4,c4_lsh,c4_both,long_lsh,long_sim,c5", help="other workloads measured briefly after the main one ('' = none)")
     # scaled copies of a workload, for profiler captures that must stay small (the defaults are the full sizes)
     ap.add_argument("--latency-calls", type=int, default=-1, help="scoring calls of the latency pass (default: 1000, fewer for long steps)")
     ap.add_argument("--requests", type=int, default=0, help="override the number of requests per step")

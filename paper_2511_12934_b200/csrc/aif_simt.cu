@@ -114,9 +114,53 @@ cudaError_t launch_scatter_rows(const aif_ctx *ctx, const int32_t *ids, int64_t 
     return e;
 }
 
+// The same for rows of VPR 16-byte vectors with VPR a divisor of 32 (128 to 512 bytes: every benchmark shape).  A warp
+// takes 8 x (32 / VPR) consecutive output rows per step: their ids arrive with one coalesced load and are handed round by
+// shuffles, every lane then has eight independent 16-byte loads in flight, each instruction covering whole rows, and no
+// division or second dependent load stands between a lane and its data.
+template <int VPR>
+__global__ void __launch_bounds__(256) k_gather_rows_w(const uint4 *__restrict__ table, const int32_t *__restrict__ ids, int64_t n, int64_t M,
+                                                       uint4 *__restrict__ out, uint32_t *status)
+{
+    constexpr int RPI = 32 / VPR, RPS = 8 * RPI;   // rows per instruction, rows per step of a warp
+    const int lane = threadIdx.x & 31, sub = lane / VPR, c = lane % VPR;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5, n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t r0 = warp * RPS; r0 < n; r0 += n_warps * RPS) {
+        int my = -1;
+        if (lane < RPS && r0 + lane < n) {
+            my = ids[r0 + lane];
+            if (my < 0 || (int64_t)my >= M) {
+                my = -1;
+                atomicOr(status, AIF_STATUS_BAD_ID);
+            }
+        }
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int src = __shfl_sync(0xffffffffu, my, u * RPI + sub);
+            v[u] = src >= 0 ? __ldg(table + (int64_t)src * VPR + c) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int64_t r = r0 + u * RPI + sub;
+            if (r < n) out[r * VPR + c] = v[u];
+        }
+    }
+}
+
 cudaError_t launch_gather_rows(const aif_ctx *ctx, const int32_t *ids, int64_t n, void *out, cudaStream_t st)
 {
     const int vpr = (int)((size_t)ctx->cfg.d * ctx->el / 16);
+    if (vpr == 8 || vpr == 16 || vpr == 32) {
+        const int rps = 8 * (32 / vpr);
+        const int64_t warps = (n + rps - 1) / rps;
+        const int grid = (int)((warps + 7) / 8 < 148 * 16 ? (warps + 7) / 8 : 148 * 16);
+        if (vpr == 8) k_gather_rows_w<8><<<grid, 256, 0, st>>>((const uint4 *)ctx->E, ids, n, ctx->cfg.M, (uint4 *)out, ctx->status);
+        else if (vpr == 16) k_gather_rows_w<16><<<grid, 256, 0, st>>>((const uint4 *)ctx->E, ids, n, ctx->cfg.M, (uint4 *)out, ctx->status);
+        else k_gather_rows_w<32><<<grid, 256, 0, st>>>((const uint4 *)ctx->E, ids, n, ctx->cfg.M, (uint4 *)out, ctx->status);
+        count_launch();
+        return cudaGetLastError();
+    }
     const int64_t total = n * vpr;
     const int grid = grid_for((total + 3) / 4, 256, 148 * 16);
     k_gather_rows<<<grid, 256, 0, st>>>((const uint4 *)ctx->E, ids, n, vpr, ctx->cfg.M, (uint4 *)out, ctx->status);

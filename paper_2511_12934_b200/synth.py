@@ -115,9 +115,13 @@ C5_MIXED = C5.with_(name="c5_wide_mixed", N=10_000, mixed_sizes=(1000, 10_000))
 C4_LSH = C4.with_(name="c4_long_sequence_lsh", blocks=BLK_CROSS | BLK_LSH_DIN | BLK_SIMTIER)
 C4_BOTH = C4.with_(name="c4_long_sequence_att_lsh", blocks=BLK_ATT | BLK_CROSS | BLK_LSH_DIN | BLK_SIMTIER)
 C4_DIN = C4.with_(name="c4_long_sequence_lsh_din", blocks=BLK_CROSS | BLK_LSH_DIN)
-CONFIGS = {w.name: w for w in (C1, C2, C3, C4, C5, C5_MIXED, C4_LSH, C4_BOTH, C4_DIN)}
+# the long-term sequence of Sections 3.3 / 4.2 (length ~10^5): LSH blocks over the whole sequence, and attention + LSH blocks
+# over the candidate's category's sub-sequence (100 categories, SIM-hard)
+LONG_LSH = C4.with_(name="long_1e5_lsh", R=4, L=100_000, blocks=BLK_CROSS | BLK_LSH_DIN | BLK_SIMTIER)
+LONG_SIM = C4.with_(name="long_1e5_sim", R=4, L=100_000, blocks=BLK_ATT | BLK_CROSS | BLK_LSH_DIN | BLK_SIMTIER, n_categories=100)
+CONFIGS = {w.name: w for w in (C1, C2, C3, C4, C5, C5_MIXED, C4_LSH, C4_BOTH, C4_DIN, LONG_LSH, LONG_SIM)}
 SHORT = {"c1": C1, "c2": C2, "c3": C3, "c4": C4, "c5": C5, "c5a": C5, "c5b": C5_MIXED, "c4_lsh": C4_LSH, "c4_both": C4_BOTH,
-         "c4_din": C4_DIN}
+         "c4_din": C4_DIN, "long_lsh": LONG_LSH, "long_sim": LONG_SIM}
 
 
 def _seed(*keys) -> np.random.Generator:
