@@ -245,12 +245,56 @@ def run_ours(args, wl):
                                               "latency_samples", "flops_per_candidate", "config", "roofline", "step_tflops",
                                               "step_frac", "e2e")}
         line["other_workloads"] = others
+    if rank == 0 and world == 1 and args.bea_sweep and wl.dtype == "bf16":
+        line["bea_bridge_sweep"] = bea_sweep(wl)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def bea_sweep(base: synth.Workload, bridges=(1, 2, 4, 8, 16), m_features=64, steps=30):
+    """Cost of Bridge Embedding Approximation over the number of bridges n (Algorithm 1; Section 5.2.2 studies quality over
+    n, this is the cost side): the user-side call that computes W = Softmax(B U^T / sqrt(d)) and V from m_features user
+    feature embeddings, and the scoring step with the BEA block on (v = w_hat V per candidate, d more input columns)."""
+    import torch
+    from paper_2511_12934_b200 import binding as B
+    from paper_2511_12934_b200 import serving
+    out = []
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for n in bridges:
+        wl = base.with_(name=f"{base.name}_bea{n}", M=min(base.M, 200_000), blocks=base.blocks | synth.BLK_BEA, n_bridge=n)
+        weights, table = synth.make_weights(wl), synth.make_item_table(wl)
+        srv = serving.Server(wl, weights, table, max_user_states=2, max_batch_candidates=wl.N)
+        rq = synth.make_request(wl, 0)
+        rq = dict(rq, bea_U=synth.normal_rows(m_features, wl.d, 1.0, wl.dtype, 77, n))
+        del rq["V"]
+        dev = srv.upload_request(rq, B.USER_PROJECTED)
+        ids = torch.from_numpy(synth.IdSampler(wl).request_ids(0)).cuda()
+        logits = torch.empty(wl.N, dtype=torch.float32, device="cuda")
+        st = srv.precompute(0, dev)
+        torch.cuda.synchronize()
+        pre, sc = [], []
+        for i in range(steps):
+            a, b, c, d = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+            st.release()
+            a.record(srv.side)
+            st = srv.precompute(1 + i, dev)
+            b.record(srv.side)
+            torch.cuda.synchronize()
+            flush.zero_()
+            c.record()
+            srv.ctx.score(st, ids, logits)
+            d.record()
+            torch.cuda.synchronize()
+            pre.append(a.elapsed_time(b)), sc.append(c.elapsed_time(d))
+        out.append({"n_bridge": n, "user_side_ms": float(np.median(pre[3:])), "score_ms": float(np.median(sc[3:])),
+                    "candidates": wl.N, "m_features": m_features})
+        srv.close()
+        del srv
+    return out
 
 
 def measure(args, wl, steps, warmup, dist, world, rank, full):
@@ -393,7 +437,7 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
 
     # the user-side call (eqs. 1-3 from raw embeddings + pre-cache + p_u) on the side stream: the time a retrieval phase has
     # to cover; one extra arena slot is not available, so a state of the pool is recomputed in place of itself
-    pre_ms = None
+    pre_ms, overlap = None, None
     if full:
         states[-1].release()
         dev_raw = srv.upload_request(synth.make_request(wl, n_states - 1), B.USER_RAW)
@@ -407,8 +451,42 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
             ts.append(a.elapsed_time(b))
             if i < 5:
                 stx.release()
-        states[-1] = stx
         pre_ms = float(np.median(ts[1:]))
+        # Overlap with a simulated retrieval phase (Section 3.1: the user side runs while the candidates are retrieved): the
+        # main stream is busy for `retrieval_ms` (a spin kernel standing in for the retrieval service), the user-side call
+        # runs on the side stream from the same starting point, scoring follows on the main stream and waits for both.  All
+        # times from events: the request takes retrieval + scoring, not retrieval + precompute + scoring.
+        stx.release()
+        hz = 1e3 * torch.cuda.get_device_properties(torch.cuda.current_device()).clock_rate   # kHz -> Hz
+        retrieval_cycles = int(max(3.0 * pre_ms, 0.3) * 1e-3 * hz)
+        ids_o = ids_dev[0] if batch else ids_dev[(n_states - 1) % pool]
+        main = torch.cuda.current_stream()
+        rows = []
+        for i in range(8):
+            e0, e_ret, e_end = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            flush.zero_()
+            e0.record(main)
+            srv.side.wait_event(e0)
+            torch.cuda._sleep(retrieval_cycles)
+            e_ret.record(main)
+            s0.record(srv.side)
+            stx = srv.precompute(20_000 + i, dev_raw)
+            s1.record(srv.side)
+            if batch:
+                srv.ctx.score_batch(states[:-1] + [stx], ids_o, offs, logits)
+            else:
+                srv.ctx.score(stx, ids_o, logits)
+            e_end.record(main)
+            torch.cuda.synchronize()
+            rows.append((e0.elapsed_time(e_ret), e0.elapsed_time(s1), e_ret.elapsed_time(e_end), e0.elapsed_time(e_end)))
+            if i < 7:
+                stx.release()
+        states[-1] = stx
+        r = np.median(np.array(rows[1:]), axis=0)
+        overlap = {"retrieval_ms": float(r[0]), "precompute_done_ms_after_start": float(r[1]), "scoring_ms_after_retrieval": float(r[2]),
+                   "request_ms": float(r[3]), "sum_if_serial_ms": float(r[0] + pre_ms + r[2]),
+                   "hidden": bool(r[1] <= r[0]), "note": "medians of 7 runs; retrieval = a spin kernel on the main stream"}
 
     # the item side of the nearline pipeline as a compute call (eq. 4 tower; bridge weights and signatures when their
     # blocks are on): 2^19 synthetic items with dI = 4 d, hI = 2 d written into the table rows they will be gathered from
@@ -498,7 +576,7 @@ def measure(args, wl, steps, warmup, dist, world, rank, full):
         "roofline": roof,
         "gather_stage": gather,
         "nearline_item_side": nearline,
-        "user_precompute": {"ms": pre_ms, "inputs": "raw embeddings (eqs. 1-3 computed)", "L": wl.L, "stream": "side"},
+        "user_precompute": {"ms": pre_ms, "inputs": "raw embeddings (eqs. 1-3 computed)", "L": wl.L, "stream": "side", "overlap": overlap},
         "replica_plan": plan,
     }
     srv.close()
@@ -516,6 +594,7 @@ def main():
     ap.add_argument("--workload", default="c2", choices=sorted(synth.SHORT))
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-bea-sweep", dest="bea_sweep", action="store_false", help="skip the cost table over the number of BEA bridges")
     ap.add_argument("--also", default="c3,c4,c4_lsh,c4_both,long_lsh,long_sim,c5", help="other workloads measured briefly after the main one ('' = none)")
     # scaled copies of a workload, for profiler captures that must stay small (the defaults are the full sizes)
     ap.add_argument("--latency-calls", type=int, default=-1, help="scoring calls of the latency pass (default: 1000, fewer for long steps)")
