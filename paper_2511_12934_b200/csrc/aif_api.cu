@@ -241,6 +241,10 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     TRY(dev_alloc(ctx, &ctx->Wseq_t, (size_t)c.dU * c.d * el, true));
     TRY(dev_alloc(ctx, &ctx->Wa_t, (size_t)c.d * c.d * el, true));
     TRY(dev_alloc(ctx, &ctx->Wb_t, (size_t)c.d * c.d * el, true));
+    TRY(dev_alloc(ctx, &ctx->Wseq_k, (size_t)c.dU * c.d * el, true));
+    TRY(dev_alloc(ctx, &ctx->Wa_k, (size_t)c.d * c.d * el, true));
+    TRY(dev_alloc(ctx, (void **)&ctx->zero_bias, 256 * 4, true));
+    if (ctx->tensor_path) TRY(dev_alloc(ctx, &ctx->ffn_rows, ((size_t)c.L_max + 128) * c.d * 2, true));
     TRY(dev_alloc(ctx, (void **)&ctx->b_a, (size_t)c.d * 4, true));
     TRY(dev_alloc(ctx, (void **)&ctx->b_b, (size_t)c.d * 4, true));
 
@@ -377,6 +381,8 @@ int aif_load_weights(aif_ctx *ctx, const aif_weights *w, aif_stream stream)
         AIF_CUDA(launch_transpose(w->W_profile, ctx->Wprofile_t, c.d, c.dU, el, st));
         AIF_CUDA(launch_transpose(w->W_seq, ctx->Wseq_t, c.d, c.dU, el, st));
         AIF_CUDA(launch_transpose(w->W_a, ctx->Wa_t, c.d, c.d, el, st));
+        AIF_CUDA(cudaMemcpyAsync(ctx->Wseq_k, w->W_seq, (size_t)c.d * c.dU * el, cudaMemcpyDeviceToDevice, st));
+        AIF_CUDA(cudaMemcpyAsync(ctx->Wa_k, w->W_a, (size_t)c.d * c.d * el, cudaMemcpyDeviceToDevice, st));
         AIF_CUDA(launch_transpose(w->W_b, ctx->Wb_t, c.d, c.d, el, st));
         AIF_CUDA(cudaMemcpyAsync(ctx->b_a, w->b_a, (size_t)c.d * 4, cudaMemcpyDeviceToDevice, st));
         AIF_CUDA(cudaMemcpyAsync(ctx->b_b, w->b_b, (size_t)c.d * 4, cudaMemcpyDeviceToDevice, st));

@@ -160,6 +160,9 @@ struct aif_ctx {
     void *w_out = nullptr;
     float *b_out = nullptr;
     void *Wprofile_t = nullptr, *Wseq_t = nullptr, *Wa_t = nullptr, *Wb_t = nullptr;
+    void *Wseq_k = nullptr, *Wa_k = nullptr;   // W_seq [d x dU], W_a [d x d] as given (K-major): operands of the tensor-core user side
+    float *zero_bias = nullptr;                // [256] zeros
+    void *ffn_rows = nullptr;                  // [L_max + 128][d] bf16: hidden FFN activations of the user state being computed
     float *b_a = nullptr, *b_b = nullptr;
     bool user_weights = false;
     void *bridges = nullptr, *W_f = nullptr;   // user side of Algorithm 1: B [n_bridge x d], W_f [d x d]

@@ -628,6 +628,23 @@ __global__ void __launch_bounds__(256) k_user_finish(int raw, const T *__restric
 
 __global__ void k_set_slot_len(SlotDev *slots, int index, int L) { slots[index].L = L; }
 
+// partial[g][k] = sum over rows g, g + n_parts, ... of rows[i][k] (bf16 rows, fp32 sums in a fixed order): the mean pooling of
+// eq. 2 over hidden FFN activations that a tensor-core layer has written
+__global__ void __launch_bounds__(256) k_pool_rows(const __nv_bfloat16 *__restrict__ rows, int L, int d, int n_parts, float *__restrict__ partial)
+{
+    const int lane = threadIdx.x & 31, g = blockIdx.x * 8 + (threadIdx.x >> 5), dq = d >> 5;
+    if (g >= n_parts) return;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int i = g; i < L; i += n_parts) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+            if (c < dq) acc[c] += __bfloat162float(rows[(size_t)i * d + lane + 32 * c]);
+    }
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+        if (c < dq) partial[(size_t)g * d + lane + 32 * c] = acc[c];
+}
+
 template <typename T>
 static cudaError_t user_network_typed(const aif_ctx *ctx, HostSlot &hs, int slot_index, const aif_user_inputs *in, int L,
                                       cudaStream_t st)
@@ -637,7 +654,21 @@ static cudaError_t user_network_typed(const aif_ctx *ctx, HostSlot &hs, int slot
     cudaError_t e;
     T *S = (T *)hs.dev.S;
     const bool raw = in->mode == AIF_USER_RAW;
-    if (raw) {
+    // Long sequences on bf16 tensor-core contexts: eq. 1's sequence projection and the first FFN layer of eq. 2 are dense
+    // layers over L rows and run through the scoring MLP's layer kernel (tcgen05); shorter ones stay on the CUDA cores,
+    // where a launch of this size is latency, not throughput.
+    const bool tc_user = raw && std::is_same<T, __nv_bfloat16>::value && ctx->tensor_path && ctx->tc_att_plan && L >= 1024 &&
+                         c.dU % 64 == 0 && d % 64 == 0;
+    if (raw && tc_user) {
+        DenseLayer lay{};
+        lay.A = in->seq, lay.W = ctx->Wseq_k, lay.bias = ctx->zero_bias, lay.out = S, lay.in_w = c.dU, lay.H = d, lay.relu = 0, lay.sign_bits = 0;
+        if ((e = tc_dense_layer(ctx, lay, L, st)) != cudaSuccess) return e;
+        // the profile row alone (block index L of the projection kernel, launched with no sequence rows)
+        k_user_project<T><<<1, 128, c.dU * sizeof(float), st>>>((const T *)in->seq, (const T *)in->profile, (const T *)ctx->Wseq_t,
+                                                                 (const T *)ctx->Wprofile_t, 0, c.dU, d, S, hs.prof_hat);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    } else if (raw) {
         k_user_project<T><<<L + 1, 128, c.dU * sizeof(float), st>>>((const T *)in->seq, (const T *)in->profile,
                                                                     (const T *)ctx->Wseq_t, (const T *)ctx->Wprofile_t, L,
                                                                     c.dU, d, S, hs.prof_hat);
@@ -670,9 +701,18 @@ static cudaError_t user_network_typed(const aif_ctx *ctx, HostSlot &hs, int slot
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         const int n_warps = kUserPartials;
-        k_user_self<T><<<n_warps / 8, 256, 8 * 3 * d * sizeof(float), st>>>(S, L, d, (const T *)ctx->Wa_t, ctx->b_a,
-                                                                            (const T *)ctx->Wb_t, ctx->b_b, hs.partial,
-                                                                            n_warps, att_rows);
+        if (tc_user && att_rows) {
+            // hidden = ReLU(attention rows W_a^T + b_a) as a dense layer, then the pooling sums (the second FFN layer is
+            // linear and is applied once to the pooled row, in k_user_finish)
+            DenseLayer lay{};
+            lay.A = att_rows, lay.W = ctx->Wa_k, lay.bias = ctx->b_a, lay.out = ctx->ffn_rows, lay.in_w = d, lay.H = d, lay.relu = 1, lay.sign_bits = 0;
+            if ((e = tc_dense_layer(ctx, lay, L, st)) != cudaSuccess) return e;
+            k_pool_rows<<<n_warps / 8, 256, 0, st>>>((const __nv_bfloat16 *)ctx->ffn_rows, L, d, n_warps, hs.partial);
+        } else {
+            k_user_self<T><<<n_warps / 8, 256, 8 * 3 * d * sizeof(float), st>>>(S, L, d, (const T *)ctx->Wa_t, ctx->b_a,
+                                                                                (const T *)ctx->Wb_t, ctx->b_b, hs.partial,
+                                                                                n_warps, att_rows);
+        }
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }

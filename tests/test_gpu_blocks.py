@@ -140,7 +140,7 @@ def test_long_sequence_shape_at_full_size_with_the_lsh_blocks(blocks):
     srv.close()
 
 
-@pytest.mark.parametrize("base,L", [("c4", 10_000), ("c5", 500), ("c2", 1000)])
+@pytest.mark.parametrize("base,L", [("c4", 10_000), ("c5", 500), ("c5", 1100), ("c2", 1000), ("c2", 1024)])
 def test_raw_user_precompute_at_long_sequences(base, L):
     """eqs. 1-3 from raw embeddings at the lengths where the tuned path is live: the self-attention rows come from the
     tensor-core attention kernel over many tiles, eq. 3 is merged from 256 key slices.  u, p_u and every row of the
