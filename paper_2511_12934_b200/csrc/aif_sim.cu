@@ -147,52 +147,81 @@ __global__ void __launch_bounds__(256) k_sim_count(ScoreLaunch sl, int64_t M, in
     }
 }
 
-// One block over the groups: first grouped position and first tile of every group (exclusive scans of the counts and of
-// the tile counts), the tile records, the number of tiles; the counts are turned into cursors (zero) for the placement.
+// One block over the groups: first grouped position of every group (exclusive scan of the counts), the tile records, the
+// number of tiles; the counts are turned into cursors (zero) for the placement.  Tiles are laid out by the size of their
+// sub-sequence, longest first (in classes of powers of two): a tile's cost is its number of key blocks, the kernels hand
+// tile t to CTA t mod grid, and a long tile that started late would be what everything else waits for.
 __global__ void __launch_bounds__(1024) k_sim_tiles(ScoreLaunch sl, int n_groups, int n_cat, int32_t *__restrict__ grp_cnt,
                                                     int32_t *__restrict__ grp_start, TileDev *__restrict__ tiles, int tile_cap,
                                                     int32_t *__restrict__ n_tiles_out)
 {
-    __shared__ int32_t part_c[1024], part_t[1024];
-    __shared__ int32_t carry_c, carry_t;
-    if (threadIdx.x == 0) carry_c = 0, carry_t = 0;
+    constexpr int kClasses = 32;
+    __shared__ int32_t part_c[1024];
+    __shared__ int32_t carry_c;
+    __shared__ int32_t cls_tiles[kClasses], cls_base[kClasses];
+    if (threadIdx.x == 0) carry_c = 0;
+    if (threadIdx.x < kClasses) cls_tiles[threadIdx.x] = 0;
     __syncthreads();
+    auto group_info = [&](int g, int &slot, int &len, int &key0) {
+        const int r = g / n_cat, c = g - r * n_cat;
+        slot = sl.reqs ? sl.reqs[r].slot : sl.single.slot;
+        const SlotDev *sd = sl.slots + slot;
+        len = sd->cat_len[c], key0 = sd->cat_off[c];
+    };
+    auto class_of = [](int len) { return len > 0 ? 32 - __clz(len) : 0; };   // 0: empty sub-sequence, else floor(log2) + 1
+    // pass 1: grouped positions (scan of the counts) and tiles per size class
     for (int g0 = 0; g0 < n_groups; g0 += 1024) {
         const int g = g0 + threadIdx.x;
         const int cnt = g < n_groups ? grp_cnt[g] : 0;
-        const int nt = (cnt + kTcTile - 1) / kTcTile;
-        part_c[threadIdx.x] = cnt, part_t[threadIdx.x] = nt;
+        part_c[threadIdx.x] = cnt;
         __syncthreads();
         for (int o = 1; o < 1024; o <<= 1) {
             const int ac = (int)threadIdx.x >= o ? part_c[threadIdx.x - o] : 0;
-            const int at = (int)threadIdx.x >= o ? part_t[threadIdx.x - o] : 0;
             __syncthreads();
-            part_c[threadIdx.x] += ac, part_t[threadIdx.x] += at;
+            part_c[threadIdx.x] += ac;
             __syncthreads();
         }
         if (g < n_groups) {
-            const int start = carry_c + part_c[threadIdx.x] - cnt, t0 = carry_t + part_t[threadIdx.x] - nt;
-            grp_start[g] = start;
-            grp_cnt[g] = 0;   // from here on the group's placement cursor
+            grp_start[g] = carry_c + part_c[threadIdx.x] - cnt;
             if (cnt > 0) {
-                const int r = g / n_cat, c = g - r * n_cat;
-                const int slot = sl.reqs ? sl.reqs[r].slot : sl.single.slot;
-                const SlotDev *sd = sl.slots + slot;
-                const int len = sd->cat_len[c], key0 = sd->cat_off[c];
-                for (int i = 0; i < nt; ++i) {
-                    if (t0 + i >= tile_cap) break;   // cannot happen for a launch within the context's limits (sim_prepare)
-                    TileDev t;
-                    t.slot = slot, t.cnt = min(kTcTile, cnt - i * kTcTile), t.pos0 = (int64_t)start + (int64_t)i * kTcTile;
-                    t.L = len, t.key0 = key0, t.pad_[0] = t.pad_[1] = 0;
-                    tiles[t0 + i] = t;
-                }
+                int slot, len, key0;
+                group_info(g, slot, len, key0);
+                atomicAdd(&cls_tiles[class_of(len)], (cnt + kTcTile - 1) / kTcTile);
             }
         }
         __syncthreads();
-        if (threadIdx.x == 1023) carry_c += part_c[1023], carry_t += part_t[1023];
+        if (threadIdx.x == 1023) carry_c += part_c[1023];
         __syncthreads();
     }
-    if (threadIdx.x == 0) *n_tiles_out = min(carry_t, tile_cap);
+    // first tile of every class, longest sub-sequences first
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int k = kClasses - 1; k >= 0; --k) {
+            cls_base[k] = run;
+            run += cls_tiles[k];
+            cls_tiles[k] = 0;   // from here on the class's cursor
+        }
+        *n_tiles_out = min(run, tile_cap);
+    }
+    __syncthreads();
+    // pass 2: the tile records; the counts become the placement cursors
+    for (int g = threadIdx.x; g < n_groups; g += 1024) {
+        const int cnt = grp_cnt[g];
+        grp_cnt[g] = 0;
+        if (cnt == 0) continue;
+        int slot, len, key0;
+        group_info(g, slot, len, key0);
+        const int nt = (cnt + kTcTile - 1) / kTcTile, k = class_of(len);
+        const int t0 = cls_base[k] + atomicAdd(&cls_tiles[k], nt);
+        const int start = grp_start[g];
+        for (int i = 0; i < nt; ++i) {
+            if (t0 + i >= tile_cap) break;   // cannot happen for a launch within the context's limits (sim_prepare)
+            TileDev t;
+            t.slot = slot, t.cnt = min(kTcTile, cnt - i * kTcTile), t.pos0 = (int64_t)start + (int64_t)i * kTcTile;
+            t.L = len, t.key0 = key0, t.pad_[0] = t.pad_[1] = 0;
+            tiles[t0 + i] = t;
+        }
+    }
 }
 
 // grouped ids and, for every grouped position, where its logit belongs
