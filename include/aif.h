@@ -108,6 +108,12 @@ typedef struct {
                                       (Section 3.3, SIM-hard: <user, category, sub-sequence>), see aif_category.  Needs
                                       the tensor-core kernels (AIF_ERR_SHAPE otherwise); mini_batch is then ignored
                                       (scores do not depend on it) */
+    int32_t versioned_table;       /* 1: the item table (and its sidecars) exists twice.  A full refresh (ids == NULL) is
+                                      written into the copy that is not being read and published as a whole: scoring
+                                      calls made before the refresh call keep reading the old copy, calls made after it
+                                      wait for the refresh and read the new one; no call ever sees a half-written table
+                                      (Section 3.4: full updates of the index table under serving).  Costs the table's
+                                      memory a second time.  0: one copy, the caller orders refreshes against scoring */
     int64_t max_batch_candidates;  /* upper bound of the candidates of one aif_score / aif_score_batch call;
                                       sizes the context's scratch memory */
 } aif_config;
@@ -192,7 +198,12 @@ int aif_load_weights(aif_ctx *ctx, const aif_weights *w, aif_stream stream);
  * table row ids[i]; an id outside [0, M) is skipped and sets AIF_STATUS_BAD_ID.  Duplicate ids in one call
  * leave either row.  ids: device int32 [n].  rows: device [n x d] storage type.  bea_w: device [n x n_bridge]
  * storage type, lsh_sig: device [n x lsh_bits/8]; required iff their blocks are on.  Bumps table_version.
- * The caller orders the call against scoring (same stream, or an event). */
+ * The caller orders the call against scoring (same stream, or an event).
+ * With versioned_table a full refresh needs no such ordering: it fills the spare copy (rows beyond n are carried over
+ * from the live one) on `stream` and becomes the live copy for every scoring call made after this call returns; those
+ * calls wait on the device for the refresh to finish.  The copy it overwrites is the one that was live before the
+ * previous full refresh: scoring calls made before that previous refresh must have finished by now.  Incremental
+ * refreshes write into the live copy and are ordered by the caller as before. */
 int aif_item_nearline_refresh(aif_ctx *ctx, const int32_t *ids, int64_t n, const void *rows, const void *bea_w,
                               const uint8_t *lsh_sig, aif_stream stream);
 

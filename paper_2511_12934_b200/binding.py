@@ -41,7 +41,7 @@ class aif_config(C.Structure):
         ("hidden", C.c_int32 * 4), ("bucket_mode", C.c_int32), ("blocks", C.c_int32), ("n_bridge", C.c_int32),
         ("lsh_bits", C.c_int32), ("n_tiers", C.c_int32), ("lsh_din_norm", C.c_int32), ("simtier_norm", C.c_int32),
         ("emit_sigmoid", C.c_int32), ("max_user_states", C.c_int32), ("mini_batch", C.c_int32), ("path", C.c_int32),
-        ("n_categories", C.c_int32), ("max_batch_candidates", C.c_int64),
+        ("n_categories", C.c_int32), ("versioned_table", C.c_int32), ("max_batch_candidates", C.c_int64),
     ]
 
 
@@ -178,11 +178,11 @@ def _stream(s) -> C.c_void_p:
 def make_config(*, dtype, M, d, L_max, hidden: Sequence[int], F=0, B=1, dc=0, dU=0, bucket_mode=BUCKET_HASH,
                 blocks=BLK_ATT | BLK_CROSS, n_bridge=8, lsh_bits=0, n_tiers=8, lsh_din_norm=NORM_MEAN,
                 simtier_norm=NORM_MEAN, emit_sigmoid=0, max_user_states=4, mini_batch=0, path=PATH_AUTO,
-                max_batch_candidates=16384, n_categories=0) -> aif_config:
+                max_batch_candidates=16384, n_categories=0, versioned_table=0) -> aif_config:
     h = list(hidden) + [0] * (4 - len(hidden))
     return aif_config(C.sizeof(aif_config), dtype, M, d, dU or d, L_max, F, B, dc, len(hidden), (C.c_int32 * 4)(*h),
                       bucket_mode, blocks, n_bridge, lsh_bits or d, n_tiers, lsh_din_norm, simtier_norm,
-                      emit_sigmoid, max_user_states, mini_batch, path, n_categories, max_batch_candidates)
+                      emit_sigmoid, max_user_states, mini_batch, path, n_categories, versioned_table, max_batch_candidates)
 
 
 class UserState:

@@ -66,6 +66,7 @@ int check_config(const aif_config *c)
     if (c->max_user_states < 1 || c->mini_batch < 0 || c->max_batch_candidates < 1) return AIF_ERR_SHAPE;
     if (c->path < AIF_PATH_AUTO || c->path > AIF_PATH_TENSOR) return AIF_ERR_ARG;
     if (c->n_categories < 0 || c->n_categories > 4096) return AIF_ERR_SHAPE;
+    if (c->versioned_table != 0 && c->versioned_table != 1) return AIF_ERR_ARG;
     if (c->n_categories > 0 && c->bucket_mode != AIF_BUCKET_MOD && c->bucket_mode != AIF_BUCKET_HASH) return AIF_ERR_ARG;
     return AIF_OK;
 }
@@ -111,6 +112,49 @@ int run_score(aif_ctx *ctx, const ScoreLaunch &sl, int64_t total, cudaStream_t s
 namespace aif {
 
 int check_user_state(aif_ctx *ctx, const aif_user_state *st) { return state_check(ctx, st); }
+
+cudaError_t wait_table_ready(const aif_ctx *ctx, cudaStream_t st)
+{
+    if (!ctx->table_ev_pending) return cudaSuccess;
+    const cudaError_t q = cudaEventQuery(ctx->table_ev);
+    if (q == cudaSuccess) {
+        ctx->table_ev_pending = false;
+        return cudaSuccess;
+    }
+    if (q != cudaErrorNotReady) return q;
+    (void)cudaGetLastError();
+    return cudaStreamWaitEvent(st, ctx->table_ev, 0);
+}
+
+// Versioned table, full refresh: the spare copy becomes the one every writer and (from now on) every reader addresses;
+// rows the refresh does not cover are carried over from the copy that was live.
+static cudaError_t begin_full_refresh(aif_ctx *ctx, int64_t n, cudaStream_t st)
+{
+    const aif_config &c = ctx->cfg;
+    // the copies are written on `st`: it must be behind the previous full refresh, whose copy is the source of the rows carried over
+    cudaError_t e = wait_table_ready(ctx, st);
+    if (e != cudaSuccess) return e;
+    std::swap(ctx->E, ctx->E_alt), std::swap(ctx->bea_w, ctx->bea_w_alt), std::swap(ctx->sig, ctx->sig_alt);
+    if (n < c.M) {
+        const size_t rest = (size_t)(c.M - n);
+        e = cudaMemcpyAsync((char *)ctx->E + (size_t)n * c.d * ctx->el, (const char *)ctx->E_alt + (size_t)n * c.d * ctx->el, rest * c.d * ctx->el,
+                            cudaMemcpyDeviceToDevice, st);
+        if (e == cudaSuccess && ctx->bea_w)
+            e = cudaMemcpyAsync((char *)ctx->bea_w + (size_t)n * c.n_bridge * ctx->el, (const char *)ctx->bea_w_alt + (size_t)n * c.n_bridge * ctx->el,
+                                rest * c.n_bridge * ctx->el, cudaMemcpyDeviceToDevice, st);
+        if (e == cudaSuccess && ctx->sig)
+            e = cudaMemcpyAsync(ctx->sig + (size_t)n * c.lsh_bits / 8, ctx->sig_alt + (size_t)n * c.lsh_bits / 8, rest * c.lsh_bits / 8,
+                                cudaMemcpyDeviceToDevice, st);
+    }
+    return e;
+}
+
+static cudaError_t end_full_refresh(aif_ctx *ctx, cudaStream_t st)
+{
+    const cudaError_t e = cudaEventRecord(ctx->table_ev, st);
+    ctx->table_ev_pending = e == cudaSuccess;
+    return e;
+}
 
 void set_last_error(const char *text) { snprintf(g_last_error, sizeof(g_last_error), "%s", text); }
 
@@ -226,6 +270,15 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     TRY(dev_alloc(ctx, &ctx->E, (size_t)c.M * c.d * el, true));
     if (c.blocks & AIF_BLK_BEA) TRY(dev_alloc(ctx, &ctx->bea_w, (size_t)c.M * c.n_bridge * el, true));
     if (c.blocks & (AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER)) TRY(dev_alloc(ctx, (void **)&ctx->sig, (size_t)c.M * c.lsh_bits / 8, true));
+    if (c.versioned_table) {
+        TRY(dev_alloc(ctx, &ctx->E_alt, (size_t)c.M * c.d * el, true));
+        if (ctx->bea_w) TRY(dev_alloc(ctx, &ctx->bea_w_alt, (size_t)c.M * c.n_bridge * el, true));
+        if (ctx->sig) TRY(dev_alloc(ctx, (void **)&ctx->sig_alt, (size_t)c.M * c.lsh_bits / 8, true));
+        if (cudaEventCreateWithFlags(&ctx->table_ev, cudaEventDisableTiming) != cudaSuccess) {
+            aif_destroy(ctx);
+            return cuda_fail(cudaGetLastError(), "cudaEventCreate");
+        }
+    }
     TRY(dev_alloc(ctx, (void **)&ctx->status, 256, true));
 
     // weights
@@ -343,6 +396,7 @@ int aif_destroy(aif_ctx *ctx)
     cudaDeviceSynchronize();
     for (auto &hs : ctx->slots)
         if (hs.ev) cudaEventDestroy(hs.ev);
+    if (ctx->table_ev) cudaEventDestroy(ctx->table_ev);
     for (int i = 0; i <= KernelTiming::kMax; ++i)
         if (ctx->timing.ev[i]) cudaEventDestroy(ctx->timing.ev[i]);
     for (int i = 0; i < PinnedRing::kSlots; ++i) {
@@ -415,7 +469,11 @@ int aif_item_nearline_refresh(aif_ctx *ctx, const int32_t *ids, int64_t n, const
     if (!ids && n > ctx->cfg.M) return AIF_ERR_SHAPE;
     if (n == 0) return AIF_OK;
     DeviceGuard g(ctx->device);
+    const bool versioned = ctx->cfg.versioned_table && !ids;
+    if (versioned) AIF_CUDA(begin_full_refresh(ctx, n, as_stream(stream)));
+    else AIF_CUDA(wait_table_ready(ctx, as_stream(stream)));
     AIF_CUDA(launch_scatter_rows(ctx, ids, n, rows, bea_w, lsh_sig, as_stream(stream)));
+    if (versioned) AIF_CUDA(end_full_refresh(ctx, as_stream(stream)));
     ctx->table_version += 1;
     ctx->stats.table_version = ctx->table_version;
     ctx->stats.refresh_calls += 1;
@@ -439,8 +497,12 @@ int aif_item_nearline_compute(aif_ctx *ctx, const int32_t *ids, int64_t n, const
     if (!ctx->nearline_plan) return AIF_ERR_NOT_READY;
     if (n == 0) return AIF_OK;
     DeviceGuard g(ctx->device);
+    const bool versioned = ctx->cfg.versioned_table && !ids;
+    if (versioned) AIF_CUDA(begin_full_refresh(ctx, n, as_stream(stream)));
+    else AIF_CUDA(wait_table_ready(ctx, as_stream(stream)));
     const int rc = nearline_compute(ctx, ids, n, I_raw, I_id, M_mm, as_stream(stream));
     if (rc != AIF_OK) return rc;
+    if (versioned) AIF_CUDA(end_full_refresh(ctx, as_stream(stream)));
     ctx->table_version += 1;
     ctx->stats.table_version = ctx->table_version;
     ctx->stats.refresh_calls += 1;
@@ -564,6 +626,7 @@ int aif_score(aif_ctx *ctx, const aif_user_state *state, const int32_t *cand_ids
     cudaStream_t st = as_stream(stream);
     const HostSlot &hs = ctx->slots[(size_t)state->index];
     AIF_CUDA(wait_user_ready(hs, st));
+    AIF_CUDA(wait_table_ready(ctx, st));
     ScoreLaunch sl{};
     sl.slots = ctx->slots_dev, sl.reqs = nullptr, sl.n_req = 1;
     sl.single = ReqDev{state->index, n, 0, 0, 0};
@@ -596,6 +659,7 @@ int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *st
     const int slot = ring.next;
     ring.next = (ring.next + 1) % PinnedRing::kSlots;
     if (ring.used[slot]) AIF_CUDA(cudaEventSynchronize(ring.ev[slot]));
+    AIF_CUDA(wait_table_ready(ctx, st));
     int tiles = 0, max_L = 0;
     for (int r = 0; r < n_req; ++r) {
         const int n = (int)(offsets[r + 1] - offsets[r]);
@@ -680,6 +744,7 @@ int aif_gather_rows(aif_ctx *ctx, const int32_t *ids, int64_t n, void *rows_out,
     if (n == 0) return AIF_OK;
     if (!ids || !rows_out) return AIF_ERR_ARG;
     DeviceGuard g(ctx->device);
+    AIF_CUDA(wait_table_ready(ctx, as_stream(stream)));
     AIF_CUDA(launch_gather_rows(ctx, ids, n, rows_out, as_stream(stream)));
     return AIF_OK;
 }
@@ -693,6 +758,7 @@ int aif_gather_sidecars(aif_ctx *ctx, const int32_t *ids, int64_t n, void *bea_w
     if (n == 0 || (!bea_w_out && !sig_out)) return AIF_OK;
     if (!ids) return AIF_ERR_ARG;
     DeviceGuard g(ctx->device);
+    AIF_CUDA(wait_table_ready(ctx, as_stream(stream)));
     AIF_CUDA(launch_gather_sidecars(ctx, ids, n, bea_w_out, sig_out, as_stream(stream)));
     return AIF_OK;
 }

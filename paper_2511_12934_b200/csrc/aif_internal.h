@@ -149,9 +149,14 @@ struct aif_ctx {
     uint64_t model_version = 0, table_version = 0;
     int64_t device_bytes = 0;
 
-    void *E = nullptr;
+    void *E = nullptr;          // the live copy of the item table and its sidecars: what every reader takes at call time
     void *bea_w = nullptr;
     uint8_t *sig = nullptr;
+    void *E_alt = nullptr;      // versioned_table: the spare copy, target of the next full refresh
+    void *bea_w_alt = nullptr;
+    uint8_t *sig_alt = nullptr;
+    cudaEvent_t table_ev = nullptr;   // end of the last full refresh of a versioned table
+    mutable bool table_ev_pending = false;
 
     // weights
     void *Wt[aif::kMaxHidden] = {};      // [in x out]
@@ -288,6 +293,7 @@ int nearline_compute(aif_ctx *ctx, const int32_t *ids, int64_t n, const void *I_
 void nearline_destroy(aif_ctx *ctx);
 // host-side checks shared by the scoring entry points (aif_api.cu)
 int check_user_state(aif_ctx *ctx, const aif_user_state *st);
+cudaError_t wait_table_ready(const aif_ctx *ctx, cudaStream_t st);   // orders st behind the last full refresh of a versioned table
 void set_last_error(const char *text);
 int tc_tiles_for(const aif_ctx *ctx, int n);
 size_t tc_tile_capacity(const aif_ctx *ctx);   // entries of the context's tile table (launches over several requests)

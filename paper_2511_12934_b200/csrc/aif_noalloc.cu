@@ -85,6 +85,7 @@ extern "C" int aif_score_noalloc(aif_ctx *ctx, const aif_user_state *state, cons
         cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
         const HostSlot &hs = ctx->slots[(size_t)state->index];
         cudaError_t e = cudaStreamWaitEvent(st, hs.ev, 0);
+        if (e == cudaSuccess) e = wait_table_ready(ctx, st);
         if (e == cudaSuccess) {
             TcScratch sc;
             tc_scratch_layout(ctx, base, kRows, &sc);

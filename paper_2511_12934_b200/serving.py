@@ -14,14 +14,15 @@ from . import synth
 
 def config_for(wl: synth.Workload, *, rows: Optional[int] = None, L_max: Optional[int] = None,
                max_user_states: Optional[int] = None, path: int = B.PATH_AUTO,
-               max_batch_candidates: Optional[int] = None) -> B.aif_config:
+               max_batch_candidates: Optional[int] = None, versioned_table: int = 0) -> B.aif_config:
     dt = B.F32 if wl.dtype == "f32" else B.BF16
     return B.make_config(
         dtype=dt, M=rows or wl.M, d=wl.d, L_max=L_max or wl.L, hidden=wl.hidden, F=wl.F, B=wl.B, dc=wl.dc,
         dU=wl.raw_dU, bucket_mode=wl.bucket_mode, blocks=wl.blocks, n_bridge=wl.n_bridge, lsh_bits=wl.lsh_bits,
         n_tiers=wl.n_tiers, lsh_din_norm=wl.lsh_din_norm, simtier_norm=wl.simtier_norm,
         emit_sigmoid=wl.emit_sigmoid, max_user_states=max_user_states or max(2, wl.R), mini_batch=wl.mini_batch,
-        path=path, max_batch_candidates=max_batch_candidates or max(1, wl.R * wl.N), n_categories=wl.n_categories)
+        path=path, max_batch_candidates=max_batch_candidates or max(1, wl.R * wl.N), n_categories=wl.n_categories,
+        versioned_table=versioned_table)
 
 
 class Server:

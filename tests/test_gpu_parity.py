@@ -498,3 +498,57 @@ def test_score_batch_host_gives_the_device_buffer_result():
     assert e.value.code == B.ERR_SHAPE
     assert srv.ctx.poll_status() == 0
     srv.close()
+
+
+def test_versioned_table_full_refresh_is_published_as_a_whole():
+    """versioned_table: a scoring call made before a full refresh keeps reading the old copy even though it runs after the
+    refresh has written (it sits behind a busy main stream while the refresh runs on a side stream); a call made after
+    the refresh reads the new copy.  A full refresh of fewer rows than the table carries the rest over; incremental
+    refreshes and the gather see the live copy; a second full refresh swaps back."""
+    wl = helpers.MINI["c2"].with_(name="versioned", N=600, blocks=helpers.ALL_BLOCKS)
+    weights = synth.make_weights(wl, zero_bias=False)
+    tab_a = synth.make_item_table(wl)
+    tab_b = synth.make_item_table(wl.with_(name="versioned_b"))
+    srv = serving.Server(wl, weights, tab_a, versioned_table=1)
+    oracle = helpers.make_oracle(wl, weights, M=tab_a["E"].shape[0])
+    rq = synth.make_request(wl, 0)
+    req = helpers.projected_request(wl, rq)
+    ids = synth.IdSampler(wl).request_ids(0)
+    st = srv.precompute(1, srv.upload_request(rq, B.USER_PROJECTED))
+    want_a, want_b = oracle.score(tab_a, req, ids), oracle.score(tab_b, req, ids)
+    assert np.abs(want_a - want_b).max() > 0.01
+    _check_logits(srv.score_ids(st, ids), want_a, TOL["bf16"])
+    ids_t = torch.from_numpy(ids).cuda()
+    out_old = torch.empty(len(ids), dtype=torch.float32, device="cuda")
+    out_new = torch.empty(len(ids), dtype=torch.float32, device="cuda")
+    dt = srv.dt
+    E_b, bw_b = B.to_device(tab_b["E"], dt), B.to_device(tab_b["bea_w"], dt)
+    sg_b = torch.from_numpy(np.ascontiguousarray(tab_b["sig"])).cuda()
+    torch.cuda.synchronize()
+    torch.cuda._sleep(40_000_000)                                  # the main stream is busy for some 20 ms
+    srv.ctx.score(st, ids_t, out_old)                              # made before the refresh: the old copy
+    with torch.cuda.stream(srv.side):
+        srv.ctx.item_nearline_refresh(None, E_b, bw_b, sg_b, stream=srv.side)   # runs at once, beside the sleeping main stream
+    srv.ctx.score(st, ids_t, out_new)                              # made after it: the new copy, once it is complete
+    torch.cuda.synchronize()
+    _check_logits(out_old.cpu().numpy(), want_a, TOL["bf16"])
+    _check_logits(out_new.cpu().numpy(), want_b, TOL["bf16"])
+    # a full refresh of the first half only: the second half is carried over from the live copy (table B)
+    half = tab_a["E"].shape[0] // 2
+    srv.ctx.item_nearline_refresh(None, B.to_device(tab_a["E"][:half], dt), B.to_device(tab_a["bea_w"][:half], dt),
+                                  torch.from_numpy(np.ascontiguousarray(tab_a["sig"][:half])).cuda())
+    mixed = {k: np.concatenate([tab_a[k][:half], tab_b[k][half:]]) for k in ("E", "bea_w", "sig")}
+    _check_logits(srv.score_ids(st, ids), oracle.score(mixed, req, ids), TOL["bf16"])
+    # incremental refresh and gather address the live copy
+    upd = np.array([int(ids[0]), int(ids[5])], dtype=np.int32)
+    for k in ("E", "bea_w", "sig"):
+        mixed[k] = mixed[k].copy()
+        mixed[k][upd] = tab_b[k][upd] if upd[0] < half else tab_a[k][upd]
+    srv.refresh_rows(upd, mixed["E"][upd], mixed["bea_w"][upd], mixed["sig"][upd])
+    _check_logits(srv.score_ids(st, ids), oracle.score(mixed, req, ids), TOL["bf16"])
+    got = torch.empty(len(ids), wl.d, dtype=torch.bfloat16, device="cuda")
+    srv.ctx.gather_rows(ids_t, got)
+    torch.cuda.synchronize()
+    assert np.array_equal(got.view(torch.int16).cpu().numpy().view(np.uint16), mixed["E"][ids])
+    assert srv.ctx.poll_status() == 0 and srv.ctx.get_stats().table_version == 4
+    srv.close()
