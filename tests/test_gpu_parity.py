@@ -552,3 +552,37 @@ def test_versioned_table_full_refresh_is_published_as_a_whole():
     assert np.array_equal(got.view(torch.int16).cpu().numpy().view(np.uint16), mixed["E"][ids])
     assert srv.ctx.poll_status() == 0 and srv.ctx.get_stats().table_version == 4
     srv.close()
+
+
+@pytest.mark.parametrize("kind", ["fused", "chain", "blocks", "categories", "simt"])
+def test_nothing_is_written_outside_the_logits(kind):
+    """Canary words on both sides of the logit array (which therefore starts on an odd 4-byte boundary) stay untouched by
+    every scoring path: the single-launch kernel, the kernel-per-layer chain, the chain with all blocks, grouped
+    candidates, and the CUDA-core kernel; ragged last tiles and a launch of several requests included."""
+    base = {"fused": helpers.MINI["c2"].with_(L=150), "chain": helpers.MINI["c2"].with_(L=300),
+            "blocks": helpers.MINI["c2"].with_(L=300, blocks=helpers.ALL_BLOCKS),
+            "categories": helpers.MINI["c2"].with_(L=300, blocks=helpers.ALL_BLOCKS, n_categories=6),
+            "simt": helpers.MINI["c1"]}[kind]
+    wl = base.with_(name=f"canary_{kind}", R=3, N=333, mini_batch=0)
+    weights, table, srv, oracle = _setup(wl)
+    sampler = synth.IdSampler(wl)
+    states, id_lists = [], []
+    for r in range(wl.R):
+        states.append(srv.precompute(r, srv.upload_request(synth.make_request(wl, r), B.USER_PROJECTED)))
+        id_lists.append(sampler.request_ids(r, 333 - 101 * r))
+    guard, sentinel = 67, -12345.5
+    for ids_l, sts in (([id_lists[0]], [states[0]]), (id_lists, states)):
+        n = sum(len(x) for x in ids_l)
+        buf = torch.full((n + 2 * guard,), sentinel, dtype=torch.float32, device="cuda")
+        ids_t = torch.from_numpy(np.concatenate(ids_l)).cuda()
+        offs = np.concatenate([[0], np.cumsum([len(x) for x in ids_l])])
+        if len(sts) == 1:
+            srv.ctx.score(sts[0], ids_t, buf[guard:guard + n])
+        else:
+            srv.ctx.score_batch(sts, ids_t, offs, buf[guard:guard + n])
+        torch.cuda.synchronize()
+        h = buf.cpu().numpy()
+        assert (h[:guard] == sentinel).all() and (h[guard + n:] == sentinel).all()
+        assert np.isfinite(h[guard:guard + n]).all() and not (h[guard:guard + n] == sentinel).any()
+    assert srv.ctx.poll_status() == 0
+    srv.close()
