@@ -3,6 +3,8 @@
 #include <cstring>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "aif_internal.h"
 
 using namespace aif;
@@ -155,6 +157,9 @@ static cudaError_t end_full_refresh(aif_ctx *ctx, cudaStream_t st)
     ctx->table_ev_pending = e == cudaSuccess;
     return e;
 }
+
+StageRange::StageRange(const char *name) { nvtxRangePushA(name); }
+StageRange::~StageRange() { nvtxRangePop(); }
 
 void set_last_error(const char *text) { snprintf(g_last_error, sizeof(g_last_error), "%s", text); }
 
@@ -463,6 +468,7 @@ int aif_load_weights(aif_ctx *ctx, const aif_weights *w, aif_stream stream)
 int aif_item_nearline_refresh(aif_ctx *ctx, const int32_t *ids, int64_t n, const void *rows, const void *bea_w,
                               const uint8_t *lsh_sig, aif_stream stream)
 {
+    StageRange range("aif_item_nearline_refresh");
     if (!ctx || !rows || n < 0) return AIF_ERR_ARG;
     if (ctx->bea_w && !bea_w) return AIF_ERR_ARG;
     if (ctx->sig && !lsh_sig) return AIF_ERR_ARG;
@@ -491,6 +497,7 @@ int aif_load_item_weights(aif_ctx *ctx, const aif_item_weights *w, aif_stream st
 int aif_item_nearline_compute(aif_ctx *ctx, const int32_t *ids, int64_t n, const void *I_raw, const void *I_id, const void *M_mm,
                               aif_stream stream)
 {
+    StageRange range("aif_item_nearline_compute");
     if (!ctx || !I_raw || n < 0) return AIF_ERR_ARG;
     if (ctx->sig && !M_mm) return AIF_ERR_ARG;
     if (!ids && n > ctx->cfg.M) return AIF_ERR_SHAPE;
@@ -513,6 +520,7 @@ int aif_item_nearline_compute(aif_ctx *ctx, const int32_t *ids, int64_t n, const
 int aif_user_precompute(aif_ctx *ctx, uint64_t request_key, const aif_user_inputs *in, int32_t L, aif_user_state **out,
                         aif_stream side_stream)
 {
+    StageRange range("aif_user_precompute");
     if (!ctx || !in || !out || in->struct_size != sizeof(aif_user_inputs)) return AIF_ERR_ARG;
     *out = nullptr;
     const aif_config &c = ctx->cfg;
@@ -616,6 +624,7 @@ int aif_user_state_export_bea(aif_ctx *ctx, const aif_user_state *state, void *V
 
 int aif_score(aif_ctx *ctx, const aif_user_state *state, const int32_t *cand_ids, int32_t n, float *logits, aif_stream stream)
 {
+    StageRange range("aif_score");
     int rc = state_check(ctx, state);
     if (rc != AIF_OK) return rc;
     if (n < 0) return AIF_ERR_SHAPE;
@@ -639,6 +648,7 @@ int aif_score(aif_ctx *ctx, const aif_user_state *state, const int32_t *cand_ids
 int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *states, const int32_t *cand_ids,
                     const int64_t *offsets, float *logits, aif_stream stream)
 {
+    StageRange range("aif_score_batch");
     if (!ctx || !states || !offsets || n_req < 0) return AIF_ERR_ARG;
     if (n_req == 0) return AIF_OK;
     if (n_req > ctx->ring.capacity) return AIF_ERR_SHAPE;
@@ -687,6 +697,7 @@ int aif_score_batch(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *st
 int aif_score_host(aif_ctx *ctx, const aif_user_state *state, const int32_t *host_ids, int32_t n, float *host_logits,
                    aif_stream stream)
 {
+    StageRange range("aif_score_host");
     int rc = state_check(ctx, state);
     if (rc != AIF_OK) return rc;
     if (n < 0 || (int64_t)n > ctx->cfg.max_batch_candidates) return AIF_ERR_SHAPE;
@@ -722,6 +733,7 @@ int aif_score_host(aif_ctx *ctx, const aif_user_state *state, const int32_t *hos
 int aif_score_batch_host(aif_ctx *ctx, int32_t n_req, const aif_user_state *const *states, const int32_t *host_ids,
                          const int64_t *offsets, float *host_logits, aif_stream stream)
 {
+    StageRange range("aif_score_batch_host");
     if (!ctx || !states || !offsets || n_req < 0) return AIF_ERR_ARG;
     if (n_req == 0) return AIF_OK;
     const int64_t total = offsets[n_req];

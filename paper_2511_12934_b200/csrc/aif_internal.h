@@ -202,6 +202,15 @@ namespace aif {
 extern std::atomic<uint64_t> g_launches;
 inline void count_launch(int n = 1) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+// A named host-side range (NVTX) around the launches of a stage or of an entry point: a timeline tool shows the kernels under
+// the stage's name.  With no tool attached a range costs two calls through an empty hook.
+struct StageRange {
+    explicit StageRange(const char *name);
+    ~StageRange();
+    StageRange(const StageRange &) = delete;
+    StageRange &operator=(const StageRange &) = delete;
+};
+
 // Timing marks: begin(st) before the first kernel of a scoring call, mark(name, st) after each kernel.
 void timing_begin(const aif_ctx *ctx, cudaStream_t st);
 void timing_mark(const aif_ctx *ctx, const char *name, cudaStream_t st);

@@ -314,9 +314,12 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
                         }
                         slab = (slab + 1u) % (uint32_t)C::kSlabs;
                     } else {
+                        // the last width may end in the middle of these 32 columns (a multiple of 16): the rest is skipped
                         const float4 *w4 = reinterpret_cast<const float4 *>(ws + c0);
+                        const int n_q = (p.n_cols - c0) >> 2;
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
+                            if (q >= n_q) break;
                             const float4 bb = b4[q], ww = w4[q];
                             dot = fmaf(fmaxf(__uint_as_float(r[4 * q]) + bb.x, 0.f), ww.x, dot);
                             dot = fmaf(fmaxf(__uint_as_float(r[4 * q + 1]) + bb.y, 0.f), ww.y, dot);
@@ -998,6 +1001,7 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl_in
     timing_begin(ctx, st);
     // a launch that fits the machine in one round of tiles: the whole pass in one kernel, one CTA per tile
     if (c.n_categories == 0 && sl.n_tiles <= kFusedMaxTiles && sl.max_L <= 256 && tc_fused_supported(c)) {
+        StageRange range("aif score_fused");
         cudaError_t e = launch_request_fused(ctx, sl, st);
         timing_mark(ctx, "score_fused", st);
         return e;
@@ -1005,6 +1009,7 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl_in
     if (c.n_categories > 0) {
         // candidates grouped by (request, category): tiles, grouped ids and the way back to the caller's order
         if (sc.rows < (size_t)sl.total + kTcTile || !ctx->sim_plan) return cudaErrorInvalidValue;
+        StageRange range("aif group");
         cudaError_t e = sim_group_candidates(ctx, sl, st);
         timing_mark(ctx, "group", st);
         if (e != cudaSuccess) return e;
@@ -1015,6 +1020,7 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl_in
         sl.tiles = (const TileDev *)sc.tiles;
     }
     if (c.blocks & AIF_BLK_CROSS) {
+        StageRange range("aif buckets");
         const int64_t n = sl.total * 8;   // eight threads per candidate
         const int grid = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
         cudaError_t e = launch_pdl(k_cross_buckets, dim3(grid), dim3(256), 0, st, sl.ids, sl.total, c.M, c.F, c.B,
@@ -1025,6 +1031,7 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl_in
     }
     const bool att_tc = ctx->tc_att_plan != nullptr;
     if (att_tc) {
+        StageRange range("aif attention");
         cudaError_t e = launch_att_tc(ctx, sl, st, sc.X, pl->x_cols, sc.rows);
         timing_mark(ctx, "attention", st);
         if (e != cudaSuccess) return e;
@@ -1039,12 +1046,14 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl_in
         const int x_din = (c.blocks & AIF_BLK_LSH_DIN) ? col : -1;
         if (c.blocks & AIF_BLK_LSH_DIN) col += c.d;
         const int x_tier = (c.blocks & AIF_BLK_SIMTIER) ? col : -1;
+        StageRange range("aif lsh");
         cudaError_t e = launch_lsh_tc(ctx, sl, st, sc.X, pl->x_cols, sc.rows, x_din, x_tier);
         timing_mark(ctx, "lsh", st);
         if (e != cudaSuccess) return e;
     }
     const bool need_att = (c.blocks & AIF_BLK_ATT) && !att_tc, need_lsh = lsh_blocks && !lsh_tc;
     if (pl->x_cols && (need_att || need_lsh || (c.blocks & AIF_BLK_BEA))) {
+        StageRange range("aif interact");
         const size_t smem = (size_t)8 * c.d * 4 + 64 * 4 + 128 * 4;
         cudaError_t e = launch_pdl(k_interact_x, dim3(sl.n_tiles), dim3(256), smem, st, md, sl, (__nv_bfloat16 *)sc.X, pl->x_cols,
                                    att_tc ? 1 : 0, lsh_tc ? 1 : 0);
@@ -1053,7 +1062,9 @@ cudaError_t launch_score_tc_scratch(const aif_ctx *ctx, const ScoreLaunch &sl_in
         if (e != cudaSuccess) return e;
     }
     static const char *names[kMaxHidden] = {"layer1", "layer2", "layer3", "layer4"};
+    static const char *range_names[kMaxHidden] = {"aif layer1", "aif layer2", "aif layer3", "aif layer4"};
     for (int k = 0; k < c.n_hidden; ++k) {
+        StageRange range(range_names[k]);
         LayerParams p{};
         p.sl = sl;
         p.n_nchunks = pl->n_nchunks[k], p.n_cols = pl->n_cols[k], p.n_k = pl->n_k[k], p.mini_batch = c.mini_batch;

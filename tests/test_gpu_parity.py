@@ -396,6 +396,23 @@ def test_single_launch_scoring_over_the_shapes_it_accepts(H2, F, dc, Bk, mode, s
     srv.close()
 
 
+@pytest.mark.parametrize("hidden", [(256, 48), (192, 16), (128, 64, 80), (512, 112)])
+def test_last_hidden_width_that_is_not_a_multiple_of_32(hidden):
+    """The kernel-per-layer path reads an accumulator 32 columns at a time; the last width only has to be a multiple of
+    16, so its last read is half used and the other half (columns no product wrote) must not reach the logit."""
+    wl = helpers.MINI["c2"].with_(name=f"h_{'_'.join(map(str, hidden))}", R=2, N=300, L=70, mini_batch=0, hidden=hidden)
+    weights, table, srv, oracle = _setup(wl, zero_bias=False)
+    sampler = synth.IdSampler(wl)
+    for r in range(wl.R):          # the second call finds whatever the first left in tensor and shared memory
+        rq = synth.make_request(wl, r)
+        ids = sampler.request_ids(r)
+        st = srv.precompute(3 + r, srv.upload_request(rq, B.USER_PROJECTED))
+        _check_logits(srv.score_ids(st, ids), oracle.score(table, helpers.projected_request(wl, rq), ids), TOL["bf16"])
+    assert srv.ctx.get_stats().tensor_path == 1
+    assert srv.ctx.poll_status() == 0
+    srv.close()
+
+
 @pytest.mark.parametrize("name", ["c3", "c4", "c5", "c5b"])
 def test_full_size_batches_on_sampled_candidates(name):
     """The multi-request shapes at their full sizes, scored in one aif_score_batch call exactly as the benchmark
