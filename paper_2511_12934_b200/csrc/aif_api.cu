@@ -275,6 +275,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     TRY(dev_alloc(ctx, &ctx->E, (size_t)c.M * c.d * el, true));
     if (c.blocks & AIF_BLK_BEA) TRY(dev_alloc(ctx, &ctx->bea_w, (size_t)c.M * c.n_bridge * el, true));
     if (c.blocks & (AIF_BLK_LSH_DIN | AIF_BLK_SIMTIER)) TRY(dev_alloc(ctx, (void **)&ctx->sig, (size_t)c.M * c.lsh_bits / 8, true));
+    TRY(dev_alloc(ctx, (void **)&ctx->e_norm, 4, true));
     if (c.versioned_table) {
         TRY(dev_alloc(ctx, &ctx->E_alt, (size_t)c.M * c.d * el, true));
         if (ctx->bea_w) TRY(dev_alloc(ctx, &ctx->bea_w_alt, (size_t)c.M * c.n_bridge * el, true));
@@ -307,7 +308,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     TRY(dev_alloc(ctx, (void **)&ctx->b_b, (size_t)c.d * 4, true));
 
     // user-state arena: fixed-size slots in one allocation
-    struct Off { size_t u, u32, S, T, V, sig, sigE, pu, pu_hl, prof, partial, ppart, Sg, sigEg, cat_off, cat_len, cat_map, cat_hist, end; } o{};
+    struct Off { size_t u, u32, S, T, V, sig, sigE, pu, pu_hl, prof, partial, ppart, Sg, sigEg, cat_off, cat_len, cat_map, cat_hist, k_norm, end; } o{};
     size_t p = 0;
     auto take = [&](size_t bytes) { size_t at = p; p += align_up(bytes ? bytes : 16, 256); return at; };
     o.u = take((size_t)c.d * el);
@@ -330,6 +331,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
     o.cat_len = take(sim ? (size_t)c.n_categories * 4 : 0);
     o.cat_map = take(sim ? (size_t)c.L_max * 4 : 0);
     o.cat_hist = take(sim ? (size_t)((c.L_max + 1023) / 1024) * c.n_categories * 4 : 0);
+    o.k_norm = take(4);
     o.end = p;
     ctx->slot_bytes = o.end;
     TRY(dev_alloc(ctx, (void **)&ctx->arena, ctx->slot_bytes * (size_t)c.max_user_states, true));
@@ -344,6 +346,7 @@ int aif_create(const aif_config *cfg, aif_ctx **out)
         hs.dev.T = base + o.T, hs.dev.V = base + o.V, hs.dev.sigS = (const uint8_t *)(base + o.sig);
         hs.dev.sigE = lsh_tc ? (const uint8_t *)(base + o.sigE) : nullptr;
         hs.dev.p_u = (const float *)(base + o.pu), hs.dev.pu_hl = base + o.pu_hl, hs.dev.L = 0;
+        hs.dev.k_norm = (const float *)(base + o.k_norm);
         hs.prof_hat = (float *)(base + o.prof), hs.partial = (float *)(base + o.partial), hs.ppart = (float *)(base + o.ppart);
         if (sim) {
             hs.dev.Sg = base + o.Sg, hs.dev.sigEg = lsh_tc ? (const uint8_t *)(base + o.sigEg) : nullptr;
@@ -479,6 +482,7 @@ int aif_item_nearline_refresh(aif_ctx *ctx, const int32_t *ids, int64_t n, const
     if (versioned) AIF_CUDA(begin_full_refresh(ctx, n, as_stream(stream)));
     else AIF_CUDA(wait_table_ready(ctx, as_stream(stream)));
     AIF_CUDA(launch_scatter_rows(ctx, ids, n, rows, bea_w, lsh_sig, as_stream(stream)));
+    AIF_CUDA(launch_row_norm_max(ctx, ctx->E, ids, n, ctx->cfg.M, ctx->e_norm, as_stream(stream)));
     if (versioned) AIF_CUDA(end_full_refresh(ctx, as_stream(stream)));
     ctx->table_version += 1;
     ctx->stats.table_version = ctx->table_version;
@@ -509,6 +513,7 @@ int aif_item_nearline_compute(aif_ctx *ctx, const int32_t *ids, int64_t n, const
     else AIF_CUDA(wait_table_ready(ctx, as_stream(stream)));
     const int rc = nearline_compute(ctx, ids, n, I_raw, I_id, M_mm, as_stream(stream));
     if (rc != AIF_OK) return rc;
+    AIF_CUDA(launch_row_norm_max(ctx, ctx->E, ids, n, ctx->cfg.M, ctx->e_norm, as_stream(stream)));
     if (versioned) AIF_CUDA(end_full_refresh(ctx, as_stream(stream)));
     ctx->table_version += 1;
     ctx->stats.table_version = ctx->table_version;

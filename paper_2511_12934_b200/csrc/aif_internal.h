@@ -34,6 +34,7 @@ struct SlotDev {
     const uint8_t *sigEg;   // [Lg x lsh_bits] +-1 bytes, or nullptr
     const int32_t *cat_off; // [n_categories] first row of every sub-sequence in Sg
     const int32_t *cat_len; // [n_categories] items of every sub-sequence
+    const float *k_norm;    // largest Euclidean norm of a row of S (set with the slot; NaN or inf rows make it so)
     int32_t L;
     int32_t pad_;
 };
@@ -155,6 +156,9 @@ struct aif_ctx {
     void *E_alt = nullptr;      // versioned_table: the spare copy, target of the next full refresh
     void *bea_w_alt = nullptr;
     uint8_t *sig_alt = nullptr;
+    // largest Euclidean norm of an item vector ever written to the table (device, only raised): with the slot's k_norm a
+    // bound on every attention score of a request, which lets the attention kernel drop its running maximum
+    float *e_norm = nullptr;
     cudaEvent_t table_ev = nullptr;   // end of the last full refresh of a versioned table
     mutable bool table_ev_pending = false;
 
@@ -220,6 +224,8 @@ ModelDev make_model(const aif_ctx *ctx);
 // aif_simt.cu
 cudaError_t launch_scatter_rows(const aif_ctx *ctx, const int32_t *ids, int64_t n, const void *rows, const void *bea_w,
                                 const uint8_t *sig, cudaStream_t st);
+// *out = max(*out, largest row norm) over rows ids[0..n) of `rows` (ids == nullptr: rows 0..n); ids outside [0, M) skipped
+cudaError_t launch_row_norm_max(const aif_ctx *ctx, const void *rows, const int32_t *ids, int64_t n, int64_t M, float *out, cudaStream_t st);
 cudaError_t launch_stage_ids(const int32_t *mapped_src, int32_t *dst, int n, cudaStream_t st);
 cudaError_t launch_gather_rows(const aif_ctx *ctx, const int32_t *ids, int64_t n, void *out, cudaStream_t st);
 cudaError_t launch_gather_sidecars(const aif_ctx *ctx, const int32_t *ids, int64_t n, void *bea_w_out, uint8_t *sig_out, cudaStream_t st);

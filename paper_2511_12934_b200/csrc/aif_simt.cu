@@ -626,7 +626,47 @@ __global__ void __launch_bounds__(256) k_user_finish(int raw, const T *__restric
     }
 }
 
-__global__ void k_set_slot_len(SlotDev *slots, int index, int L) { slots[index].L = L; }
+// the slot's length, and its key-norm bound back to zero (k_row_norm_max raises it once the rows are written)
+__global__ void k_set_slot_len(SlotDev *slots, int index, int L)
+{
+    slots[index].L = L;
+    *const_cast<float *>(slots[index].k_norm) = 0.f;
+}
+
+// Largest Euclidean norm over a set of rows, one warp per row.  Norms are non-negative, so their bit patterns order like
+// integers; a NaN row yields a pattern above every finite one and stays.
+template <typename T>
+__global__ void __launch_bounds__(256) k_row_norm_max(const T *__restrict__ rows, const int32_t *__restrict__ ids, int64_t n, int64_t M, int d,
+                                                      float *__restrict__ out)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t w0 = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5), stride = (int64_t)gridDim.x * 8;
+    int best = 0;
+    for (int64_t i = w0; i < n; i += stride) {
+        const int64_t r = ids ? (int64_t)ids[i] : i;
+        if (r < 0 || r >= M) continue;
+        const T *row = rows + (size_t)r * d;
+        float acc = 0.f;
+        for (int c = lane; c < d; c += 32) {
+            const float v = to_f(row[c]);
+            acc = fmaf(v, v, acc);
+        }
+        acc = warp_sum(acc);
+        best = max(best, __float_as_int(sqrtf(acc)) & 0x7fffffff);
+    }
+    if (lane == 0 && best > 0) atomicMax(reinterpret_cast<int *>(out), best);
+}
+
+cudaError_t launch_row_norm_max(const aif_ctx *ctx, const void *rows, const int32_t *ids, int64_t n, int64_t M, float *out, cudaStream_t st)
+{
+    if (n <= 0 || !out) return cudaSuccess;
+    const int64_t want = (n + 7) / 8;
+    const int grid = (int)(want < 148 * 8 ? want : 148 * 8);
+    if (ctx->cfg.dtype == AIF_F32) k_row_norm_max<float><<<grid, 256, 0, st>>>((const float *)rows, ids, n, M, ctx->cfg.d, out);
+    else k_row_norm_max<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)rows, ids, n, M, ctx->cfg.d, out);
+    count_launch();
+    return cudaGetLastError();
+}
 
 // partial[g][k] = sum over rows g, g + n_parts, ... of rows[i][k] (bf16 rows, fp32 sums in a fixed order): the mean pooling of
 // eq. 2 over hidden FFN activations that a tensor-core layer has written
@@ -688,6 +728,7 @@ static cudaError_t user_network_typed(const aif_ctx *ctx, HostSlot &hs, int slot
     k_set_slot_len<<<1, 1, 0, st>>>(ctx->slots_dev, slot_index, L);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = launch_row_norm_max(ctx, S, nullptr, L, L, const_cast<float *>(hs.dev.k_norm), st)) != cudaSuccess) return e;
     if (raw) {
         // eq. 2: the attention rows on the tensor cores where the shape allows, else inside k_user_self
         const T *att_rows = nullptr;

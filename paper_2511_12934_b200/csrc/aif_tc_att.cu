@@ -37,7 +37,15 @@ struct AttParams {
     int32_t x_stride;        // elements per row of X
     __nv_bfloat16 *X;        // attention rows go to columns [0, d)
     float scale_log2;        // log2(e) / sqrt(d)
+    const float *q_norm;     // device: upper bound on the Euclidean norm of a query row, or nullptr (none known)
 };
+
+// A request whose scores are bounded by this many powers of two on either side (|q| |k| log2(e) / sqrt(d), from the norm
+// bounds kept with the table and with the slot) needs no running maximum: softmax does not depend on the exponent's
+// offset, 2^+-50 is far inside the range of fp32 sums and of bf16 probabilities, whose relative precision does not
+// depend on the magnitude.  Without the maximum a block costs its warps no reduction, no exchange between the two
+// warps of a row quarter and no barrier, so the two run out of step and one's exponentials cover the other's loads.
+constexpr float kNoMaxBound = 50.0f;
 
 template <int D, int BN>
 struct AttCfg {
@@ -47,9 +55,13 @@ struct AttCfg {
     static constexpr int kKvStages = D <= 128 ? 4 : 3;
     static constexpr int kKvChunkBytes = BN * 128;      // one 64-column chunk of a key block
     static constexpr int kKvBytes = kQChunks * kKvChunkBytes;
-    static constexpr int kTmemO = 2 * BN;               // column of the (first) O accumulator
-    // d = 128 leaves 128 tensor-memory columns free: a second O accumulator, and four more warps that normalise and store
-    // a finished tile while the softmax warps and the MMAs are already on the next one
+    // tensor memory: two score buffers of BN columns | two probability buffers of BN / 2 columns (packed bf16 pairs) | O.
+    // The probabilities have columns of their own: a score buffer is free for the scores of block j + 2 as soon as the
+    // softmax warps have read block j out of it, not only once P V of block j has run.
+    static constexpr int kTmemP = 2 * BN;
+    static constexpr int kTmemO = 3 * BN;
+    // d = 128: four more warps normalise and store a finished tile while the softmax warps and the Q K^T products are
+    // already on the next one (its first P V waits until they have read the accumulator)
     static constexpr bool kSplitEpi = D <= 128;
     // softmax warps per quarter of the rows, each with its share of a block's keys: one warp alone leaves its scheduler
     // idle through every tensor-memory round trip and hand-over
@@ -108,8 +120,8 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
     uint64_t *kv_full = bars, *kv_empty = bars + kS;
     uint64_t *s_full = bars + 2 * kS, *p_full = s_full + 2, *pv_done = p_full + 2;
     uint64_t *q_full = pv_done + 2, *q_empty = q_full + 2, *o_final = q_empty + 2, *o_free = o_final + 2, *l_ready = o_free + 2;
-    uint64_t *q_first = l_ready + 2;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_first + 1);
+    uint64_t *q_first = l_ready + 2, *s_free = q_first + 1;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(s_free + 2);
     volatile uint32_t *abort_flag = tmem_slot + 1;
     float *l_s = reinterpret_cast<float *>(tmem_slot + 4);   // [2][kHalves][128] row sums handed to the output warps
     float *mx_s = l_s + (kSplit ? 2 * C::kHalves * 128 : 0);    // [2][2][128] block maxima exchanged between partner warps
@@ -125,6 +137,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
             mbar_init(smem_u32(s_full + b), 1);
             mbar_init(smem_u32(p_full + b), C::kSoftWarps * 32);
             mbar_init(smem_u32(pv_done + b), 1);
+            mbar_init(smem_u32(s_free + b), C::kSoftWarps);
             mbar_init(smem_u32(q_full + b), 32);
             mbar_init(smem_u32(q_empty + b), 5);   // the last Q K^T of the tenant, and the four softmax warps' output staging
         }
@@ -152,7 +165,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
     auto tile_epilogue = [&](int k, const AttTile &t, float l_sum, int wq, int lane) {
         const int row = wq * 32 + lane;
         const uint32_t lane_base = tmem_base + ((uint32_t)(wq * 32) << 16);
-        const uint32_t o_col = (uint32_t)(C::kTmemO + (kSplit ? (k & 1) * D : 0));
+        const uint32_t o_col = (uint32_t)C::kTmemO;
         uint64_t *o_free_k = o_free + (kSplit ? (k & 1) : 0);
         const float inv = l_sum > 0.f ? 1.0f / l_sum : 0.f;   // no key at all (an empty sub-sequence): a zero row
         bool good = false;
@@ -256,7 +269,13 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
         for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++k) {
             const AttTile t = att_tile<BN>(p, tile);
             const int L = t.L;
-            float m_used = -INFINITY, l_sum = 0.f;
+            // Decided once per tile and agreed on by the warps that meet at a barrier in the other mode: two warps
+            // reading a bound that a refresh is raising meanwhile must not come to different answers.
+            const float bound = p.q_norm ? *p.q_norm * *p.sl.slots[t.slot].k_norm * k2 : INFINITY;
+            bool fast = bound <= kNoMaxBound;    // NaN: false
+            if (kH == 2) fast = !named_bar_or(1 + wq, 64, !fast || late);
+            else fast = __all_sync(0xffffffffu, fast);
+            float m_used = fast ? 0.f : -INFINITY, l_sum = 0.f;
             for (int j = 0; j < t.nb; ++j, ++gb) {
                 const int b = (int)(gb & 1u);
                 const int valid_cols = min(BN, L - j * BN);
@@ -271,7 +290,27 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
 #pragma unroll
                     for (int c0 = 0; c0 < CW; c0 += 32)
                         tmem_ld32(ts + (uint32_t)(half * CW + c0), *reinterpret_cast<uint32_t(*)[32]>(&sc[c0]));
+                }
+                // the probability buffer's previous reader, P V of block gb - 2, must be done with it (long since, as a rule)
+                const bool p_free = gb < 2 || __all_sync(0xffffffffu, mbar_wait(smem_u32(pv_done + b), ((gb - 2) >> 1) & 1u, abort_flag));
+                if (got) {
                     tmem_ld_wait();
+                    // the scores are in registers: the buffer may take the scores of block gb + 2
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(s_free + b));
+                }
+                if (fast) {
+                    if (!got || !p_free) {   // nobody waits for this warp inside the block: it goes on empty-handed to the next meeting point
+                        if (kH == 2) {
+                            late = true;
+                            continue;
+                        }
+                        ok = false;
+                        break;
+                    }
+                } else {
+                if (got) {
                     // block maximum of the row (four independent chains)
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                     if (vc == CW) {
@@ -291,19 +330,18 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
                 }
                 if (kH == 2) {
                     // The two warps of a row quarter agree on the block maximum through shared memory (two buffers: the
-                    // partner may still read block gb - 1's value).  The barrier also orders this warp's score loads
-                    // before the partner's probability stores, which for the second half land in the first half's columns.
+                    // partner may still read block gb - 1's value).
                     float *mx = mx_s + (gb & 1u) * 256;
                     mx[half * 128 + row] = mt;
                     tc_fence_before();
-                    const bool bad = named_bar_or(1 + wq, 64, !got || late);
+                    const bool bad = named_bar_or(1 + wq, 64, !got || !p_free || late);
                     tc_fence_after();
                     if (bad) {
                         ok = false;
                         break;
                     }
                     mt = fmaxf(mt, mx[(half ^ 1) * 128 + row]);
-                } else if (!got) {
+                } else if (!got || !p_free) {
                     ok = false;
                     break;
                 }
@@ -331,7 +369,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
 #pragma unroll 1
                             for (int c0 = half * (D / kH); c0 < (half + 1) * (D / kH); c0 += 32) {
                                 uint32_t r[32];
-                                const uint32_t oc = (uint32_t)(C::kTmemO + (kSplit ? (k & 1) * D : 0) + c0);
+                                const uint32_t oc = (uint32_t)(C::kTmemO + c0);
                                 tmem_ld32(lane_base + oc, r);
                                 tmem_ld_wait();
 #pragma unroll
@@ -342,8 +380,8 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
                         }
                     }
                 }
-                // probabilities -> packed bf16 pairs over the first BN / 2 columns of the score buffer just read (P V of
-                // block gb - 2, the buffer's previous reader, precedes the Q K^T that refilled it in the MMA pipe)
+                }
+                // probabilities -> packed bf16 pairs in the block's probability buffer
                 float ls4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int c0 = 0; c0 < CW; c0 += 64) {
@@ -360,7 +398,7 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
                         const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                         packed[i] = *reinterpret_cast<const uint32_t *>(&h);
                     }
-                    tmem_st32(ts + (uint32_t)((half * CW + c0) >> 1), packed);
+                    tmem_st32(lane_base + (uint32_t)(C::kTmemP + b * (BN / 2) + ((half * CW + c0) >> 1)), packed);
                 }
                 tmem_st_wait();
                 l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
@@ -434,8 +472,8 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
                     }
                     const int s = (int)(c.gb % kS);
                     if (!mbar_wait(smem_u32(kv_full + s), (c.gb / kS) & 1u, abort_flag)) break;
-                    // the buffer's previous content, the probabilities of block gb - 2, must have been consumed by its P V
-                    if (c.gb >= 2 && !mbar_wait(smem_u32(pv_done + (c.gb & 1u)), ((c.gb - 2) >> 1) & 1u, abort_flag)) break;
+                    // the buffer's previous content, the scores of block gb - 2, must have been read by every softmax warp
+                    if (c.gb >= 2 && !mbar_wait(smem_u32(s_free + (c.gb & 1u)), ((c.gb - 2) >> 1) & 1u, abort_flag)) break;
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + (uint32_t)((c.gb & 1u) * BN);
                     const uint64_t qd = qdesc0 + (uint64_t)(uint32_t)(qb * (C::kQBytes >> 4));
@@ -455,13 +493,14 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
                 while (ok && c.tile < n_tiles) {
                     if (!mbar_wait(smem_u32(p_full + (c.gb & 1u)), (c.gb >> 1) & 1u, abort_flag)) break;
                     // the first P V of a tile overwrites O: the output of the accumulator's previous tile must have been read
-                    if (c.j == 0 && (kSplit ? c.k >= 2 && !mbar_wait(smem_u32(o_free + (c.k & 1)), (uint32_t)(((c.k - 2) >> 1) & 1), abort_flag)
-                                            : c.k > 0 && !mbar_wait(smem_u32(o_free), (uint32_t)((c.k - 1) & 1), abort_flag)))
+                    if (c.j == 0 && c.k > 0 &&
+                        !(kSplit ? mbar_wait(smem_u32(o_free + ((c.k - 1) & 1)), (uint32_t)(((c.k - 1) >> 1) & 1), abort_flag)
+                                 : mbar_wait(smem_u32(o_free), (uint32_t)((c.k - 1) & 1), abort_flag)))
                         break;
                     tc_fence_after();
                     const int s = (int)(c.gb % kS);
-                    const uint32_t o_tmem = tmem_base + (uint32_t)(C::kTmemO + (kSplit ? (c.k & 1) * D : 0));
-                    const uint32_t p_tmem = tmem_base + (uint32_t)((c.gb & 1u) * BN);   // P: 8 columns per 16 keys
+                    const uint32_t o_tmem = tmem_base + (uint32_t)C::kTmemO;
+                    const uint32_t p_tmem = tmem_base + (uint32_t)(C::kTmemP + (c.gb & 1u) * (BN / 2));   // P: 8 columns per 16 keys
                     const uint64_t vd = vdesc0 + (uint64_t)(uint32_t)(s * (C::kKvBytes >> 4));
 #pragma unroll
                     for (int kk = 0; kk < BN / 16; ++kk)   // V: 16 keys further = 16 rows x 128 bytes
@@ -664,6 +703,7 @@ cudaError_t launch_att_tc(const aif_ctx *ctx, const ScoreLaunch &sl, cudaStream_
     p.sl = sl, p.E = (const uint8_t *)ctx->E, p.M = c.M, p.mini_batch = c.mini_batch;
     p.x_stride = x_stride, p.X = (__nv_bfloat16 *)X;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.d);
+    p.q_norm = ctx->e_norm;
     // One CTA per SM walking over its tiles hides a tile's query gather and output behind its neighbours' key blocks:
     // 22 k against 31 k cycles per 8-block tile, which outweighs the static assignment's rounding (8.5 tiles per SM cost
     // 9 tile times) as soon as some SM has two tiles.
@@ -691,6 +731,7 @@ cudaError_t launch_self_att_tc(const aif_ctx *ctx, int slot_index, int L, cudaSt
     p.sl = sl, p.E = reinterpret_cast<const uint8_t *>(ctx->slots[(size_t)slot_index].dev.S), p.M = L, p.mini_batch = 0;
     p.x_stride = c.d, p.X = pl->self_rows;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)c.d);
+    p.q_norm = ctx->slots[(size_t)slot_index].dev.k_norm;   // the queries are the sequence rows themselves
     CUtensorMap tmap_x;
     cudaError_t ex = encode_x_map(&tmap_x, pl->self_rows, c.d, (size_t)c.L_max + kTcTile);
     if (ex != cudaSuccess) return ex;
