@@ -21,6 +21,8 @@
 // The running maximum is only raised when a row's block maximum exceeds it by more than 8 (in the log2 domain);
 // then the warp rescales its 32 rows of O in TMEM.  Until then probabilities stay below 2^8, which fp32 sums and
 // bf16 operands hold without loss of accuracy.  Every wait is bounded.
+#include <type_traits>
+
 #include "aif_device.cuh"
 #include "aif_internal.h"
 #include "aif_tc_ptx.cuh"
@@ -382,26 +384,38 @@ __global__ void __launch_bounds__((AttCfg<D, BN>::kThreads), 1) k_att_tc(const _
                 }
                 }
                 // probabilities -> packed bf16 pairs in the block's probability buffer
-                float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+                // The loop is bound by issue slots, so exponent and row sum are formed two at a time (f32x2), and the
+                // masking of keys past the end of the sequence exists only in the copy a ragged last block runs.
+                const uint64_t k2p = pack_f32x2(k2, k2), mneg = pack_f32x2(-m_used, -m_used);
+                uint64_t ls2[2] = {0ull, 0ull};
+                auto probabilities = [&](auto masked) {
 #pragma unroll
-                for (int c0 = 0; c0 < CW; c0 += 64) {
-                    uint32_t packed[32];
+                    for (int c0 = 0; c0 < CW; c0 += 64) {
+                        uint32_t packed[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        float p0 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i]), k2, -m_used));
-                        float p1 = fast_exp2(fmaf(__uint_as_float(sc[c0 + 2 * i + 1]), k2, -m_used));
-                        if (vc != CW) {
-                            if (c0 + 2 * i >= vc) p0 = 0.f;
-                            if (c0 + 2 * i + 1 >= vc) p1 = 0.f;
+                        for (int i = 0; i < 32; ++i) {
+                            float p0, p1;
+                            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sc[c0 + 2 * i]), __uint_as_float(sc[c0 + 2 * i + 1])), k2p, mneg), p0, p1);
+                            p0 = fast_exp2(p0), p1 = fast_exp2(p1);
+                            if (decltype(masked)::value) {
+                                if (c0 + 2 * i >= vc) p0 = 0.f;
+                                if (c0 + 2 * i + 1 >= vc) p1 = 0.f;
+                            }
+                            ls2[i & 1] = add_f32x2(ls2[i & 1], pack_f32x2(p0, p1));
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                            packed[i] = *reinterpret_cast<const uint32_t *>(&h);
                         }
-                        ls4[i & 3] += p0 + p1;
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                        packed[i] = *reinterpret_cast<const uint32_t *>(&h);
+                        tmem_st32(lane_base + (uint32_t)(C::kTmemP + b * (BN / 2) + ((half * CW + c0) >> 1)), packed);
                     }
-                    tmem_st32(lane_base + (uint32_t)(C::kTmemP + b * (BN / 2) + ((half * CW + c0) >> 1)), packed);
-                }
+                };
+                if (vc == CW) probabilities(std::false_type{});
+                else probabilities(std::true_type{});
                 tmem_st_wait();
-                l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+                {
+                    float a0, a1, b0, b1;
+                    unpack_f32x2(ls2[0], a0, a1), unpack_f32x2(ls2[1], b0, b1);
+                    l_sum += (a0 + a1) + (b0 + b1);
+                }
                 tc_fence_before();
                 mbar_arrive(smem_u32(p_full + b));
             }
