@@ -253,6 +253,46 @@ def test_sharp_softmax_exercises_the_running_max_rescaling(base, L, s_scale):
     srv.close()
 
 
+@pytest.mark.parametrize("base,L", [("c2", 700), ("c5", 300)])
+def test_softmax_with_and_without_a_running_maximum_in_one_launch(base, L):
+    """The attention kernel drops the running maximum for a request whose scores are bounded by 2^+-50 (largest item norm
+    x largest sequence-row norm x log2(e) / sqrt(d)).  Four requests in one launch: the workload's own sequence (bound of
+    a few units), the sequence scaled to a bound of 45 and of 55 (either side of the switch) and of 600; every tile takes
+    its own mode and all must agree with the oracle.  Then a refresh writes one item vector 64 times longer: the table's
+    bound only grows, every request falls back to the exact form, and the results stay the same."""
+    wl = helpers.MINI[base].with_(name=f"modes_{base}", R=4, N=300, L=L, mini_batch=0)
+    weights, table, srv, oracle = _setup(wl, zero_bias=False, max_batch_candidates=wl.R * wl.N)
+    E = synth.bf16_bits_to_f32(table["E"])
+    e_norm = float(np.sqrt((E.astype(np.float64) ** 2).sum(1)).max())
+    k2 = np.log2(np.e) / np.sqrt(wl.d)
+    sampler = synth.IdSampler(wl)
+    states, id_lists, reqs = [], [], []
+    for r, target in enumerate([None, 45.0, 55.0, 600.0]):
+        rq = synth.make_request(wl, r)
+        if target is not None:
+            S = synth.bf16_bits_to_f32(rq["S"]).astype(np.float64)
+            k_norm = float(np.sqrt((S ** 2).sum(1)).max())
+            rq["S"] = synth.to_bf16_bits((S * (target / (e_norm * k_norm * k2))).astype(np.float32))
+        states.append(srv.precompute(r, srv.upload_request(rq, B.USER_PROJECTED)))
+        id_lists.append(sampler.request_ids(r)), reqs.append(helpers.projected_request(wl, rq))
+    wants = [oracle.score(table, reqs[r], id_lists[r]) for r in range(wl.R)]
+
+    def check():
+        for o, w in zip(srv.score_many(states, id_lists), wants):
+            _check_logits(o, w, 1e-2 * max(1.0, float(np.abs(w).max())))
+        _check_logits(srv.score_ids(states[1], id_lists[1]), wants[1], 1e-2 * max(1.0, float(np.abs(wants[1]).max())))
+        assert srv.ctx.get_stats().tensor_path == 1 and srv.ctx.poll_status() == 0
+
+    check()
+    # a row no candidate uses, 64 times longer than any other
+    used = np.unique(np.concatenate(id_lists))
+    spare = int(np.setdiff1d(np.arange(table["E"].shape[0]), used)[0])
+    row = synth.to_bf16_bits(E[spare:spare + 1] * 64.0 + 1.0)
+    srv.refresh_rows(np.array([spare], dtype=np.int32), row)
+    check()
+    srv.close()
+
+
 @pytest.mark.parametrize("L", [1, 77, 128, 129, 200, 256, 257])
 def test_single_launch_scoring_at_the_sequence_lengths_around_its_key_blocks(L):
     """Launches of at most one tile per SM with sequences of at most 256 items run the whole pass in one kernel (one or
