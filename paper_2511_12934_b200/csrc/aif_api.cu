@@ -513,7 +513,6 @@ int aif_item_nearline_compute(aif_ctx *ctx, const int32_t *ids, int64_t n, const
     else AIF_CUDA(wait_table_ready(ctx, as_stream(stream)));
     const int rc = nearline_compute(ctx, ids, n, I_raw, I_id, M_mm, as_stream(stream));
     if (rc != AIF_OK) return rc;
-    AIF_CUDA(launch_row_norm_max(ctx, ctx->E, ids, n, ctx->cfg.M, ctx->e_norm, as_stream(stream)));
     if (versioned) AIF_CUDA(end_full_refresh(ctx, as_stream(stream)));
     ctx->table_version += 1;
     ctx->stats.table_version = ctx->table_version;

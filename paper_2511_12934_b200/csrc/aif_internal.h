@@ -299,8 +299,9 @@ cudaError_t tc_dense_layer(const aif_ctx *ctx, const DenseLayer &L, int64_t rows
 // the item-side tower in one kernel, hidden activations in tensor memory (aif_tc_tower.cu)
 bool tc_tower_supported(int dI, int hI, int d);
 cudaError_t tc_tower_prepare();
+// norm_max (device, may be null): raised to an upper bound of the largest Euclidean norm of an output row
 cudaError_t launch_item_tower_tc(const aif_ctx *ctx, const void *I_raw, const void *W0, const float *b0, const void *W1, const float *b1,
-                                 void *out, int64_t n, int dI, int hI, cudaStream_t st);
+                                 void *out, int64_t n, int dI, int hI, float *norm_max, cudaStream_t st);
 // item side of the nearline pipeline (aif_nearline.cu)
 int nearline_load_weights(aif_ctx *ctx, const aif_item_weights *w, cudaStream_t st);
 int nearline_compute(aif_ctx *ctx, const int32_t *ids, int64_t n, const void *I_raw, const void *I_id, const void *M_mm,

@@ -125,7 +125,8 @@ cudaError_t run_pass(aif_ctx *ctx, NearlinePlan *pl, int64_t m, const void *I_ra
     const aif_config &c = ctx->cfg;
     cudaError_t e;
     if (pl->tensor && pl->fused_tower) {
-        if ((e = launch_item_tower_tc(ctx, I_raw, pl->W0, pl->b0, pl->W1, pl->b1, rows_out, m, pl->dI, pl->hI, st)) != cudaSuccess) return e;
+        // the kernel also raises the table's norm bound from the rows it writes
+        if ((e = launch_item_tower_tc(ctx, I_raw, pl->W0, pl->b0, pl->W1, pl->b1, rows_out, m, pl->dI, pl->hI, ctx->e_norm, st)) != cudaSuccess) return e;
     } else if (pl->tensor) {
         DenseLayer l0{I_raw, pl->W0, pl->b0, pl->hidden, pl->dI, pl->hI, 1, 0};
         if ((e = tc_dense_layer(ctx, l0, m, st)) != cudaSuccess) return e;
@@ -137,6 +138,8 @@ cudaError_t run_pass(aif_ctx *ctx, NearlinePlan *pl, int64_t m, const void *I_ra
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
+    // the table's norm bound from the rows just computed (whether or not their ids turn out to lie in the table)
+    if (!(pl->tensor && pl->fused_tower) && (e = launch_row_norm_max(ctx, rows_out, nullptr, m, m, ctx->e_norm, st)) != cudaSuccess) return e;
     if (c.blocks & AIF_BLK_BEA) {
         k_item_bridge_weights<T><<<grid_for_items(m), 256, 0, st>>>((const T *)(I_id ? I_id : rows_out), m, c.d, c.n_bridge,
                                                                     (const T *)pl->bridges, (T *)bea_out);

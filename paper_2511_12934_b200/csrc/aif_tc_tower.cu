@@ -35,6 +35,7 @@ struct TowerParams {
     int32_t n_pairs, n_k1, hI, d;
     const float *b0, *b1;
     __nv_bfloat16 *out;   // [n x d]
+    float *norm_max;      // raised to the largest Euclidean norm of an output row (an upper bound: taken before rounding, widened by 2^-8)
     uint32_t *status;
 };
 
@@ -129,6 +130,7 @@ __global__ void __launch_bounds__(kTThreads, 1) k_item_tower_tc(const __grid_con
             tc_fence_after();
             if (!ok) break;
             const bool whole = row0 + wq * 32 + 32 <= p.n;
+            float ss = 0.f;   // squared norm of this thread's output row
             for (int c0 = 0; c0 < p.d; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(col0 + (uint32_t)(128 + c0), r);
@@ -142,8 +144,11 @@ __global__ void __launch_bounds__(kTThreads, 1) k_item_tower_tc(const __grid_con
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     const float4 bb = b4[q];
-                    const __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[4 * q]) + bb.x, __uint_as_float(r[4 * q + 1]) + bb.y);
-                    const __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[4 * q + 2]) + bb.z, __uint_as_float(r[4 * q + 3]) + bb.w);
+                    const float x0 = __uint_as_float(r[4 * q]) + bb.x, x1 = __uint_as_float(r[4 * q + 1]) + bb.y;
+                    const float x2 = __uint_as_float(r[4 * q + 2]) + bb.z, x3 = __uint_as_float(r[4 * q + 3]) + bb.w;
+                    ss = fmaf(x0, x0, fmaf(x1, x1, fmaf(x2, x2, fmaf(x3, x3, ss))));
+                    const __nv_bfloat162 h0 = __floats2bfloat162_rn(x0, x1);
+                    const __nv_bfloat162 h1 = __floats2bfloat162_rn(x2, x3);
                     packed[2 * q] = *reinterpret_cast<const uint32_t *>(&h0);
                     packed[2 * q + 1] = *reinterpret_cast<const uint32_t *>(&h1);
                 }
@@ -167,6 +172,12 @@ __global__ void __launch_bounds__(kTThreads, 1) k_item_tower_tc(const __grid_con
                     for (int q = 0; q < 4; ++q)
                         dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
                 }
+            }
+            if (p.norm_max) {
+                // non-negative floats order like their bit patterns; a NaN row gives a pattern above every finite one
+                const int bits = row0 + row < p.n ? (__float_as_int(sqrtf(ss) * 1.00390625f) & 0x7fffffff) : 0;
+                const int best = __reduce_max_sync(0xffffffffu, bits);
+                if (lane == 0 && best > 0) atomicMax(reinterpret_cast<int *>(p.norm_max), best);
             }
         }
         if (lane == 0) bulk_wait<0>();
@@ -286,7 +297,7 @@ cudaError_t tc_tower_prepare() { return cudaFuncSetAttribute(k_item_tower_tc, cu
 
 // out [n x d] = W1 ReLU(W0 I_raw^T + b0) + b1 for n rows of I_raw [n x dI]; all matrices bf16 row-major, biases fp32.
 cudaError_t launch_item_tower_tc(const aif_ctx *ctx, const void *I_raw, const void *W0, const float *b0, const void *W1, const float *b1,
-                                 void *out, int64_t n, int dI, int hI, cudaStream_t st)
+                                 void *out, int64_t n, int dI, int hI, float *norm_max, cudaStream_t st)
 {
     if (n <= 0) return cudaSuccess;
     const int d = ctx->cfg.d;
@@ -298,7 +309,7 @@ cudaError_t launch_item_tower_tc(const aif_ctx *ctx, const void *I_raw, const vo
     if ((e = encode2d(&mo, out, (uint64_t)d, (uint64_t)n, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) != cudaSuccess) return e;
     TowerParams p{};
     p.n = n, p.n_pairs = (int)((n + 2 * kTcTile - 1) / (2 * kTcTile)), p.n_k1 = dI / 64, p.hI = hI, p.d = d;
-    p.b0 = b0, p.b1 = b1, p.out = (__nv_bfloat16 *)out, p.status = ctx->status;
+    p.b0 = b0, p.b1 = b1, p.out = (__nv_bfloat16 *)out, p.norm_max = norm_max, p.status = ctx->status;
     const int grid = p.n_pairs < 148 ? p.n_pairs : 148;
     e = launch_pdl(k_item_tower_tc, dim3(grid), dim3(kTThreads), kTSmem, st, ma, m0, m1, mo, p);
     count_launch();

@@ -137,6 +137,43 @@ def test_scoring_on_a_table_built_by_the_nearline_call():
     srv.close()
 
 
+@pytest.mark.parametrize("dims", [(512, 256, 64), (192, 512, 64)])
+def test_item_vectors_from_the_nearline_call_raise_the_tables_norm_bound(dims):
+    """The attention kernel drops its running maximum only while (largest item norm) x (largest sequence-row norm) keeps
+    the scores within 2^+-50; the nearline call has to raise the table's bound from the rows it computes (inside the
+    one-kernel tower for the first shape, by a pass over its output for the second).  The table starts with small
+    vectors; the call then writes vectors with every component near 40, and the sequence is scaled so that scores reach
+    several hundred: scored with a stale bound the exponentials overflow.  The oracle scores on the rows read back from
+    the device (the item side's own parity is checked elsewhere)."""
+    wl = helpers.MINI["c2"].with_(name=f"nearline_norm_{dims[1]}", M=2000, N=500, L=300, mini_batch=0, hidden=(256, 256))
+    weights = synth.make_weights(wl, zero_bias=False)
+    table = synth.make_item_table(wl)
+    srv = serving.Server(wl, weights, table)
+    it = synth.make_item_side(wl, wl.M, dI=dims[0], hI=dims[1], d_mm=dims[2])
+    it["b_i1"] = (it["b_i1"] + 40.0).astype(np.float32)
+    dev = {k: (torch.from_numpy(v).cuda() if v.dtype == np.float32 else B.to_device(v, B.BF16)) for k, v in it.items()}
+    srv.ctx.load_item_weights(dev)
+    srv.ctx.item_nearline_compute(None, dev["I_raw"], dev["I_id"], dev["M_mm"])
+    ids_all = torch.arange(wl.M, dtype=torch.int32, device="cuda")
+    rows = torch.empty(wl.M, wl.d, dtype=torch.bfloat16, device="cuda")
+    srv.ctx.gather_rows(ids_all, rows)
+    torch.cuda.synchronize()
+    host = {"E": rows.view(torch.int16).cpu().numpy().view(np.uint16)}
+    assert np.abs(synth.bf16_bits_to_f32(host["E"])).mean() > 30.0
+    rq = synth.make_request(wl, 0)
+    rq["S"] = synth.to_bf16_bits(synth.bf16_bits_to_f32(rq["S"]) * 16.0)
+    oracle = helpers.make_oracle(wl, weights, M=wl.M)
+    ids = synth.IdSampler(wl).request_ids(0)
+    st = srv.precompute(1, srv.upload_request(rq, B.USER_PROJECTED))
+    want, x = oracle.score(host, helpers.projected_request(wl, rq), ids, return_inputs=True)
+    got = srv.score_ids(st, ids)
+    assert np.isfinite(got).all()
+    # bf16 intermediates of magnitude A carry about 2^-9 A of rounding error: the budget follows the MLP's inputs (about 40)
+    assert np.abs(got - want).max() <= 2e-3 * max(1.0, float(np.abs(x).max()))
+    assert srv.ctx.get_stats().tensor_path == 1 and srv.ctx.poll_status() == 0
+    srv.close()
+
+
 def test_nearline_call_errors():
     wl = helpers.MINI["c1"].with_(name="nearline_err", M=500)
     srv = serving.Server(wl, synth.make_weights(wl), synth.make_item_table(wl))
