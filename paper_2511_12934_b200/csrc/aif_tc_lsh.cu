@@ -149,11 +149,16 @@ template <int D, bool TIERS, bool WIDE>
 __device__ __forceinline__ void lsh_convert(const uint32_t (&sc)[32], float c1, float n_cap, uint32_t p_col, uint32_t (&cnt)[4])
 {
     uint32_t packed[16];
+    // the offset and the rounding multiply-add take two scores per instruction (f32x2)
+    const uint64_t d2 = pack_f32x2((float)D, (float)D), c2 = pack_f32x2(c1, c1), magic2 = pack_f32x2(12582912.0f, 12582912.0f);
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
-        const float p0 = __uint_as_float(sc[i]) + (float)D, p1 = __uint_as_float(sc[i + 1]) + (float)D;   // 2 matches
+        const uint64_t pp = add_f32x2(pack_f32x2(__uint_as_float(sc[i]), __uint_as_float(sc[i + 1])), d2);   // 2 matches
+        float p0, p1;
+        unpack_f32x2(pp, p0, p1);
         if (TIERS) {
-            float w0 = __fmaf_rd(p0, c1, 12582912.0f), w1 = __fmaf_rd(p1, c1, 12582912.0f);
+            float w0, w1;
+            unpack_f32x2(fma_rm_f32x2(pp, c2, magic2), w0, w1);
             if (WIDE) {
                 w0 = fminf(w0, n_cap), w1 = fminf(w1, n_cap);
                 const uint32_t r0 = __float_as_uint(w0) * 0x1111u, r1 = __float_as_uint(w1) * 0x1111u;
