@@ -257,12 +257,110 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
             const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(buf * 256);
             float dot = 0.f;
             const float floor_v = p.linear_out ? -INFINITY : 0.f;
-            if (got && t.cnt > 0) {
+            if (got && t.cnt > 0 && p.epi == EPI_STORE) {
+                // Activations of a hidden layer.  The accumulator is read in the 16x256b shape: a thread then owns two
+                // columns (per group of eight) over four rows, needs eight bias values per 32 columns instead of all 32,
+                // and the bias reads, which every row thread used to repeat, no longer fill the shared memory's return
+                // path.  Three instructions per pair of outputs: bias added to both (f32x2), rounded to bf16, ReLU on
+                // the rounded pair (rounding is monotonic and keeps zero: the same result in either order).
+                const int l4 = lane & 3, r8 = lane >> 2;
+                const __nv_bfloat162 floor2 = __float2bfloat162_rn(floor_v);
+                const int wrow0 = (warp & 3) * 32;
+                for (int c0 = 0; c0 < p.n_cols; c0 += 32) {
+                    uint32_t ra[16], rb[16];
+                    tmem_ld16x256(taddr + (uint32_t)c0, ra);                    // rows 0..15 of this warp's 32
+                    tmem_ld16x256(taddr + (16u << 16) + (uint32_t)c0, rb);      // rows 16..31
+                    uint64_t bias2[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) bias2[j] = *reinterpret_cast<const uint64_t *>(bs + c0 + 8 * j + 2 * l4);
+                    tmem_ld_wait();
+                    // through a staging slab (32 rows x 64 bytes, 64-byte swizzle): the rows of a full slab leave with one
+                    // asynchronous tile store, a ragged slab (last tile of a request or mini-batch) with guarded stores
+                    unsigned char *sb = stg + slab * 2048;
+                    if (lane == 0) bulk_wait_read<C::kSlabs - 1>();   // the store that last read this slab is done with it
+                    __syncwarp();
+                    auto emit = [&](const uint32_t (&r)[16], int row_h) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+#pragma unroll
+                            for (int q = 0; q < 2; ++q) {
+                                float x0, x1;
+                                unpack_f32x2(add_f32x2(pack_f32x2(__uint_as_float(r[4 * j + 2 * q]), __uint_as_float(r[4 * j + 2 * q + 1])), bias2[j]), x0, x1);
+                                const __nv_bfloat162 h = __hmax2(__floats2bfloat162_rn(x0, x1), floor2);
+                                const int rr = row_h + r8 + 8 * q;
+                                *reinterpret_cast<uint32_t *>(sb + rr * 64 + ((j ^ ((rr >> 1) & 3)) << 4) + 4 * l4) = *reinterpret_cast<const uint32_t *>(&h);
+                            }
+                    };
+                    emit(ra, 0);
+                    emit(rb, 16);
+                    if (wrow0 + 32 <= t.cnt) {
+                        fence_proxy_async();
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_2d(&tmapOut, smem_u32(sb), n0 + c0, (int)(t.pos0 + wrow0));
+                            bulk_commit();
+                        }
+                    } else {
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int rr = 8 * j + (lane >> 2), q = lane & 3;
+                            const uint4 v = *reinterpret_cast<const uint4 *>(sb + rr * 64 + ((q ^ ((rr >> 1) & 3)) << 4));
+                            if (wrow0 + rr < t.cnt)
+                                *reinterpret_cast<uint4 *>(p.out + (size_t)(t.pos0 + wrow0 + rr) * p.out_stride + n0 + c0 + q * 8) = v;
+                        }
+                        __syncwarp();
+                    }
+                    slab = (slab + 1u) % (uint32_t)C::kSlabs;
+                }
+            } else if (got && t.cnt > 0 && p.epi == EPI_DOT) {
+                // Last hidden layer: ReLU(x + b) . w_out per row, in the same 16x256b shape (eight bias and eight output
+                // weights per thread and 32 columns).  A thread sums its column pairs for its four rows; the four
+                // threads of a row are joined by shuffles at the end, and the row's own thread takes the result.
+                const int l4 = lane & 3;
+                uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};   // rows r8, r8 + 8, r8 + 16, r8 + 24 (r8 = lane / 4), two columns each
+                for (int c0 = 0; c0 < p.n_cols; c0 += 32) {
+                    uint32_t ra[16], rb[16];
+                    tmem_ld16x256(taddr + (uint32_t)c0, ra);
+                    tmem_ld16x256(taddr + (16u << 16) + (uint32_t)c0, rb);
+                    // the last width may end in the middle of these 32 columns (a multiple of 16): the rest is skipped
+                    const int n_j = (p.n_cols - c0) >> 3;
+                    uint64_t bias2[4], w2[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int col = c0 + 8 * (j < n_j ? j : 0) + 2 * l4;
+                        bias2[j] = *reinterpret_cast<const uint64_t *>(bs + col);
+                        w2[j] = *reinterpret_cast<const uint64_t *>(ws + col);
+                    }
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            if (j >= n_j) continue;   // columns no product wrote
+                            float x0, x1, y0, y1;
+                            unpack_f32x2(add_f32x2(pack_f32x2(__uint_as_float(ra[4 * j + 2 * q]), __uint_as_float(ra[4 * j + 2 * q + 1])), bias2[j]), x0, x1);
+                            unpack_f32x2(add_f32x2(pack_f32x2(__uint_as_float(rb[4 * j + 2 * q]), __uint_as_float(rb[4 * j + 2 * q + 1])), bias2[j]), y0, y1);
+                            acc[q] = fma_f32x2(pack_f32x2(fmaxf(x0, 0.f), fmaxf(x1, 0.f)), w2[j], acc[q]);
+                            acc[2 + q] = fma_f32x2(pack_f32x2(fmaxf(y0, 0.f), fmaxf(y1, 0.f)), w2[j], acc[2 + q]);
+                        }
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float lo, hi;
+                    unpack_f32x2(acc[i], lo, hi);
+                    float v = lo + hi;
+                    v += __shfl_xor_sync(0xffffffffu, v, 1);
+                    v += __shfl_xor_sync(0xffffffffu, v, 2);
+                    // row 8 i + r8 of this warp's 32 belongs to lane 8 i + r8; lane 4 r8 (among others) holds its sum
+                    v = __shfl_sync(0xffffffffu, v, 4 * (lane & 7));
+                    if ((lane >> 3) == i) dot = v;
+                }
+            } else if (got && t.cnt > 0) {
                 for (int c0 = 0; c0 < p.n_cols; c0 += 32) {
                     uint32_t r[32];
                     tmem_ld32(taddr + (uint32_t)c0, r);
                     tmem_ld_wait();
-                    const float4 *b4 = reinterpret_cast<const float4 *>(bs + c0);
                     if (p.epi == EPI_SIGN) {
                         // eq. 5: one bit per output, set where the projection is positive; eight bits per byte, first bit
                         // most significant
@@ -271,61 +369,6 @@ __global__ void __launch_bounds__(LayerCfg<MODE>::kThreads, 1) k_layer_tc(const 
                         for (int i = 0; i < 32; ++i)
                             word |= (__uint_as_float(r[i]) > 0.f ? 1u : 0u) << (8 * (i >> 3) + 7 - (i & 7));
                         if (valid) *reinterpret_cast<uint32_t *>(p.sig_out + (size_t)(t.pos0 + row) * (p.out_stride >> 3) + ((n0 + c0) >> 3)) = word;
-                    } else if (p.epi == EPI_STORE) {
-                        uint32_t packed[16];
-#pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            const float4 bb = b4[q];
-                            const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q]) + bb.x, floor_v),
-                                                                            fmaxf(__uint_as_float(r[4 * q + 1]) + bb.y, floor_v));
-                            const __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q + 2]) + bb.z, floor_v),
-                                                                            fmaxf(__uint_as_float(r[4 * q + 3]) + bb.w, floor_v));
-                            packed[2 * q] = *reinterpret_cast<const uint32_t *>(&h0);
-                            packed[2 * q + 1] = *reinterpret_cast<const uint32_t *>(&h1);
-                        }
-                        // through a staging slab: the rows of a full slab leave with one asynchronous tile store, a
-                        // ragged slab (last tile of a request or mini-batch) with guarded 16-byte stores
-                        unsigned char *sb = stg + slab * 2048;
-                        if (lane == 0) bulk_wait_read<C::kSlabs - 1>();   // the store that last read this slab is done with it
-                        __syncwarp();
-                        const int swz = (lane >> 1) & 3;
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            *reinterpret_cast<uint4 *>(sb + lane * 64 + ((q ^ swz) << 4)) =
-                                make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-                        const int wrow0 = (warp & 3) * 32;
-                        if (wrow0 + 32 <= t.cnt) {
-                            fence_proxy_async();
-                            __syncwarp();
-                            if (lane == 0) {
-                                tma_store_2d(&tmapOut, smem_u32(sb), n0 + c0, (int)(t.pos0 + wrow0));
-                                bulk_commit();
-                            }
-                        } else {
-                            __syncwarp();
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const int rr = 8 * j + (lane >> 2), q = lane & 3;
-                                const uint4 v = *reinterpret_cast<const uint4 *>(sb + rr * 64 + ((q ^ ((rr >> 1) & 3)) << 4));
-                                if (wrow0 + rr < t.cnt)
-                                    *reinterpret_cast<uint4 *>(p.out + (size_t)(t.pos0 + wrow0 + rr) * p.out_stride + n0 + c0 + q * 8) = v;
-                            }
-                            __syncwarp();
-                        }
-                        slab = (slab + 1u) % (uint32_t)C::kSlabs;
-                    } else {
-                        // the last width may end in the middle of these 32 columns (a multiple of 16): the rest is skipped
-                        const float4 *w4 = reinterpret_cast<const float4 *>(ws + c0);
-                        const int n_q = (p.n_cols - c0) >> 2;
-#pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            if (q >= n_q) break;
-                            const float4 bb = b4[q], ww = w4[q];
-                            dot = fmaf(fmaxf(__uint_as_float(r[4 * q]) + bb.x, 0.f), ww.x, dot);
-                            dot = fmaf(fmaxf(__uint_as_float(r[4 * q + 1]) + bb.y, 0.f), ww.y, dot);
-                            dot = fmaf(fmaxf(__uint_as_float(r[4 * q + 2]) + bb.z, 0.f), ww.z, dot);
-                            dot = fmaf(fmaxf(__uint_as_float(r[4 * q + 3]) + bb.w, 0.f), ww.w, dot);
-                        }
                     }
                 }
             }
