@@ -273,6 +273,16 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         : "memory");
 }
 
+// 16 lanes x 16 consecutive 32-bit columns in the 16x128b shape, the store that matches tmem_ld16x256 once two fp32
+// columns have become one packed pair: register k = 2 j + q of lane l goes to row l / 4 + 8 q of the 16 lanes at taddr,
+// column 4 j + l % 4.
+__device__ __forceinline__ void tmem_st16x128(uint32_t taddr, const uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.16x128b.x4.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
+                 "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1, int c2)
 {
     asm volatile(

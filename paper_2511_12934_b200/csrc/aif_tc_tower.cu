@@ -80,6 +80,7 @@ __global__ void __launch_bounds__(kTThreads, 1) k_item_tower_tc(const __grid_con
         if (tid < 128) b1_s[tid] = tid < p.d ? p.b1[tid] : 0.f;
         named_bar_sync(1, 256);
         unsigned char *sb = slabs + warp * 2048;
+        const int l4 = lane & 3, r8 = lane >> 2;
         bool ok = true;
         auto wait = [&](int b, uint32_t parity) {
             const bool got = ok && mbar_wait(bar(b), parity, abort_flag);
@@ -94,31 +95,43 @@ __global__ void __launch_bounds__(kTThreads, 1) k_item_tower_tc(const __grid_con
             tc_fence_after();
             if (!ok) break;
             {
-                uint32_t ra[32], rb[32];
-                auto finish = [&](const uint32_t (&r)[32], int c) {
-                    const float4 *b4 = reinterpret_cast<const float4 *>(b0_s + 32 * c);
-                    uint32_t packed[16];
+                // The accumulator is read in the 16x256b shape (a thread owns two adjacent columns of every eight over
+                // four rows): eight bias values per thread and 32 columns instead of all 32, which every row thread used
+                // to fetch through the shared memory's return path.  The packed pairs go back in the matching 16x128b
+                // shape.  A chunk's pairs land on columns the whole warp has read (its loads are complete before any
+                // of its stores is issued, and the chunk in flight lies further right).
+                uint32_t ra[2][16], rb[2][16];
+                auto fetch = [&](uint32_t (&r)[2][16], int c) {
+                    tmem_ld16x256(col0 + (uint32_t)(32 * c), r[0]);
+                    tmem_ld16x256(col0 + (16u << 16) + (uint32_t)(32 * c), r[1]);
+                };
+                auto finish = [&](const uint32_t (&r)[2][16], int c) {
+                    uint64_t bias2[4];
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const float4 bb = b4[q];
-                        const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q]) + bb.x, 0.f),
-                                                                        fmaxf(__uint_as_float(r[4 * q + 1]) + bb.y, 0.f));
-                        const __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaxf(__uint_as_float(r[4 * q + 2]) + bb.z, 0.f),
-                                                                        fmaxf(__uint_as_float(r[4 * q + 3]) + bb.w, 0.f));
-                        packed[2 * q] = *reinterpret_cast<const uint32_t *>(&h0);
-                        packed[2 * q + 1] = *reinterpret_cast<const uint32_t *>(&h1);
+                    for (int j = 0; j < 4; ++j) bias2[j] = *reinterpret_cast<const uint64_t *>(b0_s + 32 * c + 8 * j + 2 * l4);
+                    const __nv_bfloat162 zero2 = __float2bfloat162_rn(0.f);
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        uint32_t packed[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {   // k = 2 j + q
+                            float x0, x1;
+                            unpack_f32x2(add_f32x2(pack_f32x2(__uint_as_float(r[hh][2 * k]), __uint_as_float(r[hh][2 * k + 1])), bias2[k >> 1]), x0, x1);
+                            const __nv_bfloat162 h = __hmax2(__floats2bfloat162_rn(x0, x1), zero2);   // ReLU on the rounded pair: same result
+                            packed[k] = *reinterpret_cast<const uint32_t *>(&h);
+                        }
+                        tmem_st16x128(col0 + ((uint32_t)(16 * hh) << 16) + (uint32_t)(16 * c), packed);
                     }
-                    tmem_st16(col0 + (uint32_t)(16 * c), packed);
                 };
                 const int nc = p.hI >> 5;   // even
-                tmem_ld32(col0, ra);
+                fetch(ra, 0);
 #pragma unroll 1
                 for (int c = 0; c < nc; c += 2) {
                     tmem_ld_wait();
-                    tmem_ld32(col0 + (uint32_t)(32 * (c + 1)), rb);
+                    fetch(rb, c + 1);
                     finish(ra, c);
                     tmem_ld_wait();
-                    if (c + 2 < nc) tmem_ld32(col0 + (uint32_t)(32 * (c + 2)), ra);
+                    if (c + 2 < nc) fetch(ra, c + 2);
                     finish(rb, c + 1);
                 }
                 tmem_st_wait();
@@ -130,53 +143,64 @@ __global__ void __launch_bounds__(kTThreads, 1) k_item_tower_tc(const __grid_con
             tc_fence_after();
             if (!ok) break;
             const bool whole = row0 + wq * 32 + 32 <= p.n;
-            float ss = 0.f;   // squared norm of this thread's output row
+            // the same shape: rows r8 + 8 i (i = 0..3) of this warp's 32, two columns of every eight; the 32 x 32 block goes
+            // through the staging slab (64-byte swizzle, 4-byte stores, conflict-free) and leaves as one tile store
+            float ss[4] = {0.f, 0.f, 0.f, 0.f};   // this thread's share of the squared norms of its four rows
             for (int c0 = 0; c0 < p.d; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(col0 + (uint32_t)(128 + c0), r);
+                uint32_t r[2][16];
+                tmem_ld16x256(col0 + (uint32_t)(128 + c0), r[0]);
+                tmem_ld16x256(col0 + (16u << 16) + (uint32_t)(128 + c0), r[1]);
+                uint64_t bias2[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) bias2[j] = *reinterpret_cast<const uint64_t *>(b1_s + c0 + 8 * j + 2 * l4);
                 tmem_ld_wait();
                 if (c0 + 32 >= p.d) {   // the accumulators of this pair are in registers: the next pair may overwrite them
                     tc_fence_before();
                     mbar_arrive(bar(TB_TM_FREE));
                 }
-                const float4 *b4 = reinterpret_cast<const float4 *>(b1_s + c0);
-                uint32_t packed[16];
+                if (lane == 0) bulk_wait_read<0>();   // the store that last read the slab is done with it
+                __syncwarp();
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float4 bb = b4[q];
-                    const float x0 = __uint_as_float(r[4 * q]) + bb.x, x1 = __uint_as_float(r[4 * q + 1]) + bb.y;
-                    const float x2 = __uint_as_float(r[4 * q + 2]) + bb.z, x3 = __uint_as_float(r[4 * q + 3]) + bb.w;
-                    ss = fmaf(x0, x0, fmaf(x1, x1, fmaf(x2, x2, fmaf(x3, x3, ss))));
-                    const __nv_bfloat162 h0 = __floats2bfloat162_rn(x0, x1);
-                    const __nv_bfloat162 h1 = __floats2bfloat162_rn(x2, x3);
-                    packed[2 * q] = *reinterpret_cast<const uint32_t *>(&h0);
-                    packed[2 * q + 1] = *reinterpret_cast<const uint32_t *>(&h1);
-                }
+                for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {   // k = 2 j + q
+                        float x0, x1;
+                        unpack_f32x2(add_f32x2(pack_f32x2(__uint_as_float(r[hh][2 * k]), __uint_as_float(r[hh][2 * k + 1])), bias2[k >> 1]), x0, x1);
+                        ss[2 * hh + (k & 1)] = fmaf(x0, x0, fmaf(x1, x1, ss[2 * hh + (k & 1)]));
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+                        const int rr = 16 * hh + r8 + 8 * (k & 1), j = k >> 1;
+                        *reinterpret_cast<uint32_t *>(sb + rr * 64 + ((j ^ ((rr >> 1) & 3)) << 4) + 4 * l4) = *reinterpret_cast<const uint32_t *>(&h);
+                    }
                 if (whole) {
-                    if (lane == 0) bulk_wait_read<0>();   // the store that last read the slab is done with it
-                    __syncwarp();
-                    const int swz = (lane >> 1) & 3;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4 *>(sb + lane * 64 + ((q ^ swz) << 4)) =
-                            make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
                     fence_proxy_async();
                     __syncwarp();
                     if (lane == 0) {
                         tma_store_2d(&tmapOut, smem_u32(sb), c0, (int)(row0 + wq * 32));
                         bulk_commit();
                     }
-                } else if (row0 + row < p.n) {
-                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + (size_t)(row0 + row) * p.d + c0);
+                } else {
+                    __syncwarp();
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                    for (int j = 0; j < 4; ++j) {
+                        const int rr = 8 * j + (lane >> 2), q = lane & 3;
+                        const uint4 v = *reinterpret_cast<const uint4 *>(sb + rr * 64 + ((q ^ ((rr >> 1) & 3)) << 4));
+                        if (row0 + wq * 32 + rr < p.n) *reinterpret_cast<uint4 *>(p.out + (size_t)(row0 + wq * 32 + rr) * p.d + c0 + q * 8) = v;
+                    }
+                    __syncwarp();
                 }
             }
             if (p.norm_max) {
                 // non-negative floats order like their bit patterns; a NaN row gives a pattern above every finite one
-                const int bits = row0 + row < p.n ? (__float_as_int(sqrtf(ss) * 1.00390625f) & 0x7fffffff) : 0;
-                const int best = __reduce_max_sync(0xffffffffu, bits);
+                int best = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float v = ss[i];
+                    v += __shfl_xor_sync(0xffffffffu, v, 1);
+                    v += __shfl_xor_sync(0xffffffffu, v, 2);
+                    const int rr = 16 * (i >> 1) + r8 + 8 * (i & 1);
+                    if (row0 + wq * 32 + rr < p.n) best = max(best, __float_as_int(sqrtf(v) * 1.00390625f) & 0x7fffffff);
+                }
+                best = __reduce_max_sync(0xffffffffu, best);
                 if (lane == 0 && best > 0) atomicMax(reinterpret_cast<int *>(p.norm_max), best);
             }
         }
